@@ -1,0 +1,416 @@
+/*
+ * qblora_oracle.c -- TEST INFRASTRUCTURE, NOT PRODUCT CODE.
+ *
+ * A plain, slow, fp64 CPU statement of the adapted quantized linear layer of
+ * Q-BLoRA / QA-BLoRA (arXiv 2407.17029).  It exists only so that tests, the
+ * smoke check and the benchmark's CPU-baseline leg can compare the GPU library
+ * against something written directly from the paper's definitions.  It shares
+ * no code, header, table or helper with the CUDA library and the library never
+ * calls it.
+ *
+ * Conventions (storage): the paper writes W as D_in x D_out and y = W^T x
+ * (Sec. 3.1).  Here the weight is stored row-major as Ws[o][i] = W[i][o], so a
+ * row is one output feature and D_in is contiguous.  T = number of tokens.
+ *   P = D_in / lambda1, Q = D_out / lambda2, r = adapter inner dimension
+ *   (the paper's lambda * D_rank, Sec. 3.2).
+ * Every routine is the written-out definition: no blocking, no fusion.
+ *
+ * Pins (see tests/test_oracle_*.py): quantizer closed forms, round trip and
+ * brute force; B = 0; lambda = 1 textbook LoRA; dense equivalent-weight
+ * identity (Eq. 2 and the paragraph after it); finite differences and adjoint
+ * identity for the backward pass; merge identity (Sec. 3.3).
+ * Parity unpinned: only two *conventions* -- the choice of the built-in 16-level
+ * table (the paper cites NF4 without printing it) and which (lambda1, lambda2)
+ * a benchmark config means.  Everything computed downstream of them is pinned.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORC_OK 0
+#define ORC_BAD 1
+
+/* one IEEE binary32 operation, emulated through binary64 (53 >= 2*24+2, so the
+ * double rounding is innocuous for a single +,-,*,/). */
+static float f32_sub(float a, float b) { return (float)((double)a - (double)b); }
+static float f32_div(float a, float b) { return (float)((double)a / (double)b); }
+
+/* ---- standard normal quantile by bisection on erfc ---------------------- */
+static double norm_cdf(double x) { return 0.5 * erfc(-x / sqrt(2.0)); }
+static double norm_ppf(double p) {
+  double lo = -12.0, hi = 12.0;
+  for (int it = 0; it < 200; ++it) {
+    double mid = 0.5 * (lo + hi);
+    if (norm_cdf(mid) < p) lo = mid; else hi = mid;
+  }
+  return 0.5 * (lo + hi);
+}
+
+/*
+ * Built-in 16-level table used when a caller supplies none.  Sec. 3.2 says the
+ * base model is compressed with a 4-bit normal-quantile data type but prints no
+ * values, so the table is data in the interface; this default is a closed form
+ * of this project: nine non-negative levels ppf(1/2 + j/17)/ppf(1/2 + 8/17),
+ * j = 0..8, and seven negative levels -ppf(1/2 + j/15)/ppf(1/2 + 7/15),
+ * j = 1..7, sorted ascending, evaluated in fp64 and rounded once to fp32.
+ */
+int orc_default_code_table(float out[16]) {
+  double pos_den = norm_ppf(0.5 + 8.0 / 17.0);
+  double neg_den = norm_ppf(0.5 + 7.0 / 15.0);
+  for (int j = 1; j <= 7; ++j)
+    out[7 - j] = (float)(-norm_ppf(0.5 + (double)j / 15.0) / neg_den);
+  for (int j = 0; j <= 8; ++j)
+    out[7 + j] = (float)(norm_ppf(0.5 + (double)j / 17.0) / pos_den);
+  out[7] = 0.0f;
+  out[0] = -1.0f;
+  out[15] = 1.0f;
+  return ORC_OK;
+}
+
+/* ---- block-wise 4-bit quantizer (Eq. 1) --------------------------------- */
+static void set_code(uint8_t* codes, int d_in, int o, int i, int c) {
+  size_t byte = (size_t)o * (size_t)(d_in / 2) + (size_t)(i / 2);
+  if (i & 1) codes[byte] = (uint8_t)((codes[byte] & 0x0F) | (c << 4));
+  else       codes[byte] = (uint8_t)((codes[byte] & 0xF0) | c);
+}
+static int get_code(const uint8_t* codes, int d_in, int o, int i) {
+  uint8_t b = codes[(size_t)o * (size_t)(d_in / 2) + (size_t)(i / 2)];
+  return (i & 1) ? (b >> 4) : (b & 0x0F);
+}
+
+/*
+ * qfmt 0 (code table, absmax): alpha = max|w| over the block, beta absent;
+ *   code = number of midpoints between adjacent levels that fl32(w/alpha)
+ *   exceeds (nearest level, ties to the lower index).  Eq. 1's absmax variant
+ *   read with the level table in place of the integer grid.
+ * qfmt 1 (min-max, Eq. 1 with N = 4): beta = min, alpha = fl32(fl32(max-min)/15),
+ *   code = clamp(round-half-even(fl32(fl32(w-beta)/alpha)), 0, 15).
+ * A block is block_out consecutive rows by block_in consecutive columns.
+ * Degenerate block (alpha = 0): qfmt 0 -> every code is the level-0.0 index
+ * (or nearest-to-zero level); qfmt 1 -> every code 0, so w~ = beta exactly.
+ */
+int orc_quantize_blockwise(const float* W, int d_out, int d_in, int block_in,
+                           int block_out, int qfmt, const float* code,
+                           uint8_t* codes, float* alpha, float* beta) {
+  if (d_in % 2 || d_in % block_in || d_out % block_out) return ORC_BAD;
+  int G = d_in / block_in, R = d_out / block_out;
+  float mid[15];
+  int zero_idx = 0;
+  if (qfmt == 0) {
+    for (int j = 0; j < 15; ++j)
+      mid[j] = (float)(((double)code[j] + (double)code[j + 1]) / 2.0);
+    for (int j = 1; j < 16; ++j)
+      if (fabs((double)code[j]) < fabs((double)code[zero_idx])) zero_idx = j;
+  }
+  memset(codes, 0, (size_t)d_out * (size_t)(d_in / 2));
+#pragma omp parallel for schedule(static)
+  for (int rb = 0; rb < R; ++rb) {
+    for (int gb = 0; gb < G; ++gb) {
+      int o0 = rb * block_out, i0 = gb * block_in;
+      float wmin = W[(size_t)o0 * d_in + i0], wmax = wmin, amax = 0.0f;
+      for (int o = o0; o < o0 + block_out; ++o)
+        for (int i = i0; i < i0 + block_in; ++i) {
+          float w = W[(size_t)o * d_in + i];
+          if (w < wmin) wmin = w;
+          if (w > wmax) wmax = w;
+          float a = (float)fabs((double)w);
+          if (a > amax) amax = a;
+        }
+      size_t bi = (size_t)rb * G + gb;
+      if (qfmt == 0) {
+        alpha[bi] = amax;
+        for (int o = o0; o < o0 + block_out; ++o)
+          for (int i = i0; i < i0 + block_in; ++i) {
+            int c = zero_idx;
+            if (amax != 0.0f) {
+              float v = f32_div(W[(size_t)o * d_in + i], amax);
+              c = 0;
+              for (int j = 0; j < 15; ++j) if (v > mid[j]) ++c;
+            }
+            set_code(codes, d_in, o, i, c);
+          }
+      } else {
+        float d = f32_sub(wmax, wmin);
+        float a = f32_div(d, 15.0f);
+        int degenerate = (d == 0.0f) || (a == 0.0f);
+        beta[bi] = wmin;
+        alpha[bi] = degenerate ? 0.0f : a;
+        for (int o = o0; o < o0 + block_out; ++o)
+          for (int i = i0; i < i0 + block_in; ++i) {
+            int c = 0;
+            if (!degenerate) {
+              float q = f32_div(f32_sub(W[(size_t)o * d_in + i], wmin), a);
+              double rq = nearbyint((double)q); /* default mode: half to even */
+              if (rq < 0.0) rq = 0.0;
+              if (rq > 15.0) rq = 15.0;
+              c = (int)rq;
+            }
+            set_code(codes, d_in, o, i, c);
+          }
+      }
+    }
+  }
+  return ORC_OK;
+}
+
+/* w~[o][i] = alpha * level + beta with the block's (alpha, beta); level = table
+ * entry (qfmt 0, beta = 0) or the integer code (qfmt 1).  Eq. 1, left equality. */
+int orc_dequantize(const uint8_t* codes, const float* alpha, const float* beta,
+                   int d_out, int d_in, int block_in, int block_out, int qfmt,
+                   const float* code, double* Wt) {
+  if (d_in % 2 || d_in % block_in || d_out % block_out) return ORC_BAD;
+  int G = d_in / block_in;
+#pragma omp parallel for schedule(static)
+  for (int o = 0; o < d_out; ++o)
+    for (int i = 0; i < d_in; ++i) {
+      size_t bi = (size_t)(o / block_out) * G + (size_t)(i / block_in);
+      int c = get_code(codes, d_in, o, i);
+      double level = (qfmt == 0) ? (double)code[c] : (double)c;
+      double b = (qfmt == 0) ? 0.0 : (double)beta[bi];
+      Wt[(size_t)o * d_in + i] = (double)alpha[bi] * level + b;
+    }
+  return ORC_OK;
+}
+
+/* AvgPool(lambda1) over the feature axis (Sec. 3.2; written out before Eq. 2). */
+static void pool_rows(const float* X, int64_t T, int d_in, int l1, double* xp) {
+  int P = d_in / l1;
+#pragma omp parallel for schedule(static)
+  for (int64_t t = 0; t < T; ++t)
+    for (int p = 0; p < P; ++p) {
+      double s = 0.0;
+      for (int j = 0; j < l1; ++j) s += (double)X[t * d_in + (int64_t)p * l1 + j];
+      xp[t * P + p] = s / (double)l1;
+    }
+}
+
+/*
+ * Forward (Sec. 3.1 combined formula with the Sec. 3.2 adapter):
+ *   Y[t][o] = sum_i X[t][i] w~[o][i]
+ *           + s * v[t][o / lambda2],   v = (x' A) B,   x' = AvgPool_lambda1(X)
+ * The scaling s multiplies the adapter term only; repeat_interleave(lambda2)
+ * is the index o / lambda2.  With B == NULL, A is the single matrix H of
+ * Sec. 3.3 (shape [P][Q]) and v = x' H.  has_adapter == 0: base term only.
+ */
+int orc_linear_fwd(const double* Wt, int d_out, int d_in, const float* X,
+                   int64_t T, int has_adapter, int l1, int l2, int r, double s,
+                   const float* A, const float* B, double* Y) {
+  int P = 0, Q = 0;
+  double *xp = NULL, *u = NULL, *v = NULL;
+  if (has_adapter) {
+    if (d_in % l1 || d_out % l2) return ORC_BAD;
+    P = d_in / l1; Q = d_out / l2;
+    xp = (double*)malloc(sizeof(double) * (size_t)T * P);
+    v = (double*)calloc((size_t)T * Q, sizeof(double));
+    pool_rows(X, T, d_in, l1, xp);
+    if (B) {
+      u = (double*)calloc((size_t)T * r, sizeof(double));
+#pragma omp parallel for schedule(static)
+      for (int64_t t = 0; t < T; ++t) {
+        for (int k = 0; k < r; ++k) {
+          double acc = 0.0;
+          for (int p = 0; p < P; ++p) acc += xp[t * P + p] * (double)A[(size_t)p * r + k];
+          u[t * r + k] = acc;
+        }
+        for (int q = 0; q < Q; ++q) {
+          double acc = 0.0;
+          for (int k = 0; k < r; ++k) acc += u[t * r + k] * (double)B[(size_t)k * Q + q];
+          v[t * Q + q] = acc;
+        }
+      }
+    } else {
+#pragma omp parallel for schedule(static)
+      for (int64_t t = 0; t < T; ++t)
+        for (int q = 0; q < Q; ++q) {
+          double acc = 0.0;
+          for (int p = 0; p < P; ++p) acc += xp[t * P + p] * (double)A[(size_t)p * Q + q];
+          v[t * Q + q] = acc;
+        }
+    }
+  }
+#pragma omp parallel for schedule(static)
+  for (int o = 0; o < d_out; ++o)
+    for (int64_t t = 0; t < T; ++t) {
+      double acc = 0.0;
+      for (int i = 0; i < d_in; ++i)
+        acc += (double)X[t * d_in + i] * Wt[(size_t)o * d_in + i];
+      if (has_adapter) acc += s * v[t * Q + o / l2];
+      Y[t * d_out + o] = acc;
+    }
+  free(xp); free(u); free(v);
+  return ORC_OK;
+}
+
+/*
+ * Backward, obtained by differentiating the forward formula above with the
+ * base weight frozen (Sec. 3.1: only A and B are updated):
+ *   dv[t][q] = s * sum_{j<lambda2} dY[t][lambda2 q + j]
+ *   du = dv B^T,  dB = u^T dv,  dx' = du A^T,  dA = x'^T du
+ *   dX[t][i] = sum_o dY[t][o] w~[o][i] + dx'[t][i / lambda1] / lambda1
+ * Single-matrix mode (B == NULL): dA receives dH = x'^T dv and dx' = dv H^T.
+ * Any of dX, dA, dB may be NULL (skipped).  Wt may be NULL when dX is NULL.
+ */
+int orc_linear_bwd(const double* Wt, int d_out, int d_in, const float* X,
+                   const float* dY, int64_t T, int has_adapter, int l1, int l2,
+                   int r, double s, const float* A, const float* B, double* dX,
+                   double* dA, double* dB) {
+  int P = 0, Q = 0;
+  double *xp = NULL, *u = NULL, *dv = NULL, *du = NULL, *dxp = NULL;
+  if (has_adapter) {
+    if (d_in % l1 || d_out % l2) return ORC_BAD;
+    P = d_in / l1; Q = d_out / l2;
+    xp = (double*)malloc(sizeof(double) * (size_t)T * P);
+    dv = (double*)malloc(sizeof(double) * (size_t)T * Q);
+    dxp = (double*)calloc((size_t)T * P, sizeof(double));
+    pool_rows(X, T, d_in, l1, xp);
+#pragma omp parallel for schedule(static)
+    for (int64_t t = 0; t < T; ++t)
+      for (int q = 0; q < Q; ++q) {
+        double acc = 0.0;
+        for (int j = 0; j < l2; ++j) acc += (double)dY[t * d_out + (int64_t)q * l2 + j];
+        dv[t * Q + q] = s * acc;
+      }
+    if (B) {
+      u = (double*)malloc(sizeof(double) * (size_t)T * r);
+      du = (double*)malloc(sizeof(double) * (size_t)T * r);
+#pragma omp parallel for schedule(static)
+      for (int64_t t = 0; t < T; ++t) {
+        for (int k = 0; k < r; ++k) {
+          double a1 = 0.0, a2 = 0.0;
+          for (int p = 0; p < P; ++p) a1 += xp[t * P + p] * (double)A[(size_t)p * r + k];
+          for (int q = 0; q < Q; ++q) a2 += dv[t * Q + q] * (double)B[(size_t)k * Q + q];
+          u[t * r + k] = a1;
+          du[t * r + k] = a2;
+        }
+        for (int p = 0; p < P; ++p) {
+          double acc = 0.0;
+          for (int k = 0; k < r; ++k) acc += du[t * r + k] * (double)A[(size_t)p * r + k];
+          dxp[t * P + p] = acc;
+        }
+      }
+      if (dB) {
+#pragma omp parallel for schedule(static)
+        for (int k = 0; k < r; ++k)
+          for (int q = 0; q < Q; ++q) {
+            double acc = 0.0;
+            for (int64_t t = 0; t < T; ++t) acc += u[t * r + k] * dv[t * Q + q];
+            dB[(size_t)k * Q + q] = acc;
+          }
+      }
+      if (dA) {
+#pragma omp parallel for schedule(static)
+        for (int p = 0; p < P; ++p)
+          for (int k = 0; k < r; ++k) {
+            double acc = 0.0;
+            for (int64_t t = 0; t < T; ++t) acc += xp[t * P + p] * du[t * r + k];
+            dA[(size_t)p * r + k] = acc;
+          }
+      }
+    } else {
+#pragma omp parallel for schedule(static)
+      for (int64_t t = 0; t < T; ++t)
+        for (int p = 0; p < P; ++p) {
+          double acc = 0.0;
+          for (int q = 0; q < Q; ++q) acc += dv[t * Q + q] * (double)A[(size_t)p * Q + q];
+          dxp[t * P + p] = acc;
+        }
+      if (dA) {
+#pragma omp parallel for schedule(static)
+        for (int p = 0; p < P; ++p)
+          for (int q = 0; q < Q; ++q) {
+            double acc = 0.0;
+            for (int64_t t = 0; t < T; ++t) acc += xp[t * P + p] * dv[t * Q + q];
+            dA[(size_t)p * Q + q] = acc;
+          }
+      }
+    }
+  }
+  if (dX) {
+    if (!Wt) return ORC_BAD;
+#pragma omp parallel for schedule(static)
+    for (int64_t t = 0; t < T; ++t)
+      for (int i = 0; i < d_in; ++i) {
+        double acc = 0.0;
+        for (int o = 0; o < d_out; ++o)
+          acc += (double)dY[t * d_out + o] * Wt[(size_t)o * d_in + i];
+        if (has_adapter) acc += dxp[t * P + i / l1] / (double)l1;
+        dX[t * d_in + i] = acc;
+      }
+  }
+  free(xp); free(u); free(dv); free(du); free(dxp);
+  return ORC_OK;
+}
+
+/*
+ * Equivalent dense weight update (paragraph after Eq. 2): in storage order
+ *   dW[o][i] = (A B)[i / lambda1][o / lambda2] / lambda1
+ * i.e. constant on every aligned (lambda1 x lambda2) tile; the 1/lambda1 comes
+ * from the averaging (Eq. 2's condition w_in = lambda1 * w).  B == NULL: A is H.
+ */
+int orc_dense_delta_w(int d_out, int d_in, int l1, int l2, int r,
+                      const float* A, const float* B, double* dW) {
+  if (d_in % l1 || d_out % l2) return ORC_BAD;
+  int P = d_in / l1, Q = d_out / l2;
+  double* H = (double*)malloc(sizeof(double) * (size_t)P * Q);
+  for (int p = 0; p < P; ++p)
+    for (int q = 0; q < Q; ++q) {
+      double acc = 0.0;
+      if (B) for (int k = 0; k < r; ++k) acc += (double)A[(size_t)p * r + k] * (double)B[(size_t)k * Q + q];
+      else acc = (double)A[(size_t)p * Q + q];
+      H[(size_t)p * Q + q] = acc;
+    }
+  for (int o = 0; o < d_out; ++o)
+    for (int i = 0; i < d_in; ++i)
+      dW[(size_t)o * d_in + i] = H[(size_t)(i / l1) * Q + (o / l2)] / (double)l1;
+  free(H);
+  return ORC_OK;
+}
+
+/*
+ * QA-BLoRA merge (Sec. 3.3, the new-beta routine of Algorithm 2): when every
+ * quantization block lies inside one (lambda1 x lambda2) tile of the dense
+ * update, the update is a shift of that block's beta:
+ *   beta'[block] = beta[block] + s * (A B)[i0 / lambda1][o0 / lambda2] / lambda1
+ * with (o0, i0) the block's first element.  Evaluated in fp64, rounded once to
+ * fp32.  Codes and alpha are untouched.  Returns ORC_BAD when a block would
+ * straddle two tiles (lambda1 % block_in or lambda2 % block_out non-zero).
+ */
+int orc_merge(const float* beta, int d_out, int d_in, int block_in,
+              int block_out, int l1, int l2, int r, double s, const float* A,
+              const float* B, float* beta_out) {
+  if (d_in % l1 || d_out % l2 || d_in % block_in || d_out % block_out) return ORC_BAD;
+  if (l1 % block_in || l2 % block_out) return ORC_BAD;
+  int G = d_in / block_in, R = d_out / block_out, Q = d_out / l2;
+#pragma omp parallel for schedule(static)
+  for (int rb = 0; rb < R; ++rb)
+    for (int gb = 0; gb < G; ++gb) {
+      int p = (gb * block_in) / l1, q = (rb * block_out) / l2;
+      double h = 0.0;
+      if (B) for (int k = 0; k < r; ++k) h += (double)A[(size_t)p * r + k] * (double)B[(size_t)k * Q + q];
+      else h = (double)A[(size_t)p * Q + q];
+      size_t bi = (size_t)rb * G + gb;
+      beta_out[bi] = (float)((double)beta[bi] + s * h / (double)l1);
+    }
+  return ORC_OK;
+}
+
+/* Low-bit inference product: Y[t][o] = sum_i X[t][i] (alpha c + beta')[o][i]
+ * (Sec. 3.3: the merged model is used directly at low precision). */
+int orc_lowbit_gemm(const uint8_t* codes, const float* alpha, const float* beta,
+                    int d_out, int d_in, int block_in, int block_out,
+                    const float* X, int64_t T, double* Y) {
+  double* Wt = (double*)malloc(sizeof(double) * (size_t)d_out * d_in);
+  if (!Wt) return ORC_BAD;
+  int rc = orc_dequantize(codes, alpha, beta, d_out, d_in, block_in, block_out, 1, NULL, Wt);
+  if (rc == ORC_OK) rc = orc_linear_fwd(Wt, d_out, d_in, X, T, 0, 1, 1, 0, 0.0, NULL, NULL, Y);
+  free(Wt);
+  return rc;
+}
+
+#ifdef _OPENMP
+#include <omp.h>
+int orc_num_threads(void) { return omp_get_max_threads(); }
+#else
+int orc_num_threads(void) { return 1; }
+#endif
