@@ -1,0 +1,176 @@
+/*
+ * qblora.h -- C ABI of the B200 (sm_100a) adapted quantized linear layer of
+ * Q-BLoRA / QA-BLoRA (arXiv 2407.17029).
+ *
+ * Notation.  The paper writes the base weight W as D_in x D_out with y = W^T x
+ * (Sec. 3.1).  This library stores it row-major as W_s[o][i] = W[i][o]
+ * ("[out][in]", D_in contiguous).  T = tokens, g = block_in, G = D_in / g,
+ * P = D_in / lambda_in, Q = D_out / lambda_out, r = adapter inner dimension
+ * (the paper's lambda * D_rank, Sec. 3.2).
+ *
+ * Ownership.  Every pointer in a struct or argument list marked DEVICE is a
+ * CUDA device pointer owned by the caller, 16-byte aligned; the library never
+ * allocates or frees device memory in these calls, keeps no per-call state, and
+ * only enqueues work on the given stream (a cudaStream_t passed as void*,
+ * NULL = default stream).  Pointers marked HOST are ordinary host memory read
+ * during the call.  Scratch memory is the caller's `ws` buffer of at least
+ * qblora_workspace_bytes(...) bytes; its contents are undefined after a call.
+ *
+ * Errors.  Every call returns a qblora_status; nothing throws or aborts.
+ * Argument checks are made on the host before any launch.  Device-side waits
+ * are bounded: a kernel that gives up stores QBLORA_ERR_TIMEOUT into the first
+ * word of `ws`, which qblora_device_status() reads back.
+ *
+ * Determinism.  No floating-point atomics: equal inputs give bit-equal outputs.
+ */
+#ifndef QBLORA_H_
+#define QBLORA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  QBLORA_OK = 0,
+  QBLORA_ERR_INVALID_ARG = 1, /* null / misaligned pointer, sizes that do not divide, tokens < 1 */
+  QBLORA_ERR_UNSUPPORTED = 2, /* valid request this build has no kernel for */
+  QBLORA_ERR_WORKSPACE = 3,   /* ws == NULL or ws_bytes too small */
+  QBLORA_ERR_CUDA = 4,        /* a CUDA runtime call or launch failed */
+  QBLORA_ERR_TIMEOUT = 5      /* a bounded device-side wait gave up (see qblora_device_status) */
+} qblora_status;
+
+typedef enum {
+  /* w~ = alpha * code[c]; alpha = max|w| of the block, no beta.  Sec. 3.2 (the 4-bit
+   * normal-quantile base format of Q-BLoRA) with Eq. 1's absmax scaling. */
+  QBLORA_FMT_CODEBOOK_ABSMAX = 0,
+  /* w~ = alpha * c + beta; alpha = (max - min) / 15, beta = min.  Eq. 1, min-max, N = 4
+   * (the format QA-BLoRA merges into, Sec. 3.3). */
+  QBLORA_FMT_AFFINE_MINMAX = 1
+} qblora_qfmt;
+
+typedef enum { QBLORA_F32 = 0, QBLORA_BF16 = 1 } qblora_dtype;
+
+typedef enum {
+  QBLORA_OP_QUANTIZE = 0,
+  QBLORA_OP_LINEAR_FWD = 1,
+  QBLORA_OP_LINEAR_BWD = 2,
+  QBLORA_OP_MERGE = 3,
+  QBLORA_OP_LOWBIT_GEMM = 4
+} qblora_op;
+
+/* Frozen block-wise 4-bit weight: the triplet (w^, alpha, beta) of Eq. 1 / Sec. 3.3. */
+typedef struct {
+  int32_t d_in, d_out;         /* paper D_in, D_out */
+  int32_t block_in, block_out; /* quantization block: block_out rows x block_in columns of W_s */
+  int32_t qfmt;                /* qblora_qfmt */
+  float code[16];              /* HOST values, ascending; level table (code-table format only) */
+  const uint8_t* codes;        /* DEVICE [d_out][d_in/2]; byte k of row o: low nibble = code(o,2k),
+                                  high nibble = code(o,2k+1) */
+  const float* alpha;          /* DEVICE [d_out/block_out][d_in/block_in] */
+  const float* beta;           /* DEVICE same shape; NULL for the code-table format */
+} qblora_qweight;
+
+/* Balanced low-rank adapter (Sec. 3.2): x' = AvgPool_{lambda_in}(x), y' = (A B)^T x',
+ * y_adapter = scaling * repeat_interleave_{lambda_out}(y'). */
+typedef struct {
+  int32_t lambda_in, lambda_out; /* lambda_1 (input pooling), lambda_2 (output repeat) */
+  int32_t rank;                  /* r */
+  float scaling;                 /* s; multiplies the adapter term only */
+  const void* A;                 /* DEVICE bf16 [P][r] */
+  const void* B;                 /* DEVICE bf16 [r][Q]; NULL => A is the single matrix H, bf16 [P][Q],
+                                    of Sec. 3.3 / Algorithm 2 (accepted by qablora_merge only) */
+} qblora_adapter;
+
+/* Writes the built-in 16-level table (HOST out): nine non-negative levels
+ * ppf(1/2 + j/17) / ppf(1/2 + 8/17), j = 0..8, and seven negative levels
+ * -ppf(1/2 + j/15) / ppf(1/2 + 7/15), j = 1..7 (ppf = standard normal quantile), ascending,
+ * rounded to fp32.  The paper (Sec. 3.2) names a 4-bit normal-quantile type without printing its
+ * values; callers that hold another table pass it in qblora_qweight.code instead. */
+int qblora_default_code_table(float out[16]);
+
+/* Scratch bytes needed by `op` for this weight / adapter / token count (0 if none).
+ * adapter may be NULL.  Returns 0 for invalid arguments as well; the op itself reports those. */
+size_t qblora_workspace_bytes(int op, const qblora_qweight* qw, const qblora_adapter* adapter,
+                              int64_t tokens);
+
+const char* qblora_status_string(int status);
+
+/* Synchronises `stream` and returns the status word the last call using `ws` left there
+ * (QBLORA_OK, or QBLORA_ERR_TIMEOUT if a kernel's bounded wait expired). */
+int qblora_device_status(const void* ws, void* stream);
+
+/*
+ * Block-wise 4-bit quantization, Eq. 1 (Sec. 3.1).
+ *   W       DEVICE [d_out][d_in], fp32 or bf16 (w_dtype); bf16 is promoted exactly.
+ *   code    HOST level table (code-table format; ignored for min-max).
+ *   codes   DEVICE out, uint8 [d_out][d_in/2];  alpha DEVICE out fp32 [d_out/block_out][d_in/block_in];
+ *   beta    DEVICE out, same shape (min-max format); must be NULL for the code-table format.
+ * Arithmetic is IEEE fp32, one rounding per operation, so the result is unique:
+ *   code table: alpha = max|w|; v = w / alpha; code = #{ j : v > fl32((code[j]+code[j+1])/2) }
+ *               (nearest level, ties to the lower index); all-zero block: alpha = 0, code = level 0.0.
+ *   min-max:    beta = min; alpha = (max - min) / 15; code = clamp(rint((w - beta) / alpha), 0, 15),
+ *               ties to even; constant block: alpha = 0, code = 0.
+ * Requires d_in % block_in == 0, d_out % block_out == 0, d_in even.
+ */
+int qblora_quantize_blockwise(const void* W, int w_dtype, int32_t d_out, int32_t d_in,
+                              int32_t block_in, int32_t block_out, int32_t qfmt,
+                              const float code[16], uint8_t* codes, float* alpha, float* beta,
+                              void* stream);
+
+/*
+ * Forward of the adapted quantized linear (Sec. 3.1 combined formula with the Sec. 3.2 adapter;
+ * Algorithm 1's forward read as its prose):
+ *   Y[t][o] = sum_i X[t][i] * w~[o][i]  +  s * ((x' A) B)[t][o / lambda_out],
+ *   x'[t][p] = (1 / lambda_in) * sum_{j < lambda_in} X[t][lambda_in * p + j].
+ * The base weight is dequantized inside the kernel; no dense copy of it is written.
+ *   X DEVICE bf16 [tokens][d_in];  Y DEVICE out [tokens][d_out], y_dtype BF16 or F32 (F32 = the
+ *   accumulator before the final rounding).  adapter may be NULL (base term only).
+ */
+int qblora_linear_fwd(const qblora_qweight* qw, const qblora_adapter* adapter, const void* X,
+                      int64_t tokens, void* Y, int y_dtype, void* ws, size_t ws_bytes,
+                      void* stream);
+
+/*
+ * Backward of the same layer with the base weight frozen (Sec. 3.1: only A and B are trained);
+ * the paper leaves it to automatic differentiation, so it is the derivative of the forward above:
+ *   dv[t][q] = s * sum_{j < lambda_out} dY[t][lambda_out * q + j];   du = dv B^T;
+ *   dB = u^T dv  (u = x' A, recomputed from X);   dA = x'^T du;
+ *   dX[t][i] = sum_o dY[t][o] * w~[o][i]  +  (du A^T)[t][i / lambda_in] / lambda_in.
+ *   dY DEVICE bf16 [tokens][d_out];  dX DEVICE out [tokens][d_in] (dx_dtype BF16 or F32);
+ *   dA DEVICE out fp32 [P][r];  dB DEVICE out fp32 [r][Q].  Any of dX, dA, dB may be NULL (skipped).
+ *   adapter may be NULL (then dA and dB must be NULL).
+ */
+int qblora_linear_bwd(const qblora_qweight* qw, const qblora_adapter* adapter, const void* X,
+                      const void* dY, int64_t tokens, void* dX, int dx_dtype, float* dA, float* dB,
+                      void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * QA-BLoRA merge (Sec. 3.3; Algorithm 2's new-beta routine): the adapter's equivalent dense
+ * update is constant on (lambda_in x lambda_out) tiles (paragraph after Eq. 2), so when every
+ * quantization block lies inside one tile it is a shift of that block's beta:
+ *   beta'[o/block_out][i/block_in] = beta + s * (A B)[i0 / lambda_in][o0 / lambda_out] / lambda_in.
+ * qw must be in the min-max format; codes and alpha are not touched.  beta_out DEVICE fp32, same
+ * shape as beta, may alias qw->beta.  Evaluated in fp64 and rounded once to fp32.
+ * Requires lambda_in % block_in == 0 and lambda_out % block_out == 0, else QBLORA_ERR_INVALID_ARG.
+ * adapter->B == NULL: A is H [P][Q].
+ */
+int qablora_merge(const qblora_qweight* qw, const qblora_adapter* adapter, float* beta_out,
+                  void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Low-precision inference product on the merged model (Sec. 3.3):
+ *   Y[t][o] = sum_i X[t][i] * (alpha[o][i/g] * c[o][i] + beta'[o][i/g]).
+ * qw: min-max format.  X DEVICE bf16 [tokens][d_in];  Y DEVICE out [tokens][d_out], BF16 or F32.
+ * Small token counts stream the packed weight once (bandwidth-bound); large ones use the same
+ * tensor-core mainloop as qblora_linear_fwd.
+ */
+int qablora_lowbit_gemm(const qblora_qweight* qw, const void* X, int64_t tokens, void* Y,
+                        int y_dtype, void* ws, size_t ws_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QBLORA_H_ */

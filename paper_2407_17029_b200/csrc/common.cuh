@@ -1,0 +1,68 @@
+// Shared declarations of the CUDA library behind include/qblora.h.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "qblora.h"
+
+#define QB_CUDA(call)                                   \
+  do {                                                  \
+    if ((call) != cudaSuccess) return QBLORA_ERR_CUDA;  \
+  } while (0)
+
+namespace qb {
+
+// Device-side view of a frozen quantized weight (pointers are device pointers).
+struct QwView {
+  int d_in, d_out, block_in, block_out, qfmt, G;  // G = d_in / block_in
+  const uint8_t* codes;
+  const float* alpha;
+  const float* beta;
+  float level[16];  // level table (code-table format) or 0..15 (min-max format)
+};
+
+struct AdView {
+  int l1, l2, r, P, Q;
+  float s;
+  const __nv_bfloat16* A;
+  const __nv_bfloat16* B;
+};
+
+constexpr size_t kStatusBytes = 256;  // first bytes of every workspace: device status word
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// ---- entry points of the individual translation units (host side) ----------------------------
+int launch_quantize(const void* W, int w_dtype, int d_out, int d_in, int block_in, int block_out,
+                    int qfmt, const float* level, uint8_t* codes, float* alpha, float* beta,
+                    cudaStream_t st);
+
+// General path (any block shape, any size): CUDA-core kernels.
+size_t simt_ws_bytes(int op, const QwView& qw, const AdView* ad, int64_t T);
+int simt_linear_fwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, int64_t T, void* Y,
+                    int y_dtype, char* ws, cudaStream_t st);
+int simt_linear_bwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X,
+                    const __nv_bfloat16* dY, int64_t T, void* dX, int dx_dtype, float* dA, float* dB,
+                    char* ws, cudaStream_t st);
+
+size_t merge_ws_bytes(const QwView& qw, const AdView& ad);
+int launch_merge(const QwView& qw, const AdView& ad, bool single_matrix, float* beta_out, char* ws,
+                 cudaStream_t st);
+
+// Bandwidth-bound low-bit product for small token counts (block_out == 1, block_in == 64).
+bool gemv_supported(const QwView& qw, int64_t T);
+int launch_lowbit_gemv(const QwView& qw, const __nv_bfloat16* X, int64_t T, void* Y, int y_dtype,
+                       cudaStream_t st);
+
+// Tensor-core path (tcgen05 / TMEM / TMA): block_in == 64, block_out == 1.
+bool tc_supported(const QwView& qw, const AdView* ad, int64_t T);
+size_t tc_ws_bytes(int op, const QwView& qw, const AdView* ad, int64_t T);
+int tc_linear_fwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, int64_t T, void* Y,
+                  int y_dtype, char* ws, cudaStream_t st);
+int tc_linear_bwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X,
+                  const __nv_bfloat16* dY, int64_t T, void* dX, int dx_dtype, float* dA, float* dB,
+                  char* ws, cudaStream_t st);
+
+}  // namespace qb
