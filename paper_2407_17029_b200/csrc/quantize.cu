@@ -1,0 +1,169 @@
+// Block-wise 4-bit quantizer (Eq. 1).  Every floating-point step is a single IEEE fp32 operation
+// (explicit round-to-nearest intrinsics, no fused multiply-add), so codes, alpha and beta are
+// uniquely determined by the input.
+#include "common.cuh"
+
+namespace qb {
+namespace {
+
+struct QuantTable {
+  float mid[15];  // fl32 midpoints between adjacent levels
+  int zero_idx;   // index of the level closest to 0 (used for all-zero blocks)
+};
+
+__device__ __forceinline__ float load_w(const float* W, int64_t i) { return W[i]; }
+__device__ __forceinline__ float load_w(const __nv_bfloat16* W, int64_t i) {
+  return __bfloat162float(W[i]);
+}
+
+__device__ __forceinline__ int code_of_level(float v, const QuantTable& t) {
+  int c = 0;
+#pragma unroll
+  for (int j = 0; j < 15; ++j) c += (v > t.mid[j]) ? 1 : 0;
+  return c;
+}
+
+__device__ __forceinline__ int code_of_affine(float w, float beta, float alpha) {
+  float q = __fdiv_rn(__fsub_rn(w, beta), alpha);
+  float rq = rintf(q);  // ties to even
+  rq = fminf(fmaxf(rq, 0.0f), 15.0f);
+  return (int)rq;
+}
+
+// One warp per block of 64 consecutive elements of a row (block_in == 64, block_out == 1).
+// Because d_in is a multiple of 64, block b is the flat element range [64 b, 64 b + 64) and its
+// packed codes are bytes [32 b, 32 b + 32).  Lane l owns elements 2l, 2l+1 = byte l.
+template <typename TIn>
+__global__ void __launch_bounds__(256) quantize_b64_kernel(const TIn* __restrict__ W, int64_t nblocks,
+                                                           int qfmt, QuantTable tab,
+                                                           uint8_t* __restrict__ codes,
+                                                           float* __restrict__ alpha,
+                                                           float* __restrict__ beta) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warps_per_grid = (int64_t)gridDim.x * (blockDim.x >> 5);
+  for (int64_t b = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); b < nblocks;
+       b += warps_per_grid) {
+    float w0, w1;
+    if constexpr (sizeof(TIn) == 4) {
+      float2 v = reinterpret_cast<const float2*>(W)[b * 32 + lane];
+      w0 = v.x; w1 = v.y;
+    } else {
+      __nv_bfloat162 v = reinterpret_cast<const __nv_bfloat162*>(W)[b * 32 + lane];
+      w0 = __low2float(v); w1 = __high2float(v);
+    }
+    float mn = fminf(w0, w1), mx = fmaxf(w0, w1), am = fmaxf(fabsf(w0), fabsf(w1));
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) {
+      mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, s));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, s));
+      am = fmaxf(am, __shfl_xor_sync(0xffffffffu, am, s));
+    }
+    int c0, c1;
+    if (qfmt == QBLORA_FMT_CODEBOOK_ABSMAX) {
+      if (am != 0.0f) {
+        c0 = code_of_level(__fdiv_rn(w0, am), tab);
+        c1 = code_of_level(__fdiv_rn(w1, am), tab);
+      } else {
+        c0 = c1 = tab.zero_idx;
+      }
+      if (lane == 0) alpha[b] = am;
+    } else {
+      float d = __fsub_rn(mx, mn);
+      float a = __fdiv_rn(d, 15.0f);
+      bool degenerate = (d == 0.0f) || (a == 0.0f);
+      if (!degenerate) {
+        c0 = code_of_affine(w0, mn, a);
+        c1 = code_of_affine(w1, mn, a);
+      } else {
+        c0 = c1 = 0;
+      }
+      if (lane == 0) {
+        alpha[b] = degenerate ? 0.0f : a;
+        beta[b] = mn;
+      }
+    }
+    codes[b * 32 + lane] = (uint8_t)(c0 | (c1 << 4));
+  }
+}
+
+// Any block shape with an even block_in: one thread per block, two passes over its elements.
+template <typename TIn>
+__global__ void quantize_generic_kernel(const TIn* __restrict__ W, int d_out, int d_in, int block_in,
+                                        int block_out, int qfmt, QuantTable tab,
+                                        uint8_t* __restrict__ codes, float* __restrict__ alpha,
+                                        float* __restrict__ beta) {
+  const int G = d_in / block_in, R = d_out / block_out;
+  int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= (int64_t)G * R) return;
+  const int rb = (int)(b / G), gb = (int)(b % G);
+  const int o0 = rb * block_out, i0 = gb * block_in;
+  float mn = load_w(W, (int64_t)o0 * d_in + i0), mx = mn, am = 0.0f;
+  for (int o = o0; o < o0 + block_out; ++o)
+    for (int i = i0; i < i0 + block_in; ++i) {
+      float w = load_w(W, (int64_t)o * d_in + i);
+      mn = fminf(mn, w); mx = fmaxf(mx, w); am = fmaxf(am, fabsf(w));
+    }
+  float a = 0.0f;
+  bool degenerate;
+  if (qfmt == QBLORA_FMT_CODEBOOK_ABSMAX) {
+    degenerate = (am == 0.0f);
+    alpha[b] = am;
+  } else {
+    float d = __fsub_rn(mx, mn);
+    a = __fdiv_rn(d, 15.0f);
+    degenerate = (d == 0.0f) || (a == 0.0f);
+    alpha[b] = degenerate ? 0.0f : a;
+    beta[b] = mn;
+  }
+  for (int o = o0; o < o0 + block_out; ++o)
+    for (int i = i0; i < i0 + block_in; i += 2) {
+      int c[2];
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        float w = load_w(W, (int64_t)o * d_in + i + e);
+        if (qfmt == QBLORA_FMT_CODEBOOK_ABSMAX)
+          c[e] = degenerate ? tab.zero_idx : code_of_level(__fdiv_rn(w, am), tab);
+        else
+          c[e] = degenerate ? 0 : code_of_affine(w, mn, a);
+      }
+      codes[(int64_t)o * (d_in / 2) + i / 2] = (uint8_t)(c[0] | (c[1] << 4));
+    }
+}
+
+}  // namespace
+
+int launch_quantize(const void* W, int w_dtype, int d_out, int d_in, int block_in, int block_out,
+                    int qfmt, const float* level, uint8_t* codes, float* alpha, float* beta,
+                    cudaStream_t st) {
+  QuantTable tab;
+  tab.zero_idx = 0;
+  for (int j = 0; j < 15; ++j) tab.mid[j] = 0.0f;
+  if (qfmt == QBLORA_FMT_CODEBOOK_ABSMAX) {
+    for (int j = 0; j < 15; ++j)
+      tab.mid[j] = (float)(((double)level[j] + (double)level[j + 1]) / 2.0);
+    for (int j = 1; j < 16; ++j)
+      if (fabs((double)level[j]) < fabs((double)level[tab.zero_idx])) tab.zero_idx = j;
+  }
+  if (block_in == 64 && block_out == 1) {
+    int64_t nblocks = (int64_t)d_out * (d_in / 64);
+    int64_t ctas = (nblocks + 7) / 8;
+    int grid = (int)(ctas < 148 * 16 ? ctas : 148 * 16);
+    if (grid < 1) grid = 1;
+    if (w_dtype == QBLORA_F32)
+      quantize_b64_kernel<float><<<grid, 256, 0, st>>>((const float*)W, nblocks, qfmt, tab, codes, alpha, beta);
+    else
+      quantize_b64_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)W, nblocks, qfmt, tab, codes, alpha, beta);
+  } else {
+    if (block_in % 2) return QBLORA_ERR_UNSUPPORTED;
+    int64_t nblocks = (int64_t)(d_out / block_out) * (d_in / block_in);
+    int grid = (int)((nblocks + 127) / 128);
+    if (w_dtype == QBLORA_F32)
+      quantize_generic_kernel<float><<<grid, 128, 0, st>>>((const float*)W, d_out, d_in, block_in, block_out, qfmt, tab, codes, alpha, beta);
+    else
+      quantize_generic_kernel<__nv_bfloat16><<<grid, 128, 0, st>>>((const __nv_bfloat16*)W, d_out, d_in, block_in, block_out, qfmt, tab, codes, alpha, beta);
+  }
+  QB_CUDA(cudaGetLastError());
+  return QBLORA_OK;
+}
+
+}  // namespace qb

@@ -1,0 +1,82 @@
+"""Helpers shared by the GPU parity tests: numpy <-> device marshalling and the tolerance gates.
+
+Gates (floating-point outputs; the oracle is fp64):
+  strict  -- fp32 outputs (the accumulator before the final rounding) and fp32 gradients:
+             max|gpu - ora| / rms(ora) <= 1e-2.
+  bf16    -- bf16 outputs: rms(gpu - ora) / rms(ora) <= 1e-2 and, per element,
+             |gpu - ora| <= 1e-2 * rms(ora) + 2^-7 * |ora|   (one bf16 ulp of the value itself).
+Integer results (codes) and fp32 quantization parameters are compared bit for bit.
+"""
+import numpy as np
+import torch
+
+import oracle
+from paper_2407_17029_b200 import binding as qb
+from paper_2407_17029_b200 import synth
+
+DEV = "cuda:0"
+TOL = 1e-2
+
+
+def to_bf16_dev(a: np.ndarray) -> torch.Tensor:
+    bits = synth.bf16_bits(a).view(np.int16)
+    return torch.from_numpy(bits.copy()).to(DEV).view(torch.bfloat16)
+
+
+def to_dev(a: np.ndarray) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(a)).to(DEV)
+
+
+def to_np64(t: torch.Tensor) -> np.ndarray:
+    return t.detach().to(torch.float32).cpu().numpy().astype(np.float64)
+
+
+def rms(a):
+    return float(np.sqrt(np.mean(np.square(a, dtype=np.float64))))
+
+
+def gate_strict(gpu, ora, what=""):
+    gpu = np.asarray(gpu, dtype=np.float64)
+    r = max(rms(ora), 1e-30)
+    err = float(np.abs(gpu - ora).max() / r)
+    assert np.isfinite(gpu).all(), f"{what}: non-finite output"
+    assert err <= TOL, f"{what}: max|gpu-ora|/rms = {err:.3e} > {TOL}"
+    return err
+
+
+def gate_bf16(gpu, ora, what=""):
+    gpu = np.asarray(gpu, dtype=np.float64)
+    r = max(rms(ora), 1e-30)
+    assert np.isfinite(gpu).all(), f"{what}: non-finite output"
+    rel = rms(gpu - ora) / r
+    assert rel <= TOL, f"{what}: rms rel err {rel:.3e} > {TOL}"
+    bound = TOL * r + 2.0 ** -7 * np.abs(ora)
+    worst = float((np.abs(gpu - ora) / bound).max())
+    assert worst <= 1.0, f"{what}: element error {worst:.3f} x bound"
+    return rel
+
+
+def qweight_to_dev(qw: oracle.QWeight) -> qb.QWeight:
+    code = [float(x) for x in qw.code] if qw.code is not None else [0.0] * 16
+    return qb.QWeight(qw.d_out, qw.d_in, qw.block_in, qw.block_out, qw.qfmt, code, to_dev(qw.codes),
+                      to_dev(qw.alpha), to_dev(qw.beta) if qw.beta is not None else None)
+
+
+def adapter_to_dev(ad: oracle.Adapter) -> qb.Adapter:
+    return qb.Adapter(ad.lambda_in, ad.lambda_out, ad.rank, float(ad.scaling), to_bf16_dev(ad.A),
+                      to_bf16_dev(ad.B) if ad.B is not None else None)
+
+
+def visible_scaling(Wt, ad: oracle.Adapter, X) -> float:
+    """Scaling s* (fp32-representable) at which the adapter term's RMS equals the base term's."""
+    base = oracle.linear_fwd(Wt, None, X)
+    one = oracle.Adapter(ad.lambda_in, ad.lambda_out, ad.rank, 1.0, ad.A, ad.B)
+    term = oracle.linear_fwd(Wt, one, X) - base
+    return float(np.float32(rms(base) / max(rms(term), 1e-30)))
+
+
+def sample_rows(seed: int, T: int, n: int) -> np.ndarray:
+    if n >= T:
+        return np.arange(T)
+    g = np.random.Generator(np.random.Philox(key=seed + 977))
+    return np.sort(g.choice(T, size=n, replace=False))

@@ -1,0 +1,203 @@
+"""GPU parity: every entry point of the C-ABI library against the fp64 CPU oracle, element by
+element, on seeded inputs that span several tiles and ragged tails, plus edge cases."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2407_17029_b200 import synth
+from tests._parity import (DEV, adapter_to_dev, gate_bf16, gate_strict, qweight_to_dev, rms, to_bf16_dev,
+                           to_dev, to_np64, visible_scaling)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def qb():
+    from paper_2407_17029_b200 import binding
+    return binding
+
+
+# ------------------------------------------------------------------------------------- quantizer
+@pytest.mark.parametrize("qfmt", [0, 1])
+@pytest.mark.parametrize("shape,bi,bo", [((256, 1024), 64, 1), ((200, 192), 64, 1), ((64, 256), 32, 1),
+                                         ((64, 256), 8, 8), ((64, 256), 4, 8), ((1, 64), 64, 1)])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_quantize_bit_exact(qb, qfmt, shape, bi, bo, dtype):
+    W = synth.normal(31, f"qz/{shape}/{bi}x{bo}", shape, 0.02)
+    W[0, :bi] = 0.0                       # a degenerate (all-zero / constant) block
+    if dtype == "bf16":
+        W = synth.round_to_bf16(W)
+        Wd = to_bf16_dev(W)
+    else:
+        Wd = to_dev(W)
+    ref = oracle.quantize_blockwise(W, bi, bo, qfmt)
+    got = qb.quantize_blockwise(Wd, bi, bo, qfmt)
+    assert np.array_equal(got.codes.cpu().numpy(), ref.codes)
+    assert np.array_equal(got.alpha.cpu().numpy().view(np.uint32), ref.alpha.view(np.uint32))
+    if qfmt == 1:
+        assert np.array_equal(got.beta.cpu().numpy().view(np.uint32), ref.beta.view(np.uint32))
+    else:
+        assert got.beta is None
+
+
+def test_quantize_round_trip_on_device(qb):
+    # Q(D(Q(W))) == Q(W) on the level-table format, dequantizing with the oracle in between
+    W = synth.normal(32, "qz/rt", (128, 512), 0.02)
+    q1 = qb.quantize_blockwise(to_dev(W), 64, 1, 0)
+    o1 = oracle.QWeight(128, 512, 64, 1, 0, np.array(q1.code, np.float32), q1.codes.cpu().numpy(),
+                        q1.alpha.cpu().numpy(), None)
+    W1 = oracle.dequantize(o1).astype(np.float32)
+    q2 = qb.quantize_blockwise(to_dev(W1), 64, 1, 0)
+    assert torch.equal(q1.codes, q2.codes) and torch.equal(q1.alpha, q2.alpha)
+
+
+def test_quantize_custom_table(qb):
+    table = np.linspace(-1.0, 1.0, 16).astype(np.float32)
+    W = synth.normal(33, "qz/custom", (32, 128), 0.5)
+    ref = oracle.quantize_blockwise(W, 64, 1, 0, table)
+    got = qb.quantize_blockwise(to_dev(W), 64, 1, 0, [float(x) for x in table])
+    assert np.array_equal(got.codes.cpu().numpy(), ref.codes)
+
+
+# --------------------------------------------------------------------------- forward / backward
+def make_case(seed, T, d_out, d_in, l1, l2, r, qfmt=0, ab_std=0.01, bi=64, bo=1, outliers=0.0):
+    tag = f"case/{seed}"
+    W = synth.normal(seed, tag + "/W", (d_out, d_in), 0.02)
+    X, _ = synth.make_activations(seed, tag + "/X", T, d_in, outliers)
+    dY = synth.round_to_bf16(synth.normal(seed, tag + "/dY", (T, d_out)))
+    A = synth.round_to_bf16(synth.normal(seed, tag + "/A", (d_in // l1, r), ab_std))
+    B = synth.round_to_bf16(synth.normal(seed, tag + "/B", (r, d_out // l2), ab_std))
+    qw = oracle.quantize_blockwise(W, bi, bo, qfmt)
+    ad = oracle.Adapter(l1, l2, r, 1.0, A, B)
+    return qw, ad, X, dY
+
+
+CASES = [
+    # T, d_out, d_in, l1, l2, r  -- several 128-tiles with ragged tails in every dimension
+    (300, 320, 448, 64, 8, 48),
+    (300, 320, 448, 4, 4, 48),
+    (77, 136, 192, 1, 1, 16),
+    (515, 256, 640, 64, 8, 64),
+]
+
+
+@pytest.mark.parametrize("case", CASES)
+@pytest.mark.parametrize("qfmt", [0, 1])
+@pytest.mark.parametrize("visible", [False, True])
+def test_linear_fwd_parity(qb, case, qfmt, visible):
+    T, d_out, d_in, l1, l2, r = case
+    qw, ad, X, _ = make_case(41, T, d_out, d_in, l1, l2, r, qfmt)
+    Wt = oracle.dequantize(qw)
+    if visible:
+        ad.scaling = visible_scaling(Wt, ad, X)
+    ref = oracle.linear_fwd(Wt, ad, X)
+    dq, da, Xd = qweight_to_dev(qw), adapter_to_dev(ad), to_bf16_dev(X)
+    gate_strict(to_np64(qb.linear_fwd(dq, da, Xd, torch.float32)), ref, "Y f32")
+    gate_bf16(to_np64(qb.linear_fwd(dq, da, Xd, torch.bfloat16)), ref, "Y bf16")
+    if visible:
+        base = oracle.linear_fwd(Wt, None, X)
+        assert rms(ref - base) > 0.5 * rms(base)          # the adapter really is half of the output
+
+
+@pytest.mark.parametrize("case", CASES)
+@pytest.mark.parametrize("qfmt", [0, 1])
+@pytest.mark.parametrize("visible", [False, True])
+def test_linear_bwd_parity(qb, case, qfmt, visible):
+    T, d_out, d_in, l1, l2, r = case
+    qw, ad, X, dY = make_case(42, T, d_out, d_in, l1, l2, r, qfmt)
+    Wt = oracle.dequantize(qw)
+    if visible:
+        ad.scaling = visible_scaling(Wt, ad, X)
+    rdX, rdA, rdB = oracle.linear_bwd(Wt, ad, X, dY)
+    dq, da, Xd, dYd = qweight_to_dev(qw), adapter_to_dev(ad), to_bf16_dev(X), to_bf16_dev(dY)
+    dX, dA, dB = qb.linear_bwd(dq, da, Xd, dYd, torch.float32)
+    gate_strict(to_np64(dX), rdX, "dX f32")
+    gate_strict(to_np64(dA), rdA, "dA")
+    gate_strict(to_np64(dB), rdB, "dB")
+    dXb, _, _ = qb.linear_bwd(dq, da, Xd, dYd, torch.bfloat16, need_da=False, need_db=False)
+    gate_bf16(to_np64(dXb), rdX, "dX bf16")
+    # skipping outputs leaves the others unchanged (bit for bit: the library is deterministic)
+    _, dA2, dB2 = qb.linear_bwd(dq, da, Xd, dYd, need_dx=False)
+    assert torch.equal(dA, dA2) and torch.equal(dB, dB2)
+
+
+def test_zero_B_is_bit_identical_to_no_adapter(qb):
+    qw, ad, X, dY = make_case(43, 300, 320, 448, 64, 8, 48)
+    ad.B = np.zeros_like(ad.B)
+    dq, da, Xd, dYd = qweight_to_dev(qw), adapter_to_dev(ad), to_bf16_dev(X), to_bf16_dev(dY)
+    for dt in (torch.float32, torch.bfloat16):
+        assert torch.equal(qb.linear_fwd(dq, da, Xd, dt), qb.linear_fwd(dq, None, Xd, dt))
+    ref = oracle.linear_fwd(oracle.dequantize(qw), None, X)
+    gate_strict(to_np64(qb.linear_fwd(dq, None, Xd, torch.float32)), ref, "base only")
+    dX0, _, _ = qb.linear_bwd(dq, None, None, dYd, torch.float32)
+    gate_strict(to_np64(dX0), oracle.linear_bwd(oracle.dequantize(qw), None, X, dY)[0], "dX base only")
+
+
+def test_outlier_channels_and_general_block_shapes(qb):
+    # 1% input channels x20 (the MLP config's activation recipe) and a 2-D quantization block
+    qw, ad, X, dY = make_case(44, 200, 128, 512, 8, 8, 32, qfmt=1, bi=8, bo=8, outliers=0.01)
+    Wt = oracle.dequantize(qw)
+    ad.scaling = visible_scaling(Wt, ad, X)
+    dq, da, Xd, dYd = qweight_to_dev(qw), adapter_to_dev(ad), to_bf16_dev(X), to_bf16_dev(dY)
+    gate_strict(to_np64(qb.linear_fwd(dq, da, Xd, torch.float32)), oracle.linear_fwd(Wt, ad, X), "Y 2-D blocks")
+    dX, dA, dB = qb.linear_bwd(dq, da, Xd, dYd, torch.float32)
+    r = oracle.linear_bwd(Wt, ad, X, dY)
+    gate_strict(to_np64(dX), r[0], "dX"); gate_strict(to_np64(dA), r[1], "dA"); gate_strict(to_np64(dB), r[2], "dB")
+
+
+def test_single_token_and_workspace_errors(qb):
+    qw, ad, X, dY = make_case(45, 1, 128, 128, 64, 8, 16)
+    Wt = oracle.dequantize(qw)
+    dq, da, Xd = qweight_to_dev(qw), adapter_to_dev(ad), to_bf16_dev(X)
+    gate_strict(to_np64(qb.linear_fwd(dq, da, Xd, torch.float32)), oracle.linear_fwd(Wt, ad, X), "T=1")
+    small = torch.empty(16, dtype=torch.uint8, device=DEV)
+    with pytest.raises(qb.QbloraError) as e:
+        qb.linear_fwd(dq, da, Xd, ws=small)
+    assert e.value.status == qb.ERR_WORKSPACE
+    ws = qb.alloc_workspace(qb.OP_LINEAR_FWD, dq, da, 1)
+    qb.linear_fwd(dq, da, Xd, ws=ws)
+    assert qb.device_status(ws) == qb.OK
+
+
+# ------------------------------------------------------------------------- merge + low-bit product
+@pytest.mark.parametrize("single", [False, True])
+@pytest.mark.parametrize("scaling", [1.0, 37.5])
+def test_merge_bit_exact_and_identity(qb, single, scaling):
+    d_out, d_in, r = 320, 448, 48
+    qw, ad, X, _ = make_case(51, 40, d_out, d_in, 64, 8, r, qfmt=1, ab_std=0.02)
+    if single:
+        ad = oracle.Adapter(64, 8, 0, scaling, synth.round_to_bf16(synth.normal(51, "H", (d_in // 64, d_out // 8), 0.02)), None)
+    ad.scaling = scaling
+    ref = oracle.merge(qw, ad)
+    dq, da = qweight_to_dev(qw), adapter_to_dev(ad)
+    codes0, alpha0 = dq.codes.clone(), dq.alpha.clone()
+    got = qb.merge(dq, da)
+    assert np.array_equal(got.beta.cpu().numpy().view(np.uint32), ref.beta.view(np.uint32))
+    assert torch.equal(dq.codes, codes0) and torch.equal(dq.alpha, alpha0)          # untouched
+    assert got.codes.data_ptr() == dq.codes.data_ptr()
+    # merge identity: low-bit product on the merged weight == unmerged adapted forward
+    Xd = to_bf16_dev(X)
+    unmerged = oracle.linear_fwd(oracle.dequantize(qw), ad, X)
+    gate_strict(to_np64(qb.lowbit_gemm(got, Xd, torch.float32)), unmerged, "merged low-bit vs unmerged fwd")
+    if not single:
+        gate_strict(to_np64(qb.linear_fwd(dq, da, Xd, torch.float32)), unmerged, "unmerged fwd")
+    # in place
+    got2 = qb.merge(dq, da, in_place=True)
+    assert got2.beta.data_ptr() == dq.beta.data_ptr() and torch.equal(got2.beta, got.beta)
+
+
+def test_merge_rejects_misaligned_geometry(qb):
+    qw, ad, _, _ = make_case(52, 4, 128, 128, 4, 4, 16, qfmt=1)
+    with pytest.raises(qb.QbloraError) as e:
+        qb.merge(qweight_to_dev(qw), adapter_to_dev(ad))
+    assert e.value.status == qb.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("T", [1, 2, 3, 8, 16, 17, 150])
+def test_lowbit_gemm_parity(qb, T):
+    qw, _, X, _ = make_case(53, T, 328, 448, 64, 8, 16, qfmt=1)
+    ref = oracle.lowbit_gemm(qw, X)
+    dq, Xd = qweight_to_dev(qw), to_bf16_dev(X)
+    gate_strict(to_np64(qb.lowbit_gemm(dq, Xd, torch.float32)), ref, f"lowbit T={T} f32")
+    gate_bf16(to_np64(qb.lowbit_gemm(dq, Xd, torch.bfloat16)), ref, f"lowbit T={T} bf16")
