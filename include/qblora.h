@@ -102,6 +102,15 @@ const char* qblora_status_string(int status);
  * (QBLORA_OK, or QBLORA_ERR_TIMEOUT if a kernel's bounded wait expired). */
 int qblora_device_status(const void* ws, void* stream);
 
+/* Instrumentation for benchmarks (host-side state, per calling thread; no effect on results).
+ * qblora_kernel_launches(): number of kernels this library has launched so far in this process.
+ * qblora_set_timing_events(start, stop): arms a pair of cudaEvent_t; the next call of
+ * qblora_linear_fwd / qblora_linear_bwd / qablora_lowbit_gemm on this thread records `start`
+ * immediately before and `stop` immediately after its dominant kernel (the base-weight contraction)
+ * on the call's stream, then disarms.  Pass NULL, NULL to disarm.  The paper has no counterpart. */
+uint64_t qblora_kernel_launches(void);
+int qblora_set_timing_events(void* start_event, void* stop_event);
+
 /*
  * Block-wise 4-bit quantization, Eq. 1 (Sec. 3.1).
  *   W       DEVICE [d_out][d_in], fp32 or bf16 (w_dtype); bf16 is promoted exactly.

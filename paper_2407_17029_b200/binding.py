@@ -27,7 +27,8 @@ OP_QUANTIZE, OP_LINEAR_FWD, OP_LINEAR_BWD, OP_MERGE, OP_LOWBIT_GEMM = range(5)
 
 EXPORTS = ["qblora_default_code_table", "qblora_workspace_bytes", "qblora_status_string",
            "qblora_device_status", "qblora_quantize_blockwise", "qblora_linear_fwd",
-           "qblora_linear_bwd", "qablora_merge", "qablora_lowbit_gemm"]
+           "qblora_linear_bwd", "qablora_merge", "qablora_lowbit_gemm", "qblora_kernel_launches",
+           "qblora_set_timing_events"]
 
 
 class _CQWeight(ctypes.Structure):
@@ -66,6 +67,23 @@ _lib.qablora_merge.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p
                                ctypes.c_size_t, ctypes.c_void_p]
 _lib.qablora_lowbit_gemm.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p,
                                      ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+
+
+_lib.qblora_kernel_launches.restype = ctypes.c_uint64
+_lib.qblora_kernel_launches.argtypes = []
+_lib.qblora_set_timing_events.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
+
+
+def kernel_launches() -> int:
+    return int(_lib.qblora_kernel_launches())
+
+
+def set_timing_events(start, stop) -> None:
+    """Arm (torch.cuda.Event, already recorded once or created with enable_timing) or disarm (None, None)."""
+    if start is None:
+        _lib.qblora_set_timing_events(None, None)
+    else:
+        _lib.qblora_set_timing_events(start.cuda_event, stop.cuda_event)
 
 
 class QbloraError(RuntimeError):

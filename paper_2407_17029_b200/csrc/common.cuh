@@ -34,6 +34,15 @@ constexpr size_t kStatusBytes = 256;  // first bytes of every workspace: device 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// ---- instrumentation (instrument.cu) ------------------------------------------------------------
+void count_launch(int n = 1);
+// Brackets the dominant kernel of a call with the armed event pair (if any), then disarms.
+struct DominantKernelTimer {
+  cudaStream_t st; cudaEvent_t stop;
+  explicit DominantKernelTimer(cudaStream_t s);
+  ~DominantKernelTimer();
+};
+
 // ---- entry points of the individual translation units (host side) ----------------------------
 int launch_quantize(const void* W, int w_dtype, int d_out, int d_in, int block_in, int block_out,
                     int qfmt, const float* level, uint8_t* codes, float* alpha, float* beta,

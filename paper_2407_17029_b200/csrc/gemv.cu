@@ -67,6 +67,8 @@ bool gemv_supported(const QwView& qw, int64_t T) {
 
 int launch_lowbit_gemv(const QwView& qw, const __nv_bfloat16* X, int64_t T, void* Y, int y_dtype,
                        cudaStream_t st) {
+  DominantKernelTimer timer(st);
+  count_launch();
   const int rows_per_cta = 8;
   int grid = (qw.d_out + rows_per_cta - 1) / rows_per_cta;
   if (T <= 1) lowbit_gemv_kernel<1><<<grid, 256, 0, st>>>(qw, X, (int)T, Y, y_dtype);

@@ -44,12 +44,14 @@ int launch_merge(const QwView& qw, const AdView& ad, bool single, float* beta_ou
   double* H = reinterpret_cast<double*>(ws + kStatusBytes);
   int64_t n = (int64_t)ad.P * ad.Q;
   merge_h_kernel<<<(unsigned)((n + 127) / 128), 128, 0, st>>>(ad.A, ad.B, ad.P, ad.Q, ad.r, single, H);
+  count_launch();
   QB_CUDA(cudaGetLastError());
   const int R = qw.d_out / qw.block_out;
   n = (int64_t)R * qw.G;
   merge_beta_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(qw.beta, H, R, qw.G, ad.Q, qw.block_in,
                                                                qw.block_out, ad.l1, ad.l2, (double)ad.s,
                                                                beta_out);
+  count_launch();
   QB_CUDA(cudaGetLastError());
   return QBLORA_OK;
 }

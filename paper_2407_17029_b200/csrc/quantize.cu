@@ -162,6 +162,7 @@ int launch_quantize(const void* W, int w_dtype, int d_out, int d_in, int block_i
     else
       quantize_generic_kernel<__nv_bfloat16><<<grid, 128, 0, st>>>((const __nv_bfloat16*)W, d_out, d_in, block_in, block_out, qfmt, tab, codes, alpha, beta);
   }
+  count_launch();
   QB_CUDA(cudaGetLastError());
   return QBLORA_OK;
 }

@@ -106,6 +106,7 @@ int gemm(int64_t M, int64_t N, int64_t K, LA la, LB lb, EP ep, cudaStream_t st) 
   dim3 grid((unsigned)((N + 63) / 64), (unsigned)((M + 63) / 64));
   if (grid.y > 65535) return QBLORA_ERR_UNSUPPORTED;
   simt_gemm_kernel<LA, LB, EP, A_KC, B_KC><<<grid, 256, 0, st>>>((int)M, (int)N, (int)K, la, lb, ep);
+  count_launch();
   QB_CUDA(cudaGetLastError());
   return QBLORA_OK;
 }
@@ -171,6 +172,7 @@ int simt_linear_fwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, 
   if (ad) {
     int64_t n = T * ad->P;
     pool_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(X, T, qw.d_in, ad->l1, w.xp);
+    count_launch();
     QB_CUDA(cudaGetLastError());
     // u = x' A : A is [P][r] -> lb(n = k_rank, k = p) = A[p][k_rank]
     rc = gemm<true, false>(T, ad->r, ad->P, LdF32{w.xp, ad->P, 1}, LdBF16{ad->A, 1, ad->r},
@@ -183,6 +185,7 @@ int simt_linear_fwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, 
   }
   EpOut ep{Y, y_dtype, qw.d_out, ad ? w.v : nullptr, ad ? ad->Q : 0, ad ? ad->l2 : 1,
            ad ? ad->s : 0.0f, false};
+  DominantKernelTimer timer(st);
   return gemm<true, true>(T, qw.d_out, qw.d_in, LdBF16{X, qw.d_in, 1}, LdWq{qw, true}, ep, st);
 }
 
@@ -194,9 +197,11 @@ int simt_linear_bwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X,
   if (ad) {
     int64_t n = T * ad->P;
     pool_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(X, T, qw.d_in, ad->l1, w.xp);
+    count_launch();
     QB_CUDA(cudaGetLastError());
     n = T * ad->Q;
     dv_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(dY, T, qw.d_out, ad->l2, ad->s, w.dv);
+    count_launch();
     QB_CUDA(cudaGetLastError());
     // du = dv B^T : lb(n = k_rank, k = q) = B[k_rank][q]
     rc = gemm<true, true>(T, ad->r, ad->Q, LdF32{w.dv, ad->Q, 1}, LdBF16{ad->B, ad->Q, 1},
@@ -227,6 +232,7 @@ int simt_linear_bwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X,
   if (dX) {
     EpOut ep{dX, dx_dtype, qw.d_in, ad ? w.dxp : nullptr, ad ? ad->P : 0, ad ? ad->l1 : 1, 0.0f, true};
     // dX[t][i] = sum_o dY[t][o] w~[o][i] : lb(n = i, k = o)
+    DominantKernelTimer timer(st);
     return gemm<true, false>(T, qw.d_in, qw.d_out, LdBF16{dY, qw.d_out, 1}, LdWq{qw, false}, ep, st);
   }
   return QBLORA_OK;
