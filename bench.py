@@ -1,0 +1,394 @@
+#!/usr/bin/env python
+"""Benchmark of the adapted quantized linear layer (Q-BLoRA / QA-BLoRA hot path) on B200.
+
+One step = forward + backward (dX, dA, dB) of every adapted linear of the workload through the
+C-ABI library, inputs resident in HBM.  Prints ONE JSON line.  ``--impl reference`` times the fp64
+CPU oracle on the host cores instead (a bounded sample of the same workload per step).
+
+Multi-GPU: the path has no exchange step; ``--gpus N`` (launched with torch.distributed.run) runs
+N independent replicas and reports the aggregate ("replicas only", weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2407_17029_b200 import synth  # noqa: E402
+
+METRIC = "fused 4-bit+BLoRA linear fwd+bwd TFLOP/s & low-bit GEMM GB/s, % of roofline"
+
+
+# ----------------------------------------------------------------------------------- accounting
+def linear_flops(T, d_out, d_in, r, geom):
+    """Algorithmic flops of one adapted linear, forward + backward: two base contractions
+    (2*T*D_in*D_out each) and the adapter's (2*T*r*(P+Q) forward, twice that backward)."""
+    P, Q = d_in // geom.lambda_in, d_out // geom.lambda_out
+    base = 2 * (2.0 * T * d_in * d_out)
+    adapter = 3 * (2.0 * T * r * (P + Q))
+    return base, adapter
+
+
+def packed_bytes(d_out, d_in, block_in=64, with_beta=True):
+    """Algorithmic bytes of one pass over a packed weight: 4-bit codes + fp32 alpha (+ beta) per block."""
+    return d_out * d_in // 2 + (d_out * d_in // block_in) * (8 if with_beta else 4)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.th = threading.Thread(target=self._read, daemon=True)
+            self.th.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------ reference (oracle)
+def oracle_step(wl, geom, sample_rows, cache):
+    """One bounded oracle step: forward + backward of every linear on `sample_rows` token rows."""
+    import oracle
+    flops = 0.0
+    t0 = time.perf_counter()
+    for spec in wl.linears:
+        qw, Wt, li = cache[spec.name]
+        ad = oracle.Adapter(geom.lambda_in, geom.lambda_out, wl.rank, wl.scaling, li.A, li.B)
+        oracle.linear_fwd(Wt, ad, li.X)
+        oracle.linear_bwd(Wt, ad, li.X, li.dY)
+        b, a = linear_flops(sample_rows, spec.d_out, spec.d_in, wl.rank, geom)
+        flops += b + a
+    return time.perf_counter() - t0, flops
+
+
+def oracle_cache(wl, geom, sample_rows):
+    import oracle
+    cache = {}
+    for spec in wl.linears:
+        li = synth.make_linear_inputs(wl, spec, geom, seed=0, tokens=sample_rows)
+        qw = oracle.quantize_blockwise(li.W, wl.block_in, 1, wl.qfmt)
+        cache[spec.name] = (qw, oracle.dequantize(qw), li)
+        li.W = None
+    return cache
+
+
+def run_reference(args, wl, geom):
+    import oracle
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    rows = args.ref_rows
+    cache = oracle_cache(wl, geom, rows)
+    for _ in range(min(args.warmup, 1)):
+        oracle_step(wl, geom, rows, cache)
+    tot_t, tot_f = 0.0, 0.0
+    steps = min(args.steps, args.ref_max_steps)
+    for _ in range(steps):
+        t, f = oracle_step(wl, geom, rows, cache)
+        tot_t += t; tot_f += f
+    val = tot_f / tot_t / 1e12
+    cores = oracle.num_threads()
+    sample = f"{rows} of {wl.tokens} token rows per step, all linears, fwd+bwd (dX, dA, dB)"
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
+            "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": tot_t / steps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": wl.name, "geometry": geom.name, "sample": sample},
+            "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------------------- GPU arm
+def run_gpu(args, wl, geom):
+    import torch
+    from paper_2407_17029_b200 import binding as qb
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    def bf(a):
+        return torch.from_numpy(synth.bf16_bits(a).view(np.int16).copy()).to(dev).view(torch.bfloat16)
+
+    T, r = wl.tokens, wl.rank
+    peaks = measured_peaks()
+    l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
+    # ---- build the sets of resident buffers; rotate over enough distinct sets to exceed 2x L2
+    lin = []
+    step_bytes = 0
+    for spec in wl.linears:
+        li = synth.make_linear_inputs(wl, spec, geom, seed=rank)
+        dq = qb.quantize_blockwise(torch.from_numpy(li.W).to(dev), wl.block_in, 1, wl.qfmt)
+        li.W = None
+        per_set = (li.X.size + li.dY.size) * 2 * 2 + packed_bytes(spec.d_out, spec.d_in, wl.block_in, wl.qfmt == 1)
+        step_bytes += per_set
+        lin.append((spec, li, dq))
+    nsets = max(2, int(np.ceil(2.0 * l2_bytes / step_bytes)) + 1)
+    sets = []
+    for s in range(nsets):
+        items = []
+        for spec, li, dq in lin:
+            # distinct device copies (same values): what matters is that the addresses differ
+            q2 = qb.QWeight(dq.d_out, dq.d_in, dq.block_in, dq.block_out, dq.qfmt, dq.code,
+                            dq.codes.clone(), dq.alpha.clone(), dq.beta.clone() if dq.beta is not None else None)
+            ad = qb.Adapter(geom.lambda_in, geom.lambda_out, r, wl.scaling, bf(li.A), bf(li.B))
+            X, dY = bf(li.X), bf(li.dY)
+            Y = torch.empty((T, spec.d_out), dtype=torch.bfloat16, device=dev)
+            dX = torch.empty((T, spec.d_in), dtype=torch.bfloat16, device=dev)
+            dA = torch.empty(tuple(ad.A.shape), dtype=torch.float32, device=dev)
+            dB = torch.empty(tuple(ad.B.shape), dtype=torch.float32, device=dev)
+            wsf = qb.alloc_workspace(qb.OP_LINEAR_FWD, q2, ad, T)
+            wsb = qb.alloc_workspace(qb.OP_LINEAR_BWD, q2, ad, T)
+            items.append((spec, q2, ad, X, dY, Y, dX, dA, dB, wsf, wsb))
+        sets.append(items)
+
+    def step(i, ev=None):
+        for j, (spec, q2, ad, X, dY, Y, dX, dA, dB, wsf, wsb) in enumerate(sets[i % nsets]):
+            if ev is not None and j == ev[2]:
+                qb.set_timing_events(ev[0], ev[1])
+            qb.linear_fwd(q2, ad, X, ws=wsf, out=Y)
+            qb.linear_bwd(q2, ad, X, dY, ws=wsb, outs=(dX, dA, dB))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    flops_step = sum(sum(linear_flops(T, s.d_out, s.d_in, r, geom)) for s in wl.linears)
+    # dominant kernel: the forward base contraction of the largest linear
+    dom = max(range(len(wl.linears)), key=lambda j: wl.linears[j].d_out * wl.linears[j].d_in)
+    dspec = wl.linears[dom]
+    dom_flops = 2.0 * T * dspec.d_in * dspec.d_out
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True), dom) for _ in range(args.steps)]
+    launches0 = qb.kernel_launches()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for i in range(args.steps):
+        step(args.warmup + i, kev[i])
+    e1.record()
+    barrier()
+    launches = qb.kernel_launches() - launches0
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop()
+    dom_ms = statistics.mean(a.elapsed_time(b) for a, b, _ in kev)
+    for spec, q2, ad, X, dY, Y, dX, dA, dB, wsf, wsb in sets[0]:
+        assert qb.device_status(wsf) == qb.OK and qb.device_status(wsb) == qb.OK
+    if dist is not None:
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    value = flops_step * world * args.steps / (ms * 1e-3) / 1e12
+
+    # ---- end to end: host (pinned) inputs in, results out, copies inside the timed region
+    items = sets[0]
+    host = []
+    h2d = d2h = 0
+    for spec, q2, ad, X, dY, Y, dX, dA, dB, wsf, wsb in items:
+        hX, hdY = X.cpu().pin_memory(), dY.cpu().pin_memory()
+        hY, hdX = torch.empty_like(Y, device="cpu").pin_memory(), torch.empty_like(dX, device="cpu").pin_memory()
+        hdA, hdB = torch.empty_like(dA, device="cpu").pin_memory(), torch.empty_like(dB, device="cpu").pin_memory()
+        host.append((hX, hdY, hY, hdX, hdA, hdB))
+        h2d += hX.numel() * 2 + hdY.numel() * 2
+        d2h += hY.numel() * 2 + hdX.numel() * 2 + hdA.numel() * 4 + hdB.numel() * 4
+
+    def e2e_step():
+        for (spec, q2, ad, X, dY, Y, dX, dA, dB, wsf, wsb), (hX, hdY, hY, hdX, hdA, hdB) in zip(items, host):
+            X.copy_(hX, non_blocking=True); dY.copy_(hdY, non_blocking=True)
+            qb.linear_fwd(q2, ad, X, ws=wsf, out=Y)
+            qb.linear_bwd(q2, ad, X, dY, ws=wsb, outs=(dX, dA, dB))
+            hY.copy_(Y, non_blocking=True); hdX.copy_(dX, non_blocking=True)
+            hdA.copy_(dA, non_blocking=True); hdB.copy_(dB, non_blocking=True)
+
+    e2e_steps = max(3, min(args.steps, 10))
+    e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    barrier()
+    e2e_s = time.perf_counter() - t0
+    if dist is not None:
+        t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e_val = flops_step * world * e2e_steps / e2e_s / 1e12
+
+    line = {"metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": wl.name, "geometry": f"{geom.name} (lambda_in={geom.lambda_in}, lambda_out={geom.lambda_out})",
+                       "tokens": T, "linears": [f"{s.name}[{s.d_out},{s.d_in}]" for s in wl.linears], "rank": r,
+                       "quant": "4-bit, block 64 along input, " + ("min-max" if wl.qfmt else "level table + absmax"),
+                       "parallelism": "replicas only" if world > 1 else "single GPU",
+                       "l2": f"rotating over {nsets} distinct buffer sets ({nsets * step_bytes / 2**20:.0f} MiB > 2x L2)"},
+            "clocks": clocks, "gpu_launches": int(launches),
+            "e2e": {"value": e2e_val, "unit": "TFLOP/s", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                    "steps": e2e_steps},
+            "roofline": {"bound": "tensor", "kernel": f"forward base contraction {dspec.name}[{dspec.d_out},{dspec.d_in}] T={T}",
+                         "achieved": dom_flops / (dom_ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops_sustained"],
+                         "peak_kind": f"bf16 dense, sustained, {peaks['source']}", "unit": "TFLOP/s",
+                         "frac": dom_flops / (dom_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+                         "traffic": None, "ms_per_launch": dom_ms},
+            "step_flops": flops_step}
+
+    if rank == 0 and not args.no_extras:
+        line["lowbit"] = lowbit_extras(qb, torch, dev, peaks, l2_bytes)
+    if rank == 0 and not args.no_cpu_baseline and world == 1:
+        rows = args.ref_rows
+        cache = oracle_cache(wl, geom, rows)
+        import oracle
+        t, f = oracle_step(wl, geom, rows, cache)
+        line["cpu_baseline"] = {"value": f / t / 1e12, "unit": "TFLOP/s", "cores": oracle.num_threads(), "kind": "oracle",
+                                "sample": f"{rows} of {T} token rows, all linears, fwd+bwd (dX, dA, dB), {t:.1f} s"}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def lowbit_extras(qb, torch, dev, peaks, l2_bytes):
+    """Deploy path of the QA-BLoRA config: merge, then the low-bit product at 1 and 16 tokens on the
+    attention and MLP shapes; GB/s = packed-weight bytes streamed once / kernel time."""
+    wl = synth.WORKLOADS["C5"]
+    out = {}
+
+    def bf(a):
+        return torch.from_numpy(synth.bf16_bits(a).view(np.int16).copy()).to(dev).view(torch.bfloat16)
+
+    for spec in wl.linears[:2]:
+        li = synth.make_linear_inputs(wl, spec, synth.GEOM_A, seed=0, tokens=16)
+        dq = qb.quantize_blockwise(torch.from_numpy(li.W).to(dev), 64, 1, qb.FMT_AFFINE_MINMAX)
+        li.W = None
+        ad = qb.Adapter(64, 8, wl.rank, 1.0, bf(li.A), bf(li.B))
+        nbytes = packed_bytes(spec.d_out, spec.d_in)
+        ncopies = int(np.ceil(2.0 * l2_bytes / nbytes)) + 1
+        copies = []
+        for _ in range(ncopies):
+            m = qb.merge(dq, ad)
+            copies.append(qb.QWeight(m.d_out, m.d_in, 64, 1, m.qfmt, m.code, m.codes.clone(), m.alpha.clone(), m.beta.clone()))
+        # merge timing
+        wsm = qb.alloc_workspace(qb.OP_MERGE, dq, ad, 0)
+        s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for _ in range(3):
+            qb.merge(dq, ad, ws=wsm)
+        s.record()
+        for _ in range(10):
+            qb.merge(dq, ad, ws=wsm)
+        e.record(); torch.cuda.synchronize()
+        out[f"{spec.name}/merge_us"] = s.elapsed_time(e) / 10 * 1e3
+        X = bf(li.X)
+        for T in (1, 16):
+            Xt = X[:T].contiguous()
+            Y = torch.empty((T, spec.d_out), dtype=torch.bfloat16, device=dev)
+            ws = qb.alloc_workspace(qb.OP_LOWBIT_GEMM, copies[0], None, T)
+            for i in range(5):
+                qb.lowbit_gemm(copies[i % ncopies], Xt, ws=ws, out=Y)
+            reps = 40
+            s.record()
+            for i in range(reps):
+                qb.lowbit_gemm(copies[i % ncopies], Xt, ws=ws, out=Y)
+            e.record(); torch.cuda.synchronize()
+            us = s.elapsed_time(e) / reps * 1e3
+            gbs = nbytes / (us * 1e-6) / 1e9
+            out[f"{spec.name}/T{T}"] = {"us": us, "GB/s": gbs, "frac_hbm": gbs / peaks["hbm_gbs"],
+                                        "bytes": nbytes, "copies": ncopies}
+    out["peak_hbm_gbs"] = peaks["hbm_gbs"]
+    out["peak_kind"] = peaks["source"]
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="gpu", choices=["gpu", "reference"])
+    ap.add_argument("--workload", default="C2", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--geometry", default="GA", choices=["GA", "GB"])
+    ap.add_argument("--ref-rows", type=int, default=512, help="token rows per oracle step (bounded sample)")
+    ap.add_argument("--ref-max-steps", type=int, default=3)
+    ap.add_argument("--no-extras", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "gpu" else args.warmup
+    wl = synth.WORKLOADS[args.workload]
+    geom = synth.GEOM_A if args.geometry == "GA" else synth.GEOM_B
+    if args.impl == "reference":
+        run_reference(args, wl, geom)
+    else:
+        run_gpu(args, wl, geom)
+
+
+if __name__ == "__main__":
+    main()
