@@ -230,6 +230,8 @@ def run_gpu(args, wl, geom):
     sampler.start()
     time.sleep(0.3)
     kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True), dom) for _ in range(args.steps)]
+    for a, b, _ in kev:          # torch creates the CUDA event handle on first record
+        a.record(); b.record()
     launches0 = qb.kernel_launches()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
