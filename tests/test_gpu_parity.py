@@ -18,6 +18,16 @@ def qb():
     return binding
 
 
+@pytest.fixture(params=["tensor-core", "general"])
+def path(request, monkeypatch):
+    """Runs a test once on the tcgen05 path and once with the CUDA-core path forced."""
+    if request.param == "general":
+        monkeypatch.setenv("QBLORA_FORCE_GENERAL", "1")
+    else:
+        monkeypatch.delenv("QBLORA_FORCE_GENERAL", raising=False)
+    return request.param
+
+
 # ------------------------------------------------------------------------------------- quantizer
 @pytest.mark.parametrize("qfmt", [0, 1])
 @pytest.mark.parametrize("shape,bi,bo", [((256, 1024), 64, 1), ((200, 192), 64, 1), ((64, 256), 32, 1),
@@ -85,7 +95,7 @@ CASES = [
 @pytest.mark.parametrize("case", CASES)
 @pytest.mark.parametrize("qfmt", [0, 1])
 @pytest.mark.parametrize("visible", [False, True])
-def test_linear_fwd_parity(qb, case, qfmt, visible):
+def test_linear_fwd_parity(qb, path, case, qfmt, visible):
     T, d_out, d_in, l1, l2, r = case
     qw, ad, X, _ = make_case(41, T, d_out, d_in, l1, l2, r, qfmt)
     Wt = oracle.dequantize(qw)
@@ -103,7 +113,7 @@ def test_linear_fwd_parity(qb, case, qfmt, visible):
 @pytest.mark.parametrize("case", CASES)
 @pytest.mark.parametrize("qfmt", [0, 1])
 @pytest.mark.parametrize("visible", [False, True])
-def test_linear_bwd_parity(qb, case, qfmt, visible):
+def test_linear_bwd_parity(qb, path, case, qfmt, visible):
     T, d_out, d_in, l1, l2, r = case
     qw, ad, X, dY = make_case(42, T, d_out, d_in, l1, l2, r, qfmt)
     Wt = oracle.dequantize(qw)
@@ -122,7 +132,7 @@ def test_linear_bwd_parity(qb, case, qfmt, visible):
     assert torch.equal(dA, dA2) and torch.equal(dB, dB2)
 
 
-def test_zero_B_is_bit_identical_to_no_adapter(qb):
+def test_zero_B_is_bit_identical_to_no_adapter(qb, path):
     qw, ad, X, dY = make_case(43, 300, 320, 448, 64, 8, 48)
     ad.B = np.zeros_like(ad.B)
     dq, da, Xd, dYd = qweight_to_dev(qw), adapter_to_dev(ad), to_bf16_dev(X), to_bf16_dev(dY)
@@ -195,7 +205,7 @@ def test_merge_rejects_misaligned_geometry(qb):
 
 
 @pytest.mark.parametrize("T", [1, 2, 3, 8, 16, 17, 150])
-def test_lowbit_gemm_parity(qb, T):
+def test_lowbit_gemm_parity(qb, path, T):
     qw, _, X, _ = make_case(53, T, 328, 448, 64, 8, 16, qfmt=1)
     ref = oracle.lowbit_gemm(qw, X)
     dq, Xd = qweight_to_dev(qw), to_bf16_dev(X)
