@@ -6,15 +6,20 @@
 //   forward : Y^T[o][t]  = sum_i w~[o][i] X[t][i]   + sum_k B[k][o/l2]      (s u)[t][k]
 //   backward: dX^T[i][t] = sum_o w~[o][i] dY[t][o]  + sum_k A[i/l1][k]      (du/l1)[t][k]
 //
-// The dequantized weight tile is the MMA's A operand (M = 128 rows of W~ or W~^T), written to
-// shared memory by four dequant warps in the canonical 128-byte-swizzled layout (K-major in the
-// forward, MN-major in the backward, so the same [o][i]-packed codes serve both); tokens are the B
-// operand (N = 256), staged by TMA.  Accumulators live in TMEM (2 x 256 columns, double-buffered so
-// the epilogue of one tile overlaps the mainloop of the next).
+// Two CTAs on the two SMs of a TPC form a cluster and issue tcgen05.mma with cta_group::2: the
+// pair computes a 256 (weight rows) x 256 (tokens) tile.  Each CTA dequantizes its own 128 weight
+// rows into shared memory (the MMA's A operand, canonical 128-byte-swizzled layout: K-major in the
+// forward, MN-major in the backward, so the same [o][i]-packed codes serve both) and stages half of
+// the token tile by TMA (the B operand; no multicast), which halves the shared-memory traffic per
+// MMA cycle compared with a single-CTA tile -- the resource that bounds this kernel.  Accumulators
+// live in TMEM (2 x 256 columns, double-buffered so the epilogue of one tile overlaps the mainloop
+// of the next).
 //
-// Warp roles (320 threads): warp 0 TMA producer, warp 1 MMA issuer + TMEM owner, warps 2-5 dequant,
-// warps 6-9 epilogue.  Every mbarrier wait is bounded; on expiry the kernel stores
-// QBLORA_ERR_TIMEOUT in the workspace status word and every role leaves its loop.
+// Warp roles (448 threads per CTA): warp 0 TMA producer; warp 1 MMA issuer (leader CTA) or relay
+// that reports this CTA's stage readiness to the leader (other CTA), and TMEM owner; warps 2-9 two
+// dequant groups taking alternate K-blocks; warps 10-13 epilogue.  Every mbarrier wait is bounded;
+// on expiry the kernel stores QBLORA_ERR_TIMEOUT in the workspace status word and every role
+// leaves its loop.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -24,23 +29,23 @@ namespace qb {
 using namespace simt;
 namespace {
 
-constexpr int BM = 128;   // rows of the weight-side operand per tile
-constexpr int BN = 256;   // tokens per tile
-constexpr int BK = 64;    // contraction elements per stage = one quantization block
-constexpr int STAGES = 4;
-constexpr int A_BYTES = BM * BK * 2;
-constexpr int B_BYTES = BN * BK * 2;
-constexpr int P_BYTES = BM * BK / 2;
-constexpr int NUM_THREADS = 320;
-constexpr int SMEM_BYTES = STAGES * (A_BYTES + B_BYTES + P_BYTES) + 256 + 1024;
+constexpr int BM = 128;        // rows of the weight-side operand per CTA (256 per CTA pair)
+constexpr int BN = 256;        // tokens per tile (each CTA of the pair stages 128 of them)
+constexpr int BN_HALF = BN / 2;
+constexpr int BK = 64;         // contraction elements per stage = one quantization block
+constexpr int STAGES = 6;
+constexpr int A_BYTES = BM * BK * 2;        // 16 KB dequantized weight tile
+constexpr int B_BYTES = BN_HALF * BK * 2;   // 16 KB: this CTA's half of the token tile
+constexpr int P_BYTES = BM * BK / 2;        // 4 KB packed codes
+constexpr int NUM_THREADS = 448;            // 14 warps, see roles above
+constexpr int SMEM_BYTES = STAGES * (A_BYTES + B_BYTES + P_BYTES) + 512 + 1024;
 constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;  // ~1 s: far beyond any legitimate wait
 
 struct TcParams {
-  int mode;                 // 0 forward, 1 backward
   int M;                    // output rows of the tile grid: d_out (forward) / d_in (backward)
   int kb_base, kb_extra;    // K-blocks from the quantized weight / from the adapter
   int T;
-  int m_tiles, n_tiles;
+  int m_tiles, n_tiles;     // tiles of 256 rows x 256 tokens (one per CTA pair)
   int d_in, d_out, G;
   const float* alpha;
   const float* beta;
@@ -54,12 +59,28 @@ struct TcParams {
 
 // ------------------------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// arrive on a barrier of another CTA of the cluster (address from map_to_cta)
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
@@ -67,7 +88,7 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
-      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
@@ -91,12 +112,15 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm,
 __device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+// completion of all prior MMAs of the pair -> one arrival on the barrier at this offset in both CTAs
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
   asm volatile(
-      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+      ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}"
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
 }
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
@@ -129,52 +153,80 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
-
-// Eight 4-bit codes (one 32-bit word, code e in bits 4e..4e+3) -> eight bf16 values alpha*level+beta.
-// `tabv` holds level[lane & 15] in every lane, so a warp shuffle indexed by the raw shifted word
-// (the source lane is taken modulo 32, and lanes 16-31 mirror lanes 0-15) is the table lookup.
-// The product is formed in fp32 and rounded once to bf16.
-__device__ __forceinline__ void dequant_word(uint32_t w, float tabv, float alpha, float beta, uint32_t (&o)[4]) {
-  float v[8];
-#pragma unroll
-  for (int e = 0; e < 8; ++e) {
-    const float lv = __shfl_sync(0xffffffffu, tabv, (int)(w >> (4 * e)));
-    v[e] = fmaf(alpha, lv, beta);
-  }
-#pragma unroll
-  for (int e = 0; e < 4; ++e) o[e] = pack_bf16x2(v[2 * e], v[2 * e + 1]);
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+  uint32_t r;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
+  return r;
 }
 
+// Per-block dequantization table kept in registers.  The sixteen values bf16(alpha * level[c] + beta)
+// of one quantization block (fp32 product, one rounding) are split into a low-byte plane and a
+// high-byte plane of four registers each; a 4-bit code then selects its two bytes with byte-permute
+// instructions only (no shared-memory or shuffle traffic, which the tensor core's operand fetch needs).
+struct BlockTable {
+  uint32_t lp[4], hp[4];
+  __device__ __forceinline__ void build(const float (&level)[16], float alpha, float beta) {
+#pragma unroll
+    for (int m = 0; m < 4; ++m) {
+      const uint32_t p0 = pack_bf16x2(fmaf(alpha, level[4 * m + 0], beta), fmaf(alpha, level[4 * m + 1], beta));
+      const uint32_t p1 = pack_bf16x2(fmaf(alpha, level[4 * m + 2], beta), fmaf(alpha, level[4 * m + 3], beta));
+      lp[m] = prmt(p0, p1, 0x6420u);
+      hp[m] = prmt(p0, p1, 0x7531u);
+    }
+  }
+  // four codes in the low 16 bits of `a` (each masked to 3 bits) / `s2` (merge selector) -> 4 bf16
+  __device__ __forceinline__ void half(uint32_t a, uint32_t s2, uint32_t& o01, uint32_t& o23) const {
+    const uint32_t lo = prmt(prmt(lp[0], lp[1], a), prmt(lp[2], lp[3], a), s2);
+    const uint32_t hi = prmt(prmt(hp[0], hp[1], a), prmt(hp[2], hp[3], a), s2);
+    o01 = prmt(lo, hi, 0x5140u);
+    o23 = prmt(lo, hi, 0x7362u);
+  }
+  // eight codes (code e in bits 4e..4e+3 of w) -> eight bf16 values in element order
+  __device__ __forceinline__ void lookup8(uint32_t w, uint32_t (&o)[4]) const {
+    const uint32_t a = w & 0x77777777u;                               // index within an 8-entry half
+    const uint32_t s2 = ((w >> 1) & 0x44444444u) | 0x32103210u;       // byte j: j + 4 * (code >> 3)
+    half(a, s2, o[0], o[1]);
+    half(a >> 16, s2 >> 16, o[2], o[3]);
+  }
+};
+
 template <int MODE>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ CUtensorMap tm_bx,
-                  const __grid_constant__ CUtensorMap tm_p, const TcParams p) {
+                  const __grid_constant__ CUtensorMap tm_p, const __grid_constant__ TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   const uint32_t sA = base, sB = sA + STAGES * A_BYTES, sP = sB + STAGES * B_BYTES;
   const uint32_t bars = sP + STAGES * P_BYTES;
   const uint8_t* gP = smem_raw + (sP - raw);
-  auto full = [&](int s) { return bars + 8u * s; };
-  auto aready = [&](int s) { return bars + 8u * (STAGES + s); };
-  auto empty = [&](int s) { return bars + 8u * (2 * STAGES + s); };
-  auto accfull = [&](int a) { return bars + 8u * (3 * STAGES + a); };
-  auto accempty = [&](int a) { return bars + 8u * (3 * STAGES + 2 + a); };
-  const uint32_t tmem_slot = bars + 8u * (3 * STAGES + 4);
+  auto full = [&](int s) { return bars + 8u * s; };                      // TMA bytes landed (local)
+  auto aready = [&](int s) { return bars + 8u * (STAGES + s); };          // dequantized tile written (local)
+  auto empty = [&](int s) { return bars + 8u * (2 * STAGES + s); };       // MMAs reading the stage are done
+  auto peer = [&](int s) { return bars + 8u * (3 * STAGES + s); };        // leader only: the other CTA's stage is ready
+  auto accfull = [&](int a) { return bars + 8u * (4 * STAGES + a); };
+  auto accempty = [&](int a) { return bars + 8u * (4 * STAGES + 2 + a); };  // leader only: both epilogues drained
+  const uint32_t tmem_slot = bars + 8u * (4 * STAGES + 4);
   volatile uint32_t* tmem_slot_g = reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - raw));
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t rank = cluster_ctarank();       // 0 = leader (issues the MMAs of the pair)
+  const int num_clusters = gridDim.x >> 1, cluster_id = blockIdx.x >> 1;
+
   if (tid == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(full(s), 1); mbar_init(aready(s), 128); mbar_init(empty(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(accfull(a), 1); mbar_init(accempty(a), 128); }
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full(s), 1); mbar_init(aready(s), 128); mbar_init(empty(s), 1); mbar_init(peer(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) { mbar_init(accfull(a), 1); mbar_init(accempty(a), 256); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(512) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  if (warp == 1) {  // the same warp of both CTAs allocates the pair's tensor memory
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(512) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();
+  cluster_sync_all();   // barriers of both CTAs are initialised before any remote arrival
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot_g;
 
@@ -186,8 +238,9 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-        const int m0 = (tile % p.m_tiles) * BM, t0 = (tile / p.m_tiles) * BN;
+      for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
+        const int m0 = (tile % p.m_tiles) * (2 * BM) + (int)rank * BM;
+        const int t0 = (tile / p.m_tiles) * BN + (int)rank * BN_HALF;
         for (int kb = 0; kb < kb_total; ++kb, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1u;
@@ -195,8 +248,12 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
           if (kb < p.kb_base) {
             mbar_arrive_expect_tx(full(s), B_BYTES + P_BYTES);
             tma_load_2d(sB + s * B_BYTES, &tm_b, full(s), kb * BK, t0);
-            if (MODE == 0) tma_load_2d(sP + s * P_BYTES, &tm_p, full(s), kb * (BK / 2), m0);
-            else           tma_load_2d(sP + s * P_BYTES, &tm_p, full(s), m0 / 2, kb * BK);
+            if (MODE == 0) {
+              tma_load_2d(sP + s * P_BYTES, &tm_p, full(s), kb * (BK / 2), m0);
+            } else {   // two boxes of 64 rows x 32 bytes: packed[ng][k][32 B]
+              tma_load_2d(sP + s * P_BYTES, &tm_p, full(s), m0 / 2, kb * BK);
+              tma_load_2d(sP + s * P_BYTES + P_BYTES / 2, &tm_p, full(s), m0 / 2 + 32, kb * BK);
+            }
           } else {
             mbar_arrive_expect_tx(full(s), B_BYTES);
             tma_load_2d(sB + s * B_BYTES, &tm_bx, full(s), (kb - p.kb_base) * BK, t0);
@@ -209,15 +266,16 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer (one lane)
-    if (lane == 0) {
-      // instruction descriptor: D fp32, A/B bf16, B K-major, A K-major (forward) or MN-major (backward)
+    if (lane == 0 && rank == 0) {
+      // ------------------------------------------------------------------ MMA issuer (leader CTA, one lane)
+      // instruction descriptor: D fp32, A/B bf16, B K-major, A K-major (forward) or MN-major (backward),
+      // M = 256 and N = 256 across the CTA pair
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((MODE == 1 ? 1u : 0u) << 15) |
-                             ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+                             ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
       uint32_t it = 0;
       bool ok = true;
       int lt = 0;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++lt) {
+      for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters, ++lt) {
         const int a = lt & 1;
         const uint32_t aph = (lt >> 1) & 1u;
         if (!mbar_wait(accempty(a), aph ^ 1u, p.status)) { ok = false; break; }
@@ -226,7 +284,8 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
         for (int kb = 0; kb < kb_total; ++kb, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1u;
-          if (!mbar_wait(full(s), ph, p.status) || !mbar_wait(aready(s), ph, p.status)) { ok = false; break; }
+          if (!mbar_wait(full(s), ph, p.status) || !mbar_wait(aready(s), ph, p.status) ||
+              !mbar_wait(peer(s), ph, p.status)) { ok = false; break; }
           tc_fence_after();
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k) {
@@ -234,60 +293,73 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
             if (MODE == 0) adesc = smem_desc(sA + s * A_BYTES + k * 32, 16, 1024);
             else           adesc = smem_desc(sA + s * A_BYTES + k * 2048, 8192, 1024);
             bdesc = smem_desc(sB + s * B_BYTES + k * 32, 16, 1024);
-            tc_mma(d_tmem, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+            tc_mma_pair(d_tmem, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
           }
-          tc_commit(empty(s));
+          tc_commit_pair(empty(s));
         }
-        if (ok) tc_commit(accfull(a));
+        if (ok) tc_commit_pair(accfull(a));
+      }
+    } else if (lane == 0) {
+      // ------------------------------------------------------------------ relay (other CTA, one lane):
+      // tells the leader when this CTA's half of a stage (tokens landed, weight tile written) is ready
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
+        for (int kb = 0; kb < kb_total; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1u;
+          if (!mbar_wait(full(s), ph, p.status) || !mbar_wait(aready(s), ph, p.status)) { ok = false; break; }
+          mbar_arrive_cluster(map_to_cta(peer(s), 0));
+        }
       }
     }
-  } else if (warp < 6) {
-    // ------------------------------------------------------------------ dequant warps (128 threads)
-    const int d = tid - 64;
-    const float tabv = p.level[lane & 15];
-    uint32_t it = 0;
+  } else if (warp < 10) {
+    // ------------------------------------------------------------------ dequant warps: two groups of 128
+    // threads; group g fills the stages of K-blocks with (global index & 1) == g.  Thread d owns one
+    // quantization block (64 codes, one alpha/beta) of the tile per K-block.
+    const int g = (warp - 2) >> 2;
+    const int d = tid - 64 - 128 * g;
+    const uint32_t sw = (lane >> 2) & 1u;   // which 16-byte half of the 32 packed bytes to read first
     bool ok = true;
-    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-      const int m0 = (tile % p.m_tiles) * BM;
+    uint32_t it = 0;
+    for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
+      const int m0 = (tile % p.m_tiles) * (2 * BM) + (int)rank * BM;
       for (int kb = 0; kb < kb_total; ++kb, ++it) {
+        if ((int)(it & 1u) != g) continue;
         const int s = it % STAGES;
         const uint32_t ph = (it / STAGES) & 1u;
         const uint32_t a_stage = sA + s * A_BYTES;
+        uint32_t dst, xr;   // address of this thread's 128-byte row (before the chunk XOR) and XOR pattern
+        if (MODE == 0) { dst = a_stage + d * 128; xr = d & 7; }
+        else           { dst = a_stage + (d >> 6) * 8192 + (d & 63) * 128; xr = d & 7; }
         if (kb < p.kb_base) {
           float al = 0.0f, be = 0.0f;
-          const uint8_t* src;
-          uint32_t dst;   // address of 16-byte chunk 0 of this thread's 64 elements (before the XOR)
-          uint32_t xr;    // XOR pattern (row index within the 8-row swizzle atom)
           if (MODE == 0) {
             const int row = m0 + d;
             if (row < p.d_out) {
               al = __ldg(p.alpha + (int64_t)row * p.G + kb);
               if (p.beta) be = __ldg(p.beta + (int64_t)row * p.G + kb);
             }
-            src = gP + s * P_BYTES + d * 32;
-            dst = a_stage + d * 128;
-            xr = d & 7;
           } else {
-            const int k = d & 63, ng = d >> 6;
-            const int o = kb * BK + k, blk = (m0 >> 6) + ng;
+            const int o = kb * BK + (d & 63), blk = (m0 >> 6) + (d >> 6);
             if (o < p.d_out && blk < p.G) {
               al = __ldg(p.alpha + (int64_t)o * p.G + blk);
               if (p.beta) be = __ldg(p.beta + (int64_t)o * p.G + blk);
             }
-            src = gP + s * P_BYTES + k * 64 + ng * 32;
-            dst = a_stage + ng * 8192 + k * 128;
-            xr = k & 7;
           }
-          const bool landed = mbar_wait(full(s), ph, p.status) && mbar_wait(empty(s), ph ^ 1u, p.status);
-          if (!__all_sync(0xffffffffu, landed)) { ok = false; break; }   // keep the warp together for the shuffles
-          const uint4 q0 = *reinterpret_cast<const uint4*>(src);
-          const uint4 q1 = *reinterpret_cast<const uint4*>(src + 16);
+          BlockTable tab;
+          tab.build(p.level, al, be);
+          if (!mbar_wait(full(s), ph, p.status) || !mbar_wait(empty(s), ph ^ 1u, p.status)) { ok = false; break; }
+          const uint8_t* src = gP + s * P_BYTES + d * 32;
+          const uint4 q0 = *reinterpret_cast<const uint4*>(src + sw * 16);
+          const uint4 q1 = *reinterpret_cast<const uint4*>(src + (sw ^ 1u) * 16);
           const uint32_t w[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+          const uint32_t xr2 = xr ^ (sw << 2);   // load position j holds logical word j ^ (4 * sw)
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             uint32_t o4[4];
-            dequant_word(w[j], tabv, al, be, o4);
-            st_shared_v4(dst + (((uint32_t)j ^ xr) << 4), o4[0], o4[1], o4[2], o4[3]);
+            tab.lookup8(w[j], o4);
+            st_shared_v4(dst + (((uint32_t)j ^ xr2) << 4), o4[0], o4[1], o4[2], o4[3]);
           }
         } else {
           if (!mbar_wait(empty(s), ph ^ 1u, p.status)) { ok = false; break; }
@@ -295,7 +367,6 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
           if (MODE == 0) {
             // A[m = o][k] = B[kk + k][o / lambda_out], read from the transposed copy (row = q)
             const int row = m0 + d;
-            const uint32_t dst = a_stage + d * 128, xr = d & 7;
             if (row < p.d_out) {
               const uint4* src = reinterpret_cast<const uint4*>(p.ex + (int64_t)(row / p.lam) * p.ex_ld + kk);
 #pragma unroll
@@ -309,10 +380,8 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
             }
           } else {
             // A[m = i][k] = A_adapter[i / lambda_in][kk + k], read from the transposed copy (row = kk + k)
-            const int k = d & 63, ng = d >> 6;
-            const uint32_t dst = a_stage + ng * 8192 + k * 128, xr = k & 7;
-            const unsigned short* src = reinterpret_cast<const unsigned short*>(p.ex + (int64_t)(kk + k) * p.ex_ld);
-            const int i0 = m0 + ng * 64;
+            const unsigned short* src = reinterpret_cast<const unsigned short*>(p.ex + (int64_t)(kk + (d & 63)) * p.ex_ld);
+            const int i0 = m0 + (d >> 6) * 64;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
               uint32_t o4[4];
@@ -334,12 +403,13 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
   } else {
     // ------------------------------------------------------------------ epilogue warps (128 threads)
     const int q = warp & 3;                       // TMEM lane quadrant this warp may read
+    const uint32_t leader_accempty0 = map_to_cta(accempty(0), 0), leader_accempty1 = map_to_cta(accempty(1), 0);
     bool ok = true;
     int lt = 0;
-    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++lt) {
+    for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters, ++lt) {
       const int a = lt & 1;
       const uint32_t aph = (lt >> 1) & 1u;
-      const int m = (tile % p.m_tiles) * BM + q * 32 + lane;
+      const int m = (tile % p.m_tiles) * (2 * BM) + (int)rank * BM + q * 32 + lane;
       const int t0 = (tile / p.m_tiles) * BN;
       if (!mbar_wait(accfull(a), aph, p.status)) { ok = false; break; }
       tc_fence_after();
@@ -366,15 +436,17 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
         }
       }
       tc_fence_before();
-      mbar_arrive(accempty(a));
+      mbar_arrive_cluster(a == 0 ? leader_accempty0 : leader_accempty1);
     }
   }
 
+  // Neither CTA may leave (or free tensor memory) while its partner can still reach into it.
   tc_fence_before();
   __syncthreads();
+  cluster_sync_all();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
   }
 }
 
@@ -487,13 +559,12 @@ int launch_main(int mode, const QwView& qw, const AdView* ad, const __nv_bfloat1
     attr_set[mode] = true;
   }
   TcParams p{};
-  p.mode = mode;
   p.M = mode == 0 ? qw.d_out : qw.d_in;
   const int Kq = mode == 0 ? qw.d_in : qw.d_out;
   p.kb_base = (Kq + BK - 1) / BK;
   p.kb_extra = ad ? r_pad / BK : 0;
   p.T = (int)T;
-  p.m_tiles = (p.M + BM - 1) / BM;
+  p.m_tiles = (p.M + 2 * BM - 1) / (2 * BM);
   p.n_tiles = (int)((T + BN - 1) / BN);
   p.d_in = qw.d_in; p.d_out = qw.d_out; p.G = qw.G;
   p.alpha = qw.alpha; p.beta = qw.beta;
@@ -504,17 +575,18 @@ int launch_main(int mode, const QwView& qw, const AdView* ad, const __nv_bfloat1
   p.out = out; p.out_dtype = out_dtype; p.status = status;
 
   CUtensorMap tm_b, tm_bx, tm_p;
-  int rc = make_map(&tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Bop, (uint64_t)Kq, (uint64_t)T, (uint64_t)Kq * 2, BK, BN, true);
+  int rc = make_map(&tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Bop, (uint64_t)Kq, (uint64_t)T, (uint64_t)Kq * 2, BK, BN_HALF, true);
   if (rc) return rc;
-  if (ad) rc = make_map(&tm_bx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Bx, (uint64_t)r_pad, (uint64_t)T, (uint64_t)r_pad * 2, BK, BN, true);
+  if (ad) rc = make_map(&tm_bx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Bx, (uint64_t)r_pad, (uint64_t)T, (uint64_t)r_pad * 2, BK, BN_HALF, true);
   else tm_bx = tm_b;
   if (rc) return rc;
   if (mode == 0) rc = make_map(&tm_p, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qw.codes, (uint64_t)qw.d_in / 2, (uint64_t)qw.d_out, (uint64_t)qw.d_in / 2, BK / 2, BM, false);
-  else rc = make_map(&tm_p, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qw.codes, (uint64_t)qw.d_in / 2, (uint64_t)qw.d_out, (uint64_t)qw.d_in / 2, BM / 2, BK, false);
+  else rc = make_map(&tm_p, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qw.codes, (uint64_t)qw.d_in / 2, (uint64_t)qw.d_out, (uint64_t)qw.d_in / 2, BK / 2, BK, false);
   if (rc) return rc;
 
-  const int tiles = p.m_tiles * p.n_tiles;
-  const int grid = tiles < num_sms() ? tiles : num_sms();
+  const int tiles = p.m_tiles * p.n_tiles;                      // one tile per CTA pair
+  const int pairs = num_sms() / 2;
+  const int grid = 2 * (tiles < pairs ? tiles : pairs);
   {
     DominantKernelTimer timer(st);
     if (mode == 0) tc_dq_gemm_kernel<0><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(tm_b, tm_bx, tm_p, p);
