@@ -15,9 +15,9 @@
 // live in TMEM (2 x 256 columns, double-buffered so the epilogue of one tile overlaps the mainloop
 // of the next).
 //
-// Warp roles (448 threads per CTA): warp 0 TMA producer; warp 1 MMA issuer (leader CTA) or relay
-// that reports this CTA's stage readiness to the leader (other CTA), and TMEM owner; warps 2-9 two
-// dequant groups taking alternate K-blocks; warps 10-13 epilogue.  Every mbarrier wait is bounded;
+// Warp roles (448 threads per CTA): warp 0 TMA producer; warp 1 MMA issuer (leader CTA only) and
+// TMEM owner; warps 2-9 two dequant groups taking alternate K-blocks (those of the other CTA report
+// each finished stage to the leader's barrier); warps 10-13 epilogue.  Every mbarrier wait is bounded;
 // on expiry the kernel stores QBLORA_ERR_TIMEOUT in the workspace status word and every role
 // leaves its loop.
 #include <cuda.h>
@@ -80,7 +80,7 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 }
 // arrive on a barrier of another CTA of the cluster (address from map_to_cta)
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
@@ -193,7 +193,7 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
 
   if (tid == 0) {
     for (int s = 0; s < STAGES; ++s) {
-      mbar_init(full(s), 1); mbar_init(aready(s), 128); mbar_init(empty(s), 1); mbar_init(peer(s), 1);
+      mbar_init(full(s), 1); mbar_init(aready(s), 128); mbar_init(empty(s), 1); mbar_init(peer(s), 4);
     }
     for (int a = 0; a < 2; ++a) { mbar_init(accfull(a), 1); mbar_init(accempty(a), 256); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -277,19 +277,6 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
         }
         if (ok) tc_commit_pair(accfull(a));
       }
-    } else if (lane == 0) {
-      // ------------------------------------------------------------------ relay (other CTA, one lane):
-      // tells the leader when this CTA's half of a stage (tokens landed, weight tile written) is ready
-      uint32_t it = 0;
-      bool ok = true;
-      for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
-        for (int kb = 0; kb < kb_total; ++kb, ++it) {
-          const int s = it % STAGES;
-          const uint32_t ph = (it / STAGES) & 1u;
-          if (!mbar_wait(full(s), ph, p.status) || !mbar_wait(aready(s), ph, p.status)) { ok = false; break; }
-          mbar_arrive_cluster(map_to_cta(peer(s), 0));
-        }
-      }
     }
   } else if (warp < 10) {
     // ------------------------------------------------------------------ dequant warps: two groups of 128
@@ -298,6 +285,7 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
     const int g = (warp - 2) >> 2;
     const int d = tid - 64 - 128 * g;
     const float tabv = p.level[lane & 15];
+    const uint32_t leader_peer = map_to_cta(peer(0), 0);
     bool ok = true;
     uint32_t it = 0;
     for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
@@ -338,7 +326,8 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
             st_shared_v4(dst + (((uint32_t)j ^ xr) << 4), o4[0], o4[1], o4[2], o4[3]);
           }
         } else {
-          if (!mbar_wait(empty(s), ph ^ 1u, p.status)) { ok = false; break; }
+          // adapter K-blocks carry no packed codes, but the other CTA still vouches for its token half
+          if (!mbar_wait(empty(s), ph ^ 1u, p.status) || (rank != 0 && !mbar_wait(full(s), ph, p.status))) { ok = false; break; }
           const int kk = (kb - p.kb_base) * BK;
           if (MODE == 0) {
             // A[m = o][k] = B[kk + k][o / lambda_out], read from the transposed copy (row = q)
@@ -373,7 +362,13 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
           }
         }
         fence_async_proxy();   // generic-proxy stores -> visible to the tensor core's async proxy
-        mbar_arrive(aready(s));
+        if (rank == 0) {
+          mbar_arrive(aready(s));
+        } else {
+          // this CTA's stage (token half landed, weight tile written) is ready: tell the leader, once per warp
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(leader_peer + 8u * s);
+        }
       }
     }
   } else {
