@@ -24,9 +24,12 @@
 
 #include "common.cuh"
 #include "simt_gemm.cuh"
+#include "tc_ptx.cuh"
+#include "tc_small.cuh"
 
 namespace qb {
 using namespace simt;
+using namespace ptx;
 namespace {
 
 constexpr int BM = 128;        // rows of the weight-side operand per CTA (256 per CTA pair)
@@ -39,7 +42,6 @@ constexpr int B_BYTES = BN_HALF * BK * 2;   // 16 KB: this CTA's half of the tok
 constexpr int P_BYTES = BM * BK / 2;        // 4 KB packed codes
 constexpr int NUM_THREADS = 448;            // 14 warps, see roles above
 constexpr int SMEM_BYTES = STAGES * (A_BYTES + B_BYTES + P_BYTES) + 512 + 1024;
-constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;  // ~1 s: far beyond any legitimate wait
 
 struct TcParams {
   int M;                    // output rows of the tile grid: d_out (forward) / d_in (backward)
@@ -50,109 +52,13 @@ struct TcParams {
   const float* alpha;
   const float* beta;
   float level[16];
-  const __nv_bfloat16* ex;  // forward: B^T [Q][r_pad]; backward: A^T [r_pad][P]
-  int ex_ld, lam;           // leading dimension of ex; forward lambda_out, backward lambda_in
+  const __nv_bfloat16* ex;  // adapter matrix feeding the extra K-blocks: forward B [r][Q], backward A [P][r]
+  int ex_ld, ex_rows, lam;  // its leading dimension; the rank r; forward lambda_out, backward lambda_in
   void* out;                // forward Y [T][d_out]; backward dX [T][d_in]
   int out_dtype;
   int* status;
 };
 
-// ------------------------------------------------------------------------------------ PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-  return r;
-}
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
-  return r;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-// arrive on a barrier of another CTA of the cluster (address from map_to_cta)
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
-  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait: false (and the status word set) if the phase did not complete in time.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  while (!mbar_try_wait(bar, parity)) {
-    if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
-      atomicExch(status, (int)QBLORA_ERR_TIMEOUT);
-      return false;
-    }
-  }
-  return true;
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1) : "memory");
-}
-__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-// completion of all prior MMAs of the pair -> one arrival on the barrier at this offset in both CTAs
-__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
-  asm volatile(
-      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-      ::"r"(bar), "h"((uint16_t)3) : "memory");
-}
-__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
-}
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-      : "r"(taddr) : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
-// Shared-memory matrix descriptor, 128-byte swizzle.  `lbo`/`sbo` in bytes.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
-  uint64_t d = 0;
-  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
-  d |= (uint64_t)((lbo >> 4) & 0x3FFFu) << 16;
-  d |= (uint64_t)((sbo >> 4) & 0x3FFFu) << 32;
-  d |= (uint64_t)1 << 46;   // descriptor version (sm_100)
-  d |= (uint64_t)2 << 61;   // 128-byte swizzle
-  return d;
-}
-
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&v);
-}
-__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-}
 // Eight 4-bit codes (one 32-bit word, code e in bits 4e..4e+3) -> eight bf16 values alpha*level+beta.
 // `tabv` holds level[lane & 15] in every lane, so a warp shuffle indexed by the raw shifted word
 // (the source lane is taken modulo 32, and lanes 16-31 mirror lanes 0-15) is the table lookup.
@@ -248,8 +154,9 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
       // ------------------------------------------------------------------ MMA issuer (leader CTA, one lane)
       // instruction descriptor: D fp32, A/B bf16, B K-major, A K-major (forward) or MN-major (backward),
       // M = 256 and N = 256 across the CTA pair
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((MODE == 1 ? 1u : 0u) << 15) |
-                             ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
+      const uint32_t idesc_common = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) |
+                                    ((uint32_t)((2 * BM) >> 4) << 24);
+      const uint32_t idesc_kmajor = idesc_common, idesc_mnmajor = idesc_common | (1u << 15);
       uint32_t it = 0;
       bool ok = true;
       int lt = 0;
@@ -265,13 +172,15 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
           if (!mbar_wait(full(s), ph, p.status) || !mbar_wait(aready(s), ph, p.status) ||
               !mbar_wait(peer(s), ph, p.status)) { ok = false; break; }
           tc_fence_after();
+          // weight K-blocks: K-major tile in the forward, MN-major in the backward; the adapter
+          // K-blocks are written the other way round (see the dequant warps)
+          const bool a_kmajor = (MODE == 0) == (kb < p.kb_base);
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k) {
-            uint64_t adesc, bdesc;
-            if (MODE == 0) adesc = smem_desc(sA + s * A_BYTES + k * 32, 16, 1024);
-            else           adesc = smem_desc(sA + s * A_BYTES + k * 2048, 8192, 1024);
-            bdesc = smem_desc(sB + s * B_BYTES + k * 32, 16, 1024);
-            tc_mma_pair(d_tmem, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+            const uint64_t adesc = a_kmajor ? smem_desc(sA + s * A_BYTES + k * 32, 16, 1024)
+                                            : smem_desc(sA + s * A_BYTES + k * 2048, 8192, 1024);
+            const uint64_t bdesc = smem_desc(sB + s * B_BYTES + k * 32, 16, 1024);
+            tc_mma_pair(d_tmem, adesc, bdesc, a_kmajor ? idesc_kmajor : idesc_mnmajor, (kb | k) != 0 ? 1u : 0u);
           }
           tc_commit_pair(empty(s));
         }
@@ -295,9 +204,12 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
         const int s = it % STAGES;
         const uint32_t ph = (it / STAGES) & 1u;
         const uint32_t a_stage = sA + s * A_BYTES;
-        uint32_t dst, xr;   // address of this thread's 128-byte row (before the chunk XOR) and XOR pattern
-        if (MODE == 0) { dst = a_stage + d * 128; xr = d & 7; }
-        else           { dst = a_stage + (d >> 6) * 8192 + (d & 63) * 128; xr = d & 7; }
+        // K-major tile: thread d owns row d (64 K elements = 128 bytes).  MN-major tile: thread d owns
+        // K-row (d & 63) of the 64-row group (d >> 6).  Either way a 128-byte row whose 16-byte chunks
+        // are XOR-swizzled with (d & 7).
+        const bool a_kmajor = (MODE == 0) == (kb < p.kb_base);
+        const uint32_t dst = a_kmajor ? a_stage + d * 128 : a_stage + (d >> 6) * 8192 + (d & 63) * 128;
+        const uint32_t xr = d & 7;
         if (kb < p.kb_base) {
           float al = 0.0f, be = 0.0f;
           if (MODE == 0) {
@@ -330,34 +242,44 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
           if (!mbar_wait(empty(s), ph ^ 1u, p.status) || (rank != 0 && !mbar_wait(full(s), ph, p.status))) { ok = false; break; }
           const int kk = (kb - p.kb_base) * BK;
           if (MODE == 0) {
-            // A[m = o][k] = B[kk + k][o / lambda_out], read from the transposed copy (row = q)
-            const int row = m0 + d;
-            if (row < p.d_out) {
-              const uint4* src = reinterpret_cast<const uint4*>(p.ex + (int64_t)(row / p.lam) * p.ex_ld + kk);
+            // MN-major tile: A[m = o][k] = B[kk + k][o / lambda_out]; thread = (K-row, 64-wide output group),
+            // reading a contiguous run of row kk + k of B
+            const int krow = kk + (d & 63);
+            const int o0 = m0 + (d >> 6) * 64;
+            const unsigned short* src = reinterpret_cast<const unsigned short*>(p.ex) + (int64_t)krow * p.ex_ld;
+            const bool live = krow < p.ex_rows;
+            if ((p.lam & 7) == 0) {       // a 16-byte chunk (8 outputs) repeats a single element of B
 #pragma unroll
               for (int j = 0; j < 8; ++j) {
-                const uint4 v = __ldg(src + j);
-                st_shared_v4(dst + (((uint32_t)j ^ xr) << 4), v.x, v.y, v.z, v.w);
+                const int o = o0 + j * 8;
+                uint32_t v = (live && o < p.d_out) ? (uint32_t)__ldg(src + o / p.lam) : 0u;
+                v |= v << 16;
+                st_shared_v4(dst + (((uint32_t)j ^ xr) << 4), v, v, v, v);
               }
             } else {
 #pragma unroll
-              for (int j = 0; j < 8; ++j) st_shared_v4(dst + (((uint32_t)j ^ xr) << 4), 0, 0, 0, 0);
+              for (int j = 0; j < 8; ++j) {
+                uint32_t o4[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  const int oa = o0 + j * 8 + 2 * e, ob = oa + 1;
+                  const uint32_t lo = (live && oa < p.d_out) ? (uint32_t)__ldg(src + oa / p.lam) : 0u;
+                  const uint32_t hi = (live && ob < p.d_out) ? (uint32_t)__ldg(src + ob / p.lam) : 0u;
+                  o4[e] = lo | (hi << 16);
+                }
+                st_shared_v4(dst + (((uint32_t)j ^ xr) << 4), o4[0], o4[1], o4[2], o4[3]);
+              }
             }
           } else {
-            // A[m = i][k] = A_adapter[i / lambda_in][kk + k], read from the transposed copy (row = kk + k)
-            const unsigned short* src = reinterpret_cast<const unsigned short*>(p.ex + (int64_t)(kk + (d & 63)) * p.ex_ld);
-            const int i0 = m0 + (d >> 6) * 64;
+            // K-major tile: A[m = i][k] = A_adapter[i / lambda_in][kk + k]; thread = input column i,
+            // reading 128 contiguous bytes of a row of A_adapter (rank is a multiple of 8)
+            const int i = m0 + d;
+            const uint4* src = reinterpret_cast<const uint4*>(p.ex + (int64_t)(i / p.lam) * p.ex_ld + kk);
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-              uint32_t o4[4];
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const int ia = i0 + j * 8 + 2 * e, ib = ia + 1;
-                const uint32_t lo = ia < p.d_in ? (uint32_t)__ldg(src + ia / p.lam) : 0u;
-                const uint32_t hi = ib < p.d_in ? (uint32_t)__ldg(src + ib / p.lam) : 0u;
-                o4[e] = lo | (hi << 16);
-              }
-              st_shared_v4(dst + (((uint32_t)j ^ xr) << 4), o4[0], o4[1], o4[2], o4[3]);
+              uint4 v = make_uint4(0, 0, 0, 0);
+              if (i < p.d_in && kk + j * 8 < p.ex_rows) v = __ldg(src + j);
+              st_shared_v4(dst + (((uint32_t)j ^ xr) << 4), v.x, v.y, v.z, v.w);
             }
           }
         }
@@ -422,61 +344,52 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
 }
 
 // -------------------------------------------------------------------------------- adapter helpers
-// dst[c][rw] = src[rw][c] for rw < rows, zero for rows <= rw < rows_pad (dst leading dimension rows_pad).
-__global__ void transpose_pad_cols_kernel(const __nv_bfloat16* __restrict__ src, int rows, int cols, int rows_pad,
-                                          __nv_bfloat16* __restrict__ dst) {
-  int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= (int64_t)cols * rows_pad) return;
-  const int c = (int)(idx / rows_pad), rw = (int)(idx % rows_pad);
-  dst[idx] = rw < rows ? src[(int64_t)rw * cols + c] : __float2bfloat16_rn(0.0f);
+__device__ __forceinline__ void store_split(float x, __nv_bfloat16* hi, __nv_bfloat16* lo, int64_t idx) {
+  const __nv_bfloat16 h = __float2bfloat16_rn(x);
+  hi[idx] = h;
+  lo[idx] = __float2bfloat16_rn(x - __bfloat162float(h));
 }
-// dst[rw][c] = src[c][rw] for rw < rows_src... : A^T with zero rows appended: dst [r_pad][P], src A [P][r].
-__global__ void transpose_pad_rows_kernel(const __nv_bfloat16* __restrict__ A, int P, int r, int r_pad,
-                                          __nv_bfloat16* __restrict__ dst) {
-  int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= (int64_t)r_pad * P) return;
-  const int k = (int)(idx / P), pp = (int)(idx % P);
-  dst[idx] = k < r ? A[(int64_t)pp * r + k] : __float2bfloat16_rn(0.0f);
-}
-
-struct EpBf16Scaled {  // C16[m][n] = bf16(scale * acc); optional fp32 copy of acc
-  __nv_bfloat16* C16; int64_t ld16; float scale; bool divide; float* C32; int64_t ld32;
-  __device__ void operator()(int m, int n, float acc) const {
-    if (C32) C32[m * ld32 + n] = acc;
-    const float v = divide ? __fdiv_rn(acc, scale) : acc * scale;
-    C16[m * ld16 + n] = __float2bfloat16_rn(v);
+// x'[t][p] = AvgPool_{lambda_in}(X) (Sec. 3.2) as a bf16 hi + lo pair (hi + lo carries ~16 mantissa bits)
+__global__ void pool_split_kernel(const __nv_bfloat16* __restrict__ X, int64_t T, int d_in, int l1, int ldp,
+                                  __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+  const int P = d_in / l1;
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= T * P) return;
+  const int64_t t = idx / P; const int pp = (int)(idx % P);
+  const __nv_bfloat16* src = X + t * d_in + (int64_t)pp * l1;
+  float s = 0.0f;
+  if ((l1 & 7) == 0) {
+    for (int j = 0; j < l1; j += 8) {
+      const uint4 v = __ldg(reinterpret_cast<const uint4*>(src + j));
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) s += __uint_as_float(w[e] << 16) + __uint_as_float(w[e] & 0xffff0000u);
+    }
+  } else {
+    for (int j = 0; j < l1; ++j) s += __bfloat162float(src[j]);
   }
-};
-
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = []() -> EncodeTiledFn {
-    void* f = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess) return nullptr;
-    if (q != cudaDriverEntryPointSuccess) return nullptr;
-    return reinterpret_cast<EncodeTiledFn>(f);
-  }();
-  return fn;
+  store_split(__fdiv_rn(s, (float)l1), hi, lo, t * ldp + pp);
 }
-
-// 2-D tensor map: `inner` contiguous elements per row, `rows` rows, row pitch `pitch_bytes`.
-int make_map(CUtensorMap* tm, CUtensorMapDataType dt, int elem_bytes, const void* ptr, uint64_t inner,
-             uint64_t rows, uint64_t pitch_bytes, uint32_t box_inner, uint32_t box_rows, bool swizzle128) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return QBLORA_ERR_CUDA;
-  cuuint64_t dims[2] = {inner, rows};
-  cuuint64_t strides[1] = {pitch_bytes};
-  cuuint32_t box[2] = {box_inner, box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  (void)elem_bytes;
-  CUresult r = fn(tm, dt, 2, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                  swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
-                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? QBLORA_OK : QBLORA_ERR_CUDA;
+// dv[t][q] = s * sum of lambda_out consecutive output gradients (adjoint of repeat_interleave), hi + lo
+__global__ void dv_split_kernel(const __nv_bfloat16* __restrict__ dY, int64_t T, int d_out, int l2, float scaling,
+                                int ldq, __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+  const int Q = d_out / l2;
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= T * Q) return;
+  const int64_t t = idx / Q; const int q = (int)(idx % Q);
+  const __nv_bfloat16* src = dY + t * d_out + (int64_t)q * l2;
+  float a = 0.0f;
+  if ((l2 & 7) == 0) {
+    for (int j = 0; j < l2; j += 8) {
+      const uint4 v = __ldg(reinterpret_cast<const uint4*>(src + j));
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) a += __uint_as_float(w[e] << 16) + __uint_as_float(w[e] & 0xffff0000u);
+    }
+  } else {
+    for (int j = 0; j < l2; ++j) a += __bfloat162float(src[j]);
+  }
+  store_split(scaling * a, hi, lo, t * ldq + q);
 }
 
 int num_sms() {
@@ -489,38 +402,37 @@ int num_sms() {
   return n;
 }
 
+inline int round8(int x) { return (x + 7) / 8 * 8; }
+
 struct TcWs {
-  float *xp, *u32, *dv, *du32;
-  __nv_bfloat16 *u16, *bt, *du16, *at;
-  int r_pad;
+  __nv_bfloat16 *xh, *xl, *u16, *dvh, *dvl, *duh, *dul, *du16, *uh, *ul;
+  int ldp, ldq, ldr;
   size_t bytes;
 };
 
 TcWs carve(int op, const AdView* ad, int64_t T, char* ws) {
   TcWs w{};
   size_t off = kStatusBytes;
-  auto take = [&](size_t nbytes) { char* ptr = ws ? ws + off : nullptr; off += align_up(nbytes, 256); return ptr; };
+  auto take = [&](size_t elems) { char* ptr = ws ? ws + off : nullptr; off += align_up(elems * 2, 256); return (__nv_bfloat16*)ptr; };
   if (ad) {
-    w.r_pad = (ad->r + BK - 1) / BK * BK;
-    w.xp = (float*)take((size_t)T * ad->P * 4);
-    w.u32 = (float*)take((size_t)T * ad->r * 4);
+    w.ldp = round8(ad->P); w.ldq = round8(ad->Q); w.ldr = round8(ad->r);
+    w.xh = take((size_t)T * w.ldp); w.xl = take((size_t)T * w.ldp);
     if (op == QBLORA_OP_LINEAR_FWD) {
-      w.u16 = (__nv_bfloat16*)take((size_t)T * w.r_pad * 2);
-      w.bt = (__nv_bfloat16*)take((size_t)ad->Q * w.r_pad * 2);
+      w.u16 = take((size_t)T * w.ldr);
     } else {
-      w.dv = (float*)take((size_t)T * ad->Q * 4);
-      w.du32 = (float*)take((size_t)T * ad->r * 4);
-      w.du16 = (__nv_bfloat16*)take((size_t)T * w.r_pad * 2);
-      w.at = (__nv_bfloat16*)take((size_t)w.r_pad * ad->P * 2);
+      w.dvh = take((size_t)T * w.ldq); w.dvl = take((size_t)T * w.ldq);
+      w.duh = take((size_t)T * w.ldr); w.dul = take((size_t)T * w.ldr); w.du16 = take((size_t)T * w.ldr);
+      w.uh = take((size_t)T * w.ldr); w.ul = take((size_t)T * w.ldr);
     }
   }
   w.bytes = off;
   return w;
 }
 
+// Launches the fused-dequant GEMM.  Bop: X (forward) / dY (backward); Bx: the compressed adapter
+// activation [T][ldx] feeding the extra K-blocks (s * x' A forward, dv B^T / lambda_in backward).
 int launch_main(int mode, const QwView& qw, const AdView* ad, const __nv_bfloat16* Bop, const __nv_bfloat16* Bx,
-                int r_pad, const __nv_bfloat16* ex, int64_t T, void* out, int out_dtype, int* status,
-                cudaStream_t st) {
+                int ldx, int64_t T, void* out, int out_dtype, int* status, cudaStream_t st) {
   static bool attr_set[2] = {false, false};
   if (!attr_set[mode]) {
     cudaError_t e = mode == 0
@@ -533,26 +445,27 @@ int launch_main(int mode, const QwView& qw, const AdView* ad, const __nv_bfloat1
   p.M = mode == 0 ? qw.d_out : qw.d_in;
   const int Kq = mode == 0 ? qw.d_in : qw.d_out;
   p.kb_base = (Kq + BK - 1) / BK;
-  p.kb_extra = ad ? r_pad / BK : 0;
+  p.kb_extra = ad ? (ad->r + BK - 1) / BK : 0;
   p.T = (int)T;
   p.m_tiles = (p.M + 2 * BM - 1) / (2 * BM);
   p.n_tiles = (int)((T + BN - 1) / BN);
   p.d_in = qw.d_in; p.d_out = qw.d_out; p.G = qw.G;
   p.alpha = qw.alpha; p.beta = qw.beta;
   for (int j = 0; j < 16; ++j) p.level[j] = qw.level[j];
-  p.ex = ex;
-  p.ex_ld = ad ? (mode == 0 ? r_pad : ad->P) : 0;
+  p.ex = ad ? (mode == 0 ? ad->B : ad->A) : nullptr;
+  p.ex_ld = ad ? (mode == 0 ? ad->Q : ad->r) : 0;
+  p.ex_rows = ad ? ad->r : 0;
   p.lam = ad ? (mode == 0 ? ad->l2 : ad->l1) : 1;
   p.out = out; p.out_dtype = out_dtype; p.status = status;
 
   CUtensorMap tm_b, tm_bx, tm_p;
-  int rc = make_map(&tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Bop, (uint64_t)Kq, (uint64_t)T, (uint64_t)Kq * 2, BK, BN_HALF, true);
+  int rc = make_tensor_map_2d(&tm_b, false, Bop, (uint64_t)Kq, (uint64_t)T, (uint64_t)Kq * 2, BK, BN_HALF, true);
   if (rc) return rc;
-  if (ad) rc = make_map(&tm_bx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Bx, (uint64_t)r_pad, (uint64_t)T, (uint64_t)r_pad * 2, BK, BN_HALF, true);
+  if (ad) rc = make_tensor_map_2d(&tm_bx, false, Bx, (uint64_t)ad->r, (uint64_t)T, (uint64_t)ldx * 2, BK, BN_HALF, true);
   else tm_bx = tm_b;
   if (rc) return rc;
-  if (mode == 0) rc = make_map(&tm_p, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qw.codes, (uint64_t)qw.d_in / 2, (uint64_t)qw.d_out, (uint64_t)qw.d_in / 2, BK / 2, BM, false);
-  else rc = make_map(&tm_p, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qw.codes, (uint64_t)qw.d_in / 2, (uint64_t)qw.d_out, (uint64_t)qw.d_in / 2, BK / 2, BK, false);
+  if (mode == 0) rc = make_tensor_map_2d(&tm_p, true, qw.codes, (uint64_t)qw.d_in / 2, (uint64_t)qw.d_out, (uint64_t)qw.d_in / 2, BK / 2, BM, false);
+  else rc = make_tensor_map_2d(&tm_p, true, qw.codes, (uint64_t)qw.d_in / 2, (uint64_t)qw.d_out, (uint64_t)qw.d_in / 2, BK / 2, BK, false);
   if (rc) return rc;
 
   const int tiles = p.m_tiles * p.n_tiles;                      // one tile per CTA pair
@@ -568,11 +481,29 @@ int launch_main(int mode, const QwView& qw, const AdView* ad, const __nv_bfloat1
   return QBLORA_OK;
 }
 
+int launch_pool(const QwView& qw, const AdView& ad, const __nv_bfloat16* X, int64_t T, const TcWs& w, cudaStream_t st) {
+  const int64_t n = T * ad.P;
+  pool_split_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(X, T, qw.d_in, ad.l1, w.ldp, w.xh, w.xl);
+  count_launch();
+  QB_CUDA(cudaGetLastError());
+  return QBLORA_OK;
+}
+
+// u = x' A with x' = xh + xl: two K-segments against the same (exact, bf16) A
+int launch_u_gemm(const AdView& ad, int64_t T, const TcWs& w, const SgOut& out, int* status, cudaStream_t st) {
+  const SgOperand a_mat{ad.A, ad.r, false};   // (n = rank index, k = p) at A[k * r + n]
+  SgSegment segs[2] = {{{w.xh, w.ldp, true}, a_mat, ad.P}, {{w.xl, w.ldp, true}, a_mat, ad.P}};
+  return small_gemm((int)T, ad.r, segs, 2, out, status, st);
+}
+
 }  // namespace
 
-bool tc_supported(const QwView& qw, const AdView*, int64_t T) {
-  return qw.block_in == BK && qw.block_out == 1 && qw.d_in % BK == 0 && qw.d_out % 8 == 0 && T >= 1 &&
-         T < (int64_t)1 << 31;
+bool tc_supported(const QwView& qw, const AdView* ad, int64_t T) {
+  if (!(qw.block_in == BK && qw.block_out == 1 && qw.d_in % BK == 0 && qw.d_out % 8 == 0 && T >= 1 &&
+        T < (int64_t)1 << 31))
+    return false;
+  // TMA over the adapter matrices needs 16-byte row pitches
+  return !ad || (ad->r % 8 == 0 && ad->Q % 8 == 0);
 }
 
 size_t tc_ws_bytes(int op, const QwView&, const AdView* ad, int64_t T) { return carve(op, ad, T, nullptr).bytes; }
@@ -580,67 +511,66 @@ size_t tc_ws_bytes(int op, const QwView&, const AdView* ad, int64_t T) { return 
 int tc_linear_fwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, int64_t T, void* Y, int y_dtype,
                   char* ws, cudaStream_t st) {
   TcWs w = carve(QBLORA_OP_LINEAR_FWD, ad, T, ws);
-  int rc;
+  int* status = reinterpret_cast<int*>(ws);
   if (ad) {
-    int64_t n = T * ad->P;
-    pool_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(X, T, qw.d_in, ad->l1, w.xp);
-    count_launch();
-    QB_CUDA(cudaGetLastError());
-    if (w.r_pad != ad->r) QB_CUDA(cudaMemsetAsync(w.u16, 0, (size_t)T * w.r_pad * 2, st));
-    // u16 = bf16(s * x' A): the scaling rides on the compressed activation, B stays exact
-    rc = gemm<true, false>(T, ad->r, ad->P, LdF32{w.xp, ad->P, 1}, LdBF16{ad->A, 1, ad->r},
-                           EpBf16Scaled{w.u16, w.r_pad, ad->s, false, nullptr, 0}, st);
+    int rc = launch_pool(qw, *ad, X, T, w, st);
     if (rc) return rc;
-    n = (int64_t)ad->Q * w.r_pad;
-    transpose_pad_cols_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(ad->B, ad->r, ad->Q, w.r_pad, w.bt);
-    count_launch();
-    QB_CUDA(cudaGetLastError());
+    // u16 = bf16(s * x' A): the scaling rides on the compressed activation, B stays exact
+    SgOut out{};
+    out.scaled = w.u16; out.ld16 = w.ldr; out.scale = ad->s; out.divide = false;
+    rc = launch_u_gemm(*ad, T, w, out, status, st);
+    if (rc) return rc;
   }
-  return launch_main(0, qw, ad, X, w.u16, w.r_pad, w.bt, T, Y, y_dtype, reinterpret_cast<int*>(ws), st);
+  return launch_main(0, qw, ad, X, w.u16, w.ldr, T, Y, y_dtype, status, st);
 }
 
 int tc_linear_bwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, const __nv_bfloat16* dY, int64_t T,
                   void* dX, int dx_dtype, float* dA, float* dB, char* ws, cudaStream_t st) {
   TcWs w = carve(QBLORA_OP_LINEAR_BWD, ad, T, ws);
+  int* status = reinterpret_cast<int*>(ws);
   int rc;
   if (ad) {
-    int64_t n = T * ad->Q;
-    dv_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(dY, T, qw.d_out, ad->l2, ad->s, w.dv);
+    const int64_t n = T * ad->Q;
+    dv_split_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(dY, T, qw.d_out, ad->l2, ad->s, w.ldq, w.dvh, w.dvl);
     count_launch();
     QB_CUDA(cudaGetLastError());
-    if (dX && w.r_pad != ad->r) QB_CUDA(cudaMemsetAsync(w.du16, 0, (size_t)T * w.r_pad * 2, st));
-    // du = dv B^T (fp32 for dA) and du16 = bf16(du / lambda_in) for the dX contraction
-    rc = gemm<true, true>(T, ad->r, ad->Q, LdF32{w.dv, ad->Q, 1}, LdBF16{ad->B, ad->Q, 1},
-                          EpBf16Scaled{w.du16, w.r_pad, (float)ad->l1, true, w.du32, ad->r}, st);
-    if (rc) return rc;
+    {  // du = dv B^T (hi + lo for dA) and du16 = bf16(du / lambda_in) for the dX contraction
+      const SgOperand b_mat{ad->B, ad->Q, true};   // (n = rank index, k = q) at B[n * Q + k]
+      SgSegment segs[2] = {{{w.dvh, w.ldq, true}, b_mat, ad->Q}, {{w.dvl, w.ldq, true}, b_mat, ad->Q}};
+      SgOut out{};
+      out.hi = w.duh; out.lo = w.dul; out.scaled = w.du16; out.ld16 = w.ldr; out.scale = (float)ad->l1; out.divide = true;
+      rc = small_gemm((int)T, ad->r, segs, 2, out, status, st);
+      if (rc) return rc;
+    }
     if (dA || dB) {
-      n = T * ad->P;
-      pool_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(X, T, qw.d_in, ad->l1, w.xp);
-      count_launch();
-      QB_CUDA(cudaGetLastError());
+      rc = launch_pool(qw, *ad, X, T, w, st);
+      if (rc) return rc;
     }
     if (dB) {
-      rc = gemm<true, false>(T, ad->r, ad->P, LdF32{w.xp, ad->P, 1}, LdBF16{ad->A, 1, ad->r},
-                             EpStoreF32{w.u32, ad->r}, st);
+      SgOut uo{};
+      uo.hi = w.uh; uo.lo = w.ul; uo.ld16 = w.ldr;
+      rc = launch_u_gemm(*ad, T, w, uo, status, st);
       if (rc) return rc;
-      rc = gemm<false, false>(ad->r, ad->Q, T, LdF32{w.u32, 1, ad->r}, LdF32{w.dv, 1, ad->Q},
-                              EpStoreF32{dB, ad->Q}, st);
+      // dB[k][q] = sum_t u[t][k] dv[t][q]: both operands token-major, i.e. MN-contiguous
+      const SgOperand uh{w.uh, w.ldr, false}, ul{w.ul, w.ldr, false}, dh{w.dvh, w.ldq, false}, dl{w.dvl, w.ldq, false};
+      SgSegment segs[3] = {{uh, dh, (int)T}, {ul, dh, (int)T}, {uh, dl, (int)T}};
+      SgOut out{};
+      out.f32 = dB; out.ld32 = ad->Q;
+      rc = small_gemm(ad->r, ad->Q, segs, 3, out, status, st);
       if (rc) return rc;
     }
     if (dA) {
-      rc = gemm<false, false>(ad->P, ad->r, T, LdF32{w.xp, 1, ad->P}, LdF32{w.du32, 1, ad->r},
-                              EpStoreF32{dA, ad->r}, st);
+      // dA[p][k] = sum_t x'[t][p] du[t][k]
+      const SgOperand xh{w.xh, w.ldp, false}, xl{w.xl, w.ldp, false}, dh{w.duh, w.ldr, false}, dl{w.dul, w.ldr, false};
+      SgSegment segs[3] = {{xh, dh, (int)T}, {xl, dh, (int)T}, {xh, dl, (int)T}};
+      SgOut out{};
+      out.f32 = dA; out.ld32 = ad->r;
+      rc = small_gemm(ad->P, ad->r, segs, 3, out, status, st);
       if (rc) return rc;
-    }
-    if (dX) {
-      n = (int64_t)w.r_pad * ad->P;
-      transpose_pad_rows_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(ad->A, ad->P, ad->r, w.r_pad, w.at);
-      count_launch();
-      QB_CUDA(cudaGetLastError());
     }
   }
   if (!dX) return QBLORA_OK;
-  return launch_main(1, qw, ad, dY, w.du16, w.r_pad, w.at, T, dX, dx_dtype, reinterpret_cast<int*>(ws), st);
+  return launch_main(1, qw, ad, dY, w.du16, w.ldr, T, dX, dx_dtype, status, st);
 }
 
 }  // namespace qb
