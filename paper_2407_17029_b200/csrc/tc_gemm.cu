@@ -406,6 +406,7 @@ inline int round8(int x) { return (x + 7) / 8 * 8; }
 
 struct TcWs {
   __nv_bfloat16 *xh, *xl, *u16, *dvh, *dvl, *duh, *dul, *du16, *uh, *ul;
+  float* partial;   // split-K scratch shared by the dA and dB products
   int ldp, ldq, ldr;
   size_t bytes;
 };
@@ -423,6 +424,9 @@ TcWs carve(int op, const AdView* ad, int64_t T, char* ws) {
       w.dvh = take((size_t)T * w.ldq); w.dvl = take((size_t)T * w.ldq);
       w.duh = take((size_t)T * w.ldr); w.dul = take((size_t)T * w.ldr); w.du16 = take((size_t)T * w.ldr);
       w.uh = take((size_t)T * w.ldr); w.ul = take((size_t)T * w.ldr);
+      const size_t pa = (size_t)small_gemm_splits(ad->P, ad->r, (int)T) * ad->P * ad->r;
+      const size_t pb = (size_t)small_gemm_splits(ad->r, ad->Q, (int)T) * ad->r * ad->Q;
+      w.partial = (float*)take(2 * (pa > pb ? pa : pb));
     }
   }
   w.bytes = off;
@@ -556,7 +560,7 @@ int tc_linear_bwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, co
       SgSegment segs[3] = {{uh, dh, (int)T}, {ul, dh, (int)T}, {uh, dl, (int)T}};
       SgOut out{};
       out.f32 = dB; out.ld32 = ad->Q;
-      rc = small_gemm(ad->r, ad->Q, segs, 3, out, status, st);
+      rc = small_gemm(ad->r, ad->Q, segs, 3, out, status, st, w.partial);
       if (rc) return rc;
     }
     if (dA) {
@@ -565,7 +569,7 @@ int tc_linear_bwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, co
       SgSegment segs[3] = {{xh, dh, (int)T}, {xl, dh, (int)T}, {xh, dl, (int)T}};
       SgOut out{};
       out.f32 = dA; out.ld32 = ad->r;
-      rc = small_gemm(ad->P, ad->r, segs, 3, out, status, st);
+      rc = small_gemm(ad->P, ad->r, segs, 3, out, status, st, w.partial);
       if (rc) return rc;
     }
   }

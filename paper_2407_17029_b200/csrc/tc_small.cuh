@@ -27,7 +27,11 @@ struct SgOut {
 };
 
 // All segments must use the same operand majors.  `status` = device status word (bounded waits).
-int small_gemm(int M, int N, const SgSegment* segs, int nseg, const SgOut& out, int* status, cudaStream_t st);
+// `partial` (optional, fp32 output only): scratch of small_gemm_splits(M, N, K) * M * N floats; the
+// contraction is then split over that many CTAs per output tile and summed in a fixed order.
+int small_gemm(int M, int N, const SgSegment* segs, int nseg, const SgOut& out, int* status, cudaStream_t st,
+               float* partial = nullptr);
+int small_gemm_splits(int M, int N, int K);
 
 // Encodes a 2-D tensor map (shared with the main kernel's host code).
 int make_tensor_map_2d(void* tm, bool is_u8, const void* ptr, uint64_t inner, uint64_t rows, uint64_t pitch_bytes,

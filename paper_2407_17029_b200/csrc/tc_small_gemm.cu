@@ -22,6 +22,8 @@ struct SgMaps {
 struct SgParams {
   int M, N, bn, nseg;
   int kblocks[SG_MAX_SEG];
+  int splits;               // gridDim.z; each z takes a contiguous share of every segment's K-blocks
+  int64_t split_stride;     // elements between the fp32 partial outputs of consecutive z
   int a_kmajor, b_kmajor;
   SgOut out;
   int* status;
@@ -61,7 +63,9 @@ small_gemm_kernel(const __grid_constant__ SgMaps maps, const __grid_constant__ S
       uint32_t it = 0;
       bool ok = true;
       for (int g = 0; g < p.nseg && ok; ++g) {
-        for (int kb = 0; kb < p.kblocks[g]; ++kb, ++it) {
+        const int per = (p.kblocks[g] + p.splits - 1) / p.splits;
+        const int kb0 = (int)blockIdx.z * per, kb1 = min(kb0 + per, p.kblocks[g]);
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % SG_STAGES;
           const uint32_t ph = (it / SG_STAGES) & 1u;
           if (!mbar_wait(empty(s), ph ^ 1u, p.status)) { ok = false; break; }
@@ -94,7 +98,9 @@ small_gemm_kernel(const __grid_constant__ SgMaps maps, const __grid_constant__ S
       uint32_t it = 0;
       bool ok = true;
       for (int g = 0; g < p.nseg && ok; ++g) {
-        for (int kb = 0; kb < p.kblocks[g]; ++kb, ++it) {
+        const int per = (p.kblocks[g] + p.splits - 1) / p.splits;
+        const int kb0 = (int)blockIdx.z * per, kb1 = min(kb0 + per, p.kblocks[g]);
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % SG_STAGES;
           const uint32_t ph = (it / SG_STAGES) & 1u;
           if (!mbar_wait(full(s), ph, p.status)) { ok = false; break; }
@@ -110,12 +116,18 @@ small_gemm_kernel(const __grid_constant__ SgMaps maps, const __grid_constant__ S
           tc_commit(empty(s));
         }
       }
-      if (ok) tc_commit(accfull);
+      if (ok) tc_commit(accfull);   // (a share with no K-blocks still arrives: nothing was issued)
     }
   } else {
     // epilogue: thread = output row; 32 columns per TMEM load
     const int q = warp & 3;
     const int m = m0 + q * 32 + lane;
+    int my_kblocks = 0;   // a share of the split that received no K-block contributes zeros
+    for (int g = 0; g < p.nseg; ++g) {
+      const int per = (p.kblocks[g] + p.splits - 1) / p.splits;
+      const int kb0 = (int)blockIdx.z * per, kb1 = min(kb0 + per, p.kblocks[g]);
+      my_kblocks += max(kb1 - kb0, 0);
+    }
     if (mbar_wait(accfull, 0, p.status)) {
       tc_fence_after();
       for (int c = 0; c < p.bn / 32; ++c) {
@@ -123,10 +135,14 @@ small_gemm_kernel(const __grid_constant__ SgMaps maps, const __grid_constant__ S
         if (nb >= p.N) break;
         uint32_t v[32];
         tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), v);
+        if (my_kblocks == 0) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = 0u;
+        }
         if (m >= p.M) continue;
         const SgOut& o = p.out;
         if (o.f32) {
-          float* dst = o.f32 + (int64_t)m * o.ld32 + nb;
+          float* dst = o.f32 + (int64_t)blockIdx.z * p.split_stride + (int64_t)m * o.ld32 + nb;
           if ((o.ld32 & 3) == 0 && nb + 32 <= p.N) {
 #pragma unroll
             for (int j = 0; j < 32; j += 4)
@@ -138,15 +154,36 @@ small_gemm_kernel(const __grid_constant__ SgMaps maps, const __grid_constant__ S
           }
         }
         if (o.hi || o.lo || o.scaled) {
+          const int64_t row = (int64_t)m * o.ld16 + nb;
+          if ((o.ld16 & 7) == 0 && nb + 32 <= p.N) {   // 16-byte stores of eight bf16
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            if (nb + j >= p.N) break;
-            const float x = __uint_as_float(v[j]);
-            const int64_t idx = (int64_t)m * o.ld16 + nb + j;
-            const __nv_bfloat16 h = __float2bfloat16_rn(x);
-            if (o.hi) o.hi[idx] = h;
-            if (o.lo) o.lo[idx] = __float2bfloat16_rn(x - __bfloat162float(h));
-            if (o.scaled) o.scaled[idx] = __float2bfloat16_rn(o.divide ? __fdiv_rn(x, o.scale) : x * o.scale);
+            for (int j = 0; j < 32; j += 8) {
+              uint32_t h[4], l[4], sc[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const float x0 = __uint_as_float(v[j + 2 * e]), x1 = __uint_as_float(v[j + 2 * e + 1]);
+                const __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
+                h[e] = *reinterpret_cast<const uint32_t*>(&hh);
+                const __nv_bfloat162 ll = __floats2bfloat162_rn(x0 - __low2float(hh), x1 - __high2float(hh));
+                l[e] = *reinterpret_cast<const uint32_t*>(&ll);
+                const __nv_bfloat162 ss = o.divide ? __floats2bfloat162_rn(__fdiv_rn(x0, o.scale), __fdiv_rn(x1, o.scale))
+                                                   : __floats2bfloat162_rn(x0 * o.scale, x1 * o.scale);
+                sc[e] = *reinterpret_cast<const uint32_t*>(&ss);
+              }
+              if (o.hi) *reinterpret_cast<uint4*>(o.hi + row + j) = make_uint4(h[0], h[1], h[2], h[3]);
+              if (o.lo) *reinterpret_cast<uint4*>(o.lo + row + j) = make_uint4(l[0], l[1], l[2], l[3]);
+              if (o.scaled) *reinterpret_cast<uint4*>(o.scaled + row + j) = make_uint4(sc[0], sc[1], sc[2], sc[3]);
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              if (nb + j >= p.N) break;
+              const float x = __uint_as_float(v[j]);
+              const __nv_bfloat16 h = __float2bfloat16_rn(x);
+              if (o.hi) o.hi[row + j] = h;
+              if (o.lo) o.lo[row + j] = __float2bfloat16_rn(x - __bfloat162float(h));
+              if (o.scaled) o.scaled[row + j] = __float2bfloat16_rn(o.divide ? __fdiv_rn(x, o.scale) : x * o.scale);
+            }
           }
         }
       }
@@ -158,6 +195,16 @@ small_gemm_kernel(const __grid_constant__ SgMaps maps, const __grid_constant__ S
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(256) : "memory");
   }
+}
+
+// out[m][n] = sum over z (in order) of part[z][m][n]
+__global__ void reduce_splits_kernel(const float* __restrict__ part, int splits, int64_t MN, int N, float* __restrict__ out,
+                                     int64_t ld) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= MN) return;
+  float acc = 0.0f;
+  for (int z = 0; z < splits; ++z) acc += part[(int64_t)z * MN + idx];
+  out[(idx / N) * ld + idx % N] = acc;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -199,7 +246,21 @@ int make_tensor_map_2d(void* tm, bool is_u8, const void* ptr, uint64_t inner, ui
   return r == CUDA_SUCCESS ? QBLORA_OK : QBLORA_ERR_CUDA;
 }
 
-int small_gemm(int M, int N, const SgSegment* segs, int nseg, const SgOut& out, int* status, cudaStream_t st) {
+int small_gemm_splits(int M, int N, int K) {
+  const int n64 = (N + 63) / 64 * 64;
+  const int bn = n64 < 256 ? n64 : 256;
+  const int tiles = ((N + bn - 1) / bn) * ((M + SG_BM - 1) / SG_BM);
+  const int kb = (K + SG_BK - 1) / SG_BK;
+  int want = 148 / tiles;
+  if (want > 32) want = 32;
+  if (want > kb) want = kb;
+  if (want < 1) want = 1;
+  const int per = (kb + want - 1) / want;
+  return (kb + per - 1) / per;   // every share owns at least one K-block
+}
+
+int small_gemm(int M, int N, const SgSegment* segs, int nseg, const SgOut& out, int* status, cudaStream_t st,
+               float* partial) {
   if (nseg < 1 || nseg > SG_MAX_SEG || M < 1 || N < 1) return QBLORA_ERR_INVALID_ARG;
   static bool attr_set = false;
   if (!attr_set) {
@@ -226,10 +287,27 @@ int small_gemm(int M, int N, const SgSegment* segs, int nseg, const SgOut& out, 
   for (int g = nseg; g < SG_MAX_SEG; ++g) { maps.a[g] = maps.a[0]; maps.b[g] = maps.b[0]; p.kblocks[g] = 0; }
   p.out = out;
   p.status = status;
-  dim3 grid((unsigned)((N + p.bn - 1) / p.bn), (unsigned)((M + SG_BM - 1) / SG_BM));
+  p.splits = 1;
+  p.split_stride = 0;
+  if (partial) {   // split the contraction; only the fp32 output is supported in this mode
+    if (!out.f32 || out.hi || out.lo || out.scaled) return QBLORA_ERR_INVALID_ARG;
+    p.splits = small_gemm_splits(M, N, segs[0].K);
+    if (p.splits > 1) {
+      p.out.f32 = partial;
+      p.out.ld32 = N;
+      p.split_stride = (int64_t)M * N;
+    }
+  }
+  dim3 grid((unsigned)((N + p.bn - 1) / p.bn), (unsigned)((M + SG_BM - 1) / SG_BM), (unsigned)p.splits);
   small_gemm_kernel<<<grid, SG_THREADS, SG_SMEM, st>>>(maps, p);
   count_launch();
   QB_CUDA(cudaGetLastError());
+  if (p.splits > 1) {
+    const int64_t MN = (int64_t)M * N;
+    reduce_splits_kernel<<<(unsigned)((MN + 255) / 256), 256, 0, st>>>(partial, p.splits, MN, N, out.f32, out.ld32);
+    count_launch();
+    QB_CUDA(cudaGetLastError());
+  }
   return QBLORA_OK;
 }
 
