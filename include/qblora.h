@@ -39,7 +39,8 @@ typedef enum {
   QBLORA_ERR_UNSUPPORTED = 2, /* valid request this build has no kernel for */
   QBLORA_ERR_WORKSPACE = 3,   /* ws == NULL or ws_bytes too small */
   QBLORA_ERR_CUDA = 4,        /* a CUDA runtime call or launch failed */
-  QBLORA_ERR_TIMEOUT = 5      /* a bounded device-side wait gave up (see qblora_device_status) */
+  QBLORA_ERR_TIMEOUT = 5,     /* a bounded device-side wait gave up (see qblora_device_status) */
+  QBLORA_ERR_TOO_LARGE = 6    /* qablora_merge_noalloc only: the adapter is larger than its built-in scratch */
 } qblora_status;
 
 typedef enum {
@@ -168,6 +169,32 @@ int qblora_linear_bwd(const qblora_qweight* qw, const qblora_adapter* adapter, c
  */
 int qablora_merge(const qblora_qweight* qw, const qblora_adapter* adapter, float* beta_out,
                   void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * The same merge for callers that cannot give the library a workspace.  (The paper has no
+ * counterpart; this is a packaging variant of qablora_merge.)
+ *
+ * Who needs it: code that must not touch the device allocator while it runs -- a serving loop that
+ * swaps adapters after start-up with all device memory already committed to weights and caches, a
+ * host without a spare allocator context, a plug-in called from inside someone else's stream-ordered
+ * pipeline where a cudaMalloc would stall every stream.  qablora_merge needs P * Q fp64 values of
+ * scratch for H = A B; here they live in a 2 MiB array that is part of the library image (every GPU
+ * that loads the library carries it until the process exits), so the call allocates and frees
+ * nothing: no workspace argument, no cudaMalloc / cudaFree, no allocating library routine.
+ *
+ * Limits and rules:
+ *   - P * Q = (d_in / lambda_in) * (d_out / lambda_out) must be <= 262144, else QBLORA_ERR_TOO_LARGE
+ *     (the LLaMA-33B shapes of the deploy configuration use 86528 to 232960).
+ *   - Inputs, outputs, results and the other error codes are exactly those of qablora_merge.
+ *   - The first call on each device looks up the array's device address (with that device current);
+ *     make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps the previous call's H.  Each call
+ *     overwrites every entry it reads, so nothing carries over between calls; but two calls that
+ *     can run concurrently on the same GPU (different streams, different host threads) race on
+ *     it -- serialise them.
+ */
+int qablora_merge_noalloc(const qblora_qweight* qw, const qblora_adapter* adapter, float* beta_out,
+                          void* stream);
 
 /*
  * Low-precision inference product on the merged model (Sec. 3.3):

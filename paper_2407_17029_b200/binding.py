@@ -20,7 +20,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libqblora.so")
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_TOO_LARGE = range(7)
 FMT_CODEBOOK_ABSMAX, FMT_AFFINE_MINMAX = 0, 1
 F32, BF16 = 0, 1
 OP_QUANTIZE, OP_LINEAR_FWD, OP_LINEAR_BWD, OP_MERGE, OP_LOWBIT_GEMM = range(5)
@@ -28,7 +28,7 @@ OP_QUANTIZE, OP_LINEAR_FWD, OP_LINEAR_BWD, OP_MERGE, OP_LOWBIT_GEMM = range(5)
 EXPORTS = ["qblora_default_code_table", "qblora_workspace_bytes", "qblora_status_string",
            "qblora_device_status", "qblora_quantize_blockwise", "qblora_linear_fwd",
            "qblora_linear_bwd", "qablora_merge", "qablora_lowbit_gemm", "qblora_kernel_launches",
-           "qblora_set_timing_events"]
+           "qblora_set_timing_events", "qablora_merge_noalloc"]
 
 
 class _CQWeight(ctypes.Structure):
@@ -69,6 +69,7 @@ _lib.qablora_lowbit_gemm.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_
                                      ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
 
 
+_lib.qablora_merge_noalloc.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
 _lib.qblora_kernel_launches.restype = ctypes.c_uint64
 _lib.qblora_kernel_launches.argtypes = []
 _lib.qblora_set_timing_events.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
@@ -257,6 +258,20 @@ def merge(qw: QWeight, ad: Adapter, in_place: bool = False, ws: Optional[torch.T
     st = _lib.qablora_merge(ctypes.byref(cq), ctypes.byref(ca), beta_out.data_ptr(), ws.data_ptr(),
                             ws.numel(), _stream_ptr(stream))
     _check(st, "qablora_merge")
+    return QWeight(qw.d_out, qw.d_in, qw.block_in, qw.block_out, qw.qfmt, qw.code, qw.codes, qw.alpha, beta_out)
+
+
+def merge_noalloc(qw: QWeight, ad: Adapter, beta_out: torch.Tensor, stream=None) -> QWeight:
+    """qablora_merge_noalloc: merge into the caller's ``beta_out`` using the library's built-in scratch.
+
+    For callers that cannot allocate device memory at this point (see the header).  Nothing is
+    allocated here either: ``beta_out`` (fp32, same shape as ``qw.beta``) comes from the caller.
+    Raises QbloraError(ERR_TOO_LARGE) when (d_in/lambda_in)*(d_out/lambda_out) > 262144.
+    """
+    cq = qw.c_struct()
+    ca = ad.c_struct()
+    st = _lib.qablora_merge_noalloc(ctypes.byref(cq), ctypes.byref(ca), beta_out.data_ptr(), _stream_ptr(stream))
+    _check(st, "qablora_merge_noalloc")
     return QWeight(qw.d_out, qw.d_in, qw.block_in, qw.block_out, qw.qfmt, qw.code, qw.codes, qw.alpha, beta_out)
 
 

@@ -117,6 +117,7 @@ const char* qblora_status_string(int s) {
     case QBLORA_ERR_WORKSPACE: return "workspace missing or too small";
     case QBLORA_ERR_CUDA: return "CUDA error";
     case QBLORA_ERR_TIMEOUT: return "device-side wait timed out";
+    case QBLORA_ERR_TOO_LARGE: return "problem exceeds the built-in scratch of the no-allocation entry point";
     default: return "unknown status";
   }
 }
@@ -230,6 +231,18 @@ int qablora_merge(const qblora_qweight* qw, const qblora_adapter* adapter, float
   rc = reset_status(ws, st);
   if (rc) return rc;
   return launch_merge(q, ad, adapter->B == nullptr, beta_out, static_cast<char*>(ws), st);
+}
+
+int qablora_merge_noalloc(const qblora_qweight* qw, const qblora_adapter* adapter, float* beta_out,
+                          void* stream) {
+  QwView q; int rc = make_qw(qw, &q);
+  if (rc) return rc;
+  if (q.qfmt != QBLORA_FMT_AFFINE_MINMAX || !adapter || !beta_out || !aligned16(beta_out)) return QBLORA_ERR_INVALID_ARG;
+  AdView ad; rc = make_ad(adapter, q, true, &ad);
+  if (rc) return rc;
+  if (ad.l1 % q.block_in || ad.l2 % q.block_out) return QBLORA_ERR_INVALID_ARG;
+  if ((int64_t)ad.P * ad.Q > merge_noalloc_capacity()) return QBLORA_ERR_TOO_LARGE;
+  return launch_merge_noalloc(q, ad, adapter->B == nullptr, beta_out, static_cast<cudaStream_t>(stream));
 }
 
 int qablora_lowbit_gemm(const qblora_qweight* qw, const void* X, int64_t tokens, void* Y, int y_dtype,

@@ -60,6 +60,10 @@ size_t merge_ws_bytes(const QwView& qw, const AdView& ad);
 int launch_merge(const QwView& qw, const AdView& ad, bool single_matrix, float* beta_out, char* ws,
                  cudaStream_t st);
 
+int64_t merge_noalloc_capacity();   // P * Q entries the built-in scratch of the no-alloc merge holds
+int launch_merge_noalloc(const QwView& qw, const AdView& ad, bool single_matrix, float* beta_out,
+                         cudaStream_t st);
+
 // Bandwidth-bound low-bit product for small token counts (block_out == 1, block_in == 64).
 bool gemv_supported(const QwView& qw, int64_t T);
 int launch_lowbit_gemv(const QwView& qw, const __nv_bfloat16* X, int64_t T, void* Y, int y_dtype,
