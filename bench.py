@@ -27,6 +27,10 @@ if ROOT not in sys.path:
 
 from paper_2407_17029_b200 import synth  # noqa: E402
 
+# dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, per launch, from the ncu
+# capture summarised in profiles/ncu_full_tc_dq_gemm_C2.md (set to None when that kernel changes)
+MEASURED_DRAM_TRAFFIC = {("C2", "GA"): 27.6e6 + 0.27e6}
+
 METRIC = "fused 4-bit+BLoRA linear fwd+bwd TFLOP/s & low-bit GEMM GB/s, % of roofline"
 
 
@@ -301,7 +305,7 @@ def run_gpu(args, wl, geom):
                          "achieved": dom_flops / (dom_ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops_sustained"],
                          "peak_kind": f"bf16 dense, sustained, {peaks['source']}", "unit": "TFLOP/s",
                          "frac": dom_flops / (dom_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
-                         "traffic": None, "ms_per_launch": dom_ms},
+                         "traffic": MEASURED_DRAM_TRAFFIC.get((wl.name, geom.name)), "ms_per_launch": dom_ms},
             "step_flops": flops_step}
 
     if rank == 0 and not args.no_extras:
