@@ -349,6 +349,55 @@ __device__ __forceinline__ void store_split(float x, __nv_bfloat16* hi, __nv_bfl
   hi[idx] = h;
   lo[idx] = __float2bfloat16_rn(x - __bfloat162float(h));
 }
+// Fast path of both segment sums below: out[t][w] = f(sum of `lam` consecutive bf16 of row t), f = /lam
+// (AvgPool) or *scale (adjoint of repeat_interleave), written as a bf16 hi + lo pair.  One 16-byte load
+// (8 elements) per thread; windows wider than a chunk are finished with warp shuffles.  Needs width % 8
+// == 0 and lam in {1, 2, 4} or 8 * 2^k <= 256 with chunks-per-row % (lam / 8) == 0 (true when lam | width).
+template <bool DIVIDE>
+__global__ void __launch_bounds__(256) segsum_split_kernel(const __nv_bfloat16* __restrict__ src, int64_t rows, int width,
+                                                           int lam, float scale, int ld_out,
+                                                           __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+  const int chunks_per_row = width >> 3;
+  const int64_t total = rows * chunks_per_row;
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const bool live = idx < total;
+  float v[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) v[e] = 0.0f;
+  int64_t t = 0; int c = 0;
+  if (live) {
+    t = idx / chunks_per_row; c = (int)(idx - t * chunks_per_row);
+    const uint4 q4 = __ldg(reinterpret_cast<const uint4*>(src + t * width) + c);
+    const uint32_t w[4] = {q4.x, q4.y, q4.z, q4.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) { v[2 * e] = __uint_as_float(w[e] << 16); v[2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u); }
+  }
+  if (lam >= 8) {
+    float sacc = ((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7]));
+    const int lanes = lam >> 3;   // power of two, <= 32; windows never straddle a warp (256 % lanes == 0, rows aligned)
+    for (int off = 1; off < lanes; off <<= 1) sacc += __shfl_xor_sync(0xffffffffu, sacc, off);
+    if (live && (c & (lanes - 1)) == 0) {
+      const float r = DIVIDE ? __fdiv_rn(sacc, (float)lam) : scale * sacc;
+      store_split(r, hi, lo, t * ld_out + c / lanes);
+    }
+  } else if (live) {
+    const int per = 8 / lam;      // windows inside this chunk
+    for (int j = 0; j < per; ++j) {
+      float sacc = 0.0f;
+      for (int e = 0; e < lam; ++e) sacc += v[j * lam + e];
+      const float r = DIVIDE ? __fdiv_rn(sacc, (float)lam) : scale * sacc;
+      store_split(r, hi, lo, t * ld_out + c * per + j);
+    }
+  }
+}
+inline bool segsum_fast_ok(int width, int lam) {
+  if (width % 8) return false;
+  if (lam == 1 || lam == 2 || lam == 4) return true;
+  if (lam % 8) return false;
+  const int lanes = lam / 8;
+  return lanes <= 32 && (lanes & (lanes - 1)) == 0 && (width / 8) % lanes == 0;
+}
+
 // x'[t][p] = AvgPool_{lambda_in}(X) (Sec. 3.2) as a bf16 hi + lo pair (hi + lo carries ~16 mantissa bits)
 __global__ void pool_split_kernel(const __nv_bfloat16* __restrict__ X, int64_t T, int d_in, int l1, int ldp,
                                   __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
@@ -487,7 +536,12 @@ int launch_main(int mode, const QwView& qw, const AdView* ad, const __nv_bfloat1
 
 int launch_pool(const QwView& qw, const AdView& ad, const __nv_bfloat16* X, int64_t T, const TcWs& w, cudaStream_t st) {
   const int64_t n = T * ad.P;
-  pool_split_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(X, T, qw.d_in, ad.l1, w.ldp, w.xh, w.xl);
+  if (segsum_fast_ok(qw.d_in, ad.l1)) {
+    const int64_t chunks = T * (qw.d_in / 8);
+    segsum_split_kernel<true><<<(unsigned)((chunks + 255) / 256), 256, 0, st>>>(X, T, qw.d_in, ad.l1, 0.0f, w.ldp, w.xh, w.xl);
+  } else {
+    pool_split_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(X, T, qw.d_in, ad.l1, w.ldp, w.xh, w.xl);
+  }
   count_launch();
   QB_CUDA(cudaGetLastError());
   return QBLORA_OK;
@@ -535,7 +589,12 @@ int tc_linear_bwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, co
   int rc;
   if (ad) {
     const int64_t n = T * ad->Q;
-    dv_split_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(dY, T, qw.d_out, ad->l2, ad->s, w.ldq, w.dvh, w.dvl);
+    if (segsum_fast_ok(qw.d_out, ad->l2)) {
+      const int64_t chunks = T * (qw.d_out / 8);
+      segsum_split_kernel<false><<<(unsigned)((chunks + 255) / 256), 256, 0, st>>>(dY, T, qw.d_out, ad->l2, ad->s, w.ldq, w.dvh, w.dvl);
+    } else {
+      dv_split_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(dY, T, qw.d_out, ad->l2, ad->s, w.ldq, w.dvh, w.dvl);
+    }
     count_launch();
     QB_CUDA(cudaGetLastError());
     {  // du = dv B^T (hi + lo for dA) and du16 = bf16(du / lambda_in) for the dX contraction

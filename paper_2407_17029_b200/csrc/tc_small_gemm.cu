@@ -272,6 +272,8 @@ int small_gemm(int M, int N, const SgSegment* segs, int nseg, const SgOut& out, 
   p.M = M; p.N = N; p.nseg = nseg;
   const int n64 = (N + 63) / 64 * 64;
   p.bn = n64 < 256 ? n64 : 256;
+  // few row tiles and no split: narrower column tiles put more CTAs to work (the kernel is latency-bound)
+  while (!partial && p.bn > 64 && ((N + p.bn - 1) / p.bn) * ((M + SG_BM - 1) / SG_BM) < 96 && (p.bn / 2) % 64 == 0) p.bn /= 2;
   p.a_kmajor = segs[0].a.k_contig ? 1 : 0;
   p.b_kmajor = segs[0].b.k_contig ? 1 : 0;
   for (int g = 0; g < nseg; ++g) {
