@@ -59,20 +59,46 @@ struct TcParams {
   int* status;
 };
 
-// Eight 4-bit codes (one 32-bit word, code e in bits 4e..4e+3) -> eight bf16 values alpha*level+beta.
-// `tabv` holds level[lane & 15] in every lane, so a warp shuffle indexed by the raw shifted word
-// (the source lane is taken modulo 32, and lanes 16-31 mirror lanes 0-15) is the table lookup.
-// The product is formed in fp32 and rounded once to bf16.
-__device__ __forceinline__ void dequant_word(uint32_t w, float tabv, float alpha, float beta, uint32_t (&o)[4]) {
-  float v[8];
-#pragma unroll
-  for (int e = 0; e < 8; ++e) {
-    const float lv = __shfl_sync(0xffffffffu, tabv, (int)(w >> (4 * e)));
-    v[e] = fmaf(alpha, lv, beta);
-  }
-#pragma unroll
-  for (int e = 0; e < 4; ++e) o[e] = pack_bf16x2(v[2 * e], v[2 * e + 1]);
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+  uint32_t r;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
+  return r;
 }
+
+// Per-block dequantization table kept in registers.  The sixteen values bf16(alpha * level[c] + beta)
+// of one quantization block (fp32 product, one rounding) are split into a low-byte plane and a
+// high-byte plane of four registers each; a 4-bit code then selects its two bytes with byte-permute
+// instructions only.  Measured on this part a byte permute issues at the rate of any integer ALU
+// operation (2 cycles per warp instruction per scheduler) while a warp shuffle takes 4 and occupies
+// the shared-memory data pipe the tensor core's operand fetch needs, so this lookup (21 ALU ops per
+// 8 codes, table build amortised over 64) beats a shuffle-indexed table (8 shuffles + 7 shifts +
+// 8 FMAs + 4 conversions per 8 codes).
+struct BlockTable {
+  uint32_t lp[4], hp[4];
+  __device__ __forceinline__ void build(const float (&level)[16], float alpha, float beta) {
+#pragma unroll
+    for (int m = 0; m < 4; ++m) {
+      const uint32_t p0 = pack_bf16x2(fmaf(alpha, level[4 * m + 0], beta), fmaf(alpha, level[4 * m + 1], beta));
+      const uint32_t p1 = pack_bf16x2(fmaf(alpha, level[4 * m + 2], beta), fmaf(alpha, level[4 * m + 3], beta));
+      lp[m] = prmt(p0, p1, 0x6420u);
+      hp[m] = prmt(p0, p1, 0x7531u);
+    }
+  }
+  // four codes in the low 16 bits of `a` (each masked to 3 bits) / `s2` (merge selector) -> 4 bf16
+  __device__ __forceinline__ void half(uint32_t a, uint32_t s2, uint32_t& o01, uint32_t& o23) const {
+    const uint32_t lo = prmt(prmt(lp[0], lp[1], a), prmt(lp[2], lp[3], a), s2);
+    const uint32_t hi = prmt(prmt(hp[0], hp[1], a), prmt(hp[2], hp[3], a), s2);
+    o01 = prmt(lo, hi, 0x5140u);
+    o23 = prmt(lo, hi, 0x7362u);
+  }
+  // eight codes (code e in bits 4e..4e+3 of w) -> eight bf16 values in element order
+  __device__ __forceinline__ void lookup8(uint32_t w, uint32_t (&o)[4]) const {
+    const uint32_t a = w & 0x77777777u;                               // index within an 8-entry half
+    const uint32_t s2 = ((w >> 1) & 0x44444444u) | 0x32103210u;       // byte j: j + 4 * (code >> 3)
+    half(a, s2, o[0], o[1]);
+    half(a >> 16, s2 >> 16, o[2], o[3]);
+  }
+};
 
 template <int MODE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
@@ -193,7 +219,6 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
     // quantization block (64 codes, one alpha/beta) of the tile per K-block.
     const int g = (warp - 2) >> 2;
     const int d = tid - 64 - 128 * g;
-    const float tabv = p.level[lane & 15];
     const uint32_t leader_peer = map_to_cta(peer(0), 0);
     bool ok = true;
     uint32_t it = 0;
@@ -225,8 +250,9 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
               if (p.beta) be = __ldg(p.beta + (int64_t)o * p.G + blk);
             }
           }
-          const bool landed = mbar_wait(full(s), ph, p.status) && mbar_wait(empty(s), ph ^ 1u, p.status);
-          if (!__all_sync(0xffffffffu, landed)) { ok = false; break; }   // keep the warp together for the shuffles
+          BlockTable tab;
+          tab.build(p.level, al, be);
+          if (!mbar_wait(full(s), ph, p.status) || !mbar_wait(empty(s), ph ^ 1u, p.status)) { ok = false; break; }
           const uint8_t* src = gP + s * P_BYTES + d * 32;
           const uint4 q0 = *reinterpret_cast<const uint4*>(src);
           const uint4 q1 = *reinterpret_cast<const uint4*>(src + 16);
@@ -234,7 +260,7 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             uint32_t o4[4];
-            dequant_word(w[j], tabv, al, be, o4);
+            tab.lookup8(w[j], o4);
             st_shared_v4(dst + (((uint32_t)j ^ xr) << 4), o4[0], o4[1], o4[2], o4[3]);
           }
         } else {
