@@ -254,10 +254,11 @@ int qablora_lowbit_gemm(const qblora_qweight* qw, const void* X, int64_t tokens,
   const size_t need = ws_bytes_impl(QBLORA_OP_LOWBIT_GEMM, q, nullptr, tokens);
   if (!ws || !aligned16(ws) || ws_bytes < need) return QBLORA_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const __nv_bfloat16* Xb = static_cast<const __nv_bfloat16*>(X);
+  // the decode kernel clears the status word itself: one launch per call
+  if (gemv_supported(q, tokens)) return launch_lowbit_gemv(q, Xb, tokens, Y, y_dtype, static_cast<int*>(ws), st);
   rc = reset_status(ws, st);
   if (rc) return rc;
-  const __nv_bfloat16* Xb = static_cast<const __nv_bfloat16*>(X);
-  if (gemv_supported(q, tokens)) return launch_lowbit_gemv(q, Xb, tokens, Y, y_dtype, st);
   if (!force_general() && tc_supported(q, nullptr, tokens))
     return tc_linear_fwd(q, nullptr, Xb, tokens, Y, y_dtype, static_cast<char*>(ws), st);
   return simt_linear_fwd(q, nullptr, Xb, tokens, Y, y_dtype, static_cast<char*>(ws), st);

@@ -67,7 +67,7 @@ int launch_merge_noalloc(const QwView& qw, const AdView& ad, bool single_matrix,
 // Bandwidth-bound low-bit product for small token counts (block_out == 1, block_in == 64).
 bool gemv_supported(const QwView& qw, int64_t T);
 int launch_lowbit_gemv(const QwView& qw, const __nv_bfloat16* X, int64_t T, void* Y, int y_dtype,
-                       cudaStream_t st);
+                       int* status, cudaStream_t st);
 
 // Tensor-core path (tcgen05 / TMEM / TMA): block_in == 64, block_out == 1.
 bool tc_supported(const QwView& qw, const AdView* ad, int64_t T);

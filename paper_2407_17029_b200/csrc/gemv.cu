@@ -1,28 +1,41 @@
 // Low-bit product for small token counts (decode, T <= 16):
 //   Y[t][o] = sum_i X[t][i] * (alpha[o][i/64] * c[o][i] + beta'[o][i/64])            (Sec. 3.3)
-// The packed weight is streamed exactly once (DRAM traffic = codes + alpha + beta).  Measured: the
-// kernel is bound by instruction issue and load latency (about 120 warp instructions per 16 rows x 64
-// codes, four warps per scheduler), reaching 25-35 % of the HBM copy bandwidth at T = 1.
+// The packed weight is streamed exactly once (DRAM traffic = codes + alpha + beta).
 //
-// Mapping.  A CTA of eight warps owns 16 output rows; warp w takes the w-th eighth of the 64-wide
-// quantization groups of those rows, and the eight partial results are summed through shared memory
-// in warp order (deterministic).  Inside a warp the work is shaped for mma.sync.m16n8k16 (bf16, fp32
-// accumulate): the 16 rows are the M
-// side, up to 8 tokens per N tile.  A thread (g = lane / 4, tg = lane % 4) loads, for rows g and
-// g + 8, the 8 bytes holding codes 16 tg .. 16 tg + 15 of the current group and turns each 32-bit word
-// into four bf16 pairs (128 + c) with one logic op per pair (the nibbles land in the mantissa of
-// 128.0).  Because the order of the k index inside an MMA is free as long as both operands agree,
-// nibble pairs (e, e + 4) are used as they fall out of the word and the token operand is permuted to
-// match with byte permutes.  A second MMA chain with A = 1.0 yields S = sum of x over the group in
-// the accumulator layout, and the group contributes
+// Structure.  One persistent CTA per SM.  A producer thread streams tiles of 32 output rows x 16
+// quantization groups (16 KB of codes as four 128-byte-swizzled TMA boxes, plus the 32 x 16 alpha
+// and beta values) through a shared-memory ring guarded by mbarriers, so no compute warp ever waits
+// on DRAM latency or does global address arithmetic for the weight.  Each of the sixteen compute
+// warps owns one of the tile's 16 groups and all 32 rows (two MMA row tiles), so the token operand
+// of a group is fetched once per warp and tile.  Partial sums stay in registers across the K tiles
+// of a row block and are summed through shared memory in warp order at the end of the block
+// (deterministic).
+//
+// Arithmetic.  The work of a warp is shaped for mma.sync.m16n8k16 (bf16, fp32 accumulate): 16 rows
+// are the M side, up to 8 tokens per N tile.  A thread (g = lane / 4, tg = lane % 4) reads, for rows
+// g + 8 q (q = 0..3), the 8 bytes holding codes 16 tg .. 16 tg + 15 of the group and turns each
+// 32-bit word into four bf16 pairs (128 + c) with one logic op per pair (the nibbles land in the
+// mantissa of 128.0).  Because the order of the k index inside an MMA is free as long as both
+// operands agree, nibble pairs (e, e + 4) are used as they fall out of the word and the token operand
+// is permuted to match with byte permutes.  With S = sum of x over the group (computed once per CTA
+// into shared memory), the group contributes
 //   alpha * sum((128 + c) x) + (beta - 128 alpha) * S  =  alpha * sum(c x) + beta * S.
-#include "common.cuh"
+// When T * D_in is small enough the permuted token fragments are also kept in shared memory for the
+// life of the CTA; otherwise they are rebuilt per group from global x (L1-resident).
+#include "tc_ptx.cuh"
+#include "tc_small.cuh"
 
 namespace qb {
+using namespace ptx;
 namespace {
 
-constexpr int GV_WARPS = 8;
-constexpr int GV_ROWS = 16;
+constexpr int GT_ROWS = 32;            // rows per tile (two MMA row tiles)
+constexpr int GT_GROUPS = 16;          // quantization groups per tile (1024 codes per row), one per warp
+constexpr int GT_WARPS = 16;           // compute warps; warp 16 is the producer
+constexpr int GT_THREADS = (GT_WARPS + 1) * 32;
+constexpr int GT_CODE_BYTES = GT_ROWS * GT_GROUPS * 32;   // 16 KB = four boxes of [32 rows][128 B]
+constexpr int GT_SCALE_BYTES = GT_ROWS * GT_GROUPS * 4;   // 2 KB each for alpha and beta
+constexpr int GT_STAGE_BYTES = GT_CODE_BYTES + 2 * GT_SCALE_BYTES;
 
 __device__ __forceinline__ uint32_t gv_prmt(uint32_t a, uint32_t b, uint32_t sel) {
   uint32_t r;
@@ -31,140 +44,509 @@ __device__ __forceinline__ uint32_t gv_prmt(uint32_t a, uint32_t b, uint32_t sel
 }
 __device__ __forceinline__ void gv_mma(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                        uint32_t b1) {
-  asm volatile(
+  asm(
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+// first MMA of a chain: accumulator input is zero
+__device__ __forceinline__ void gv_mma0(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                        uint32_t b1) {
+  asm(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+      : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.0f));
+}
+// (w & m) | c as ONE three-input logic op.  Mask and magic are passed in registers: written with two
+// literals the compiler emits two logic ops (one literal each), which costs a third of the kernel.
+__device__ __forceinline__ uint32_t gv_and_or(uint32_t w, uint32_t m, uint32_t c) {
+  uint32_t v;
+  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(v) : "r"(w), "r"(m), "r"(c));
+  return v;
+}
+// constants of the unpackers, kept in registers (see gv_and_or)
+struct GvConst {
+  uint32_t m0, m1, c;
+  __device__ __forceinline__ GvConst(uint32_t m0_, uint32_t m1_, uint32_t c_) : m0(m0_), m1(m1_), c(c_) {
+    asm volatile("" : "+r"(m0), "+r"(m1), "+r"(c));
+  }
+};
 // word of 8 codes -> (128 + c) bf16 pairs: v[e] = (code e, code e + 4), e = 0..3
-__device__ __forceinline__ void gv_unpack(uint32_t w, uint32_t (&v)[4]) {
-  v[0] = (w & 0x000F000Fu) | 0x43004300u;
-  v[1] = ((w >> 4) & 0x000F000Fu) | 0x43004300u;
-  v[2] = ((w >> 8) & 0x000F000Fu) | 0x43004300u;
-  v[3] = ((w >> 12) & 0x000F000Fu) | 0x43004300u;
+// (k.m0 = 0x000F000F, k.c = 0x43004300)
+__device__ __forceinline__ void gv_unpack(uint32_t w, uint32_t (&v)[4], const GvConst& k) {
+  v[0] = gv_and_or(w, k.m0, k.c);
+  v[1] = gv_and_or(w >> 4, k.m0, k.c);
+  v[2] = gv_and_or(w >> 8, k.m0, k.c);
+  v[3] = gv_and_or(w >> 12, k.m0, k.c);
+}
+// 16 consecutive x values (two 16-byte words) -> the eight B registers of the four MMAs of a thread:
+// f[2 (2 wd + h)] / f[2 (2 wd + h) + 1] pair x at positions (2h, 2h+4) / (2h+1, 2h+5) of word wd
+__device__ __forceinline__ void gv_permute_x(const uint4& x0, const uint4& x1, uint32_t (&f)[8]) {
+  const uint32_t xr[2][4] = {{x0.x, x0.y, x0.z, x0.w}, {x1.x, x1.y, x1.z, x1.w}};
+#pragma unroll
+  for (int wd = 0; wd < 2; ++wd)
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      f[2 * (2 * wd + h)] = gv_prmt(xr[wd][h], xr[wd][h + 2], 0x5410u);
+      f[2 * (2 * wd + h) + 1] = gv_prmt(xr[wd][h], xr[wd][h + 2], 0x7632u);
+    }
+}
+__device__ __forceinline__ float gv_sum16(const uint4& x0, const uint4& x1) {
+  const uint32_t w[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+  float a = 0.0f;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) a += __uint_as_float(w[i] << 16) + __uint_as_float(w[i] & 0xFFFF0000u);
+  return a;
+}
+// ---- fp16 variants (shared-memory token operand only) --------------------------------------------
+// With a 10-bit mantissa two neighbouring nibbles fit below the magic exponent, so a word needs one
+// shift instead of three: v[0], v[2] = 1024 + c for codes (0,4), (2,6); v[1], v[3] = 1024 + 16 c for
+// codes (1,5), (3,7).  The token operand carries 1/16 at the odd positions to match.
+// (k.m0 = 0x000F000F, k.m1 = 0x00F000F0, k.c = 0x64006400)
+__device__ __forceinline__ void gv_unpack_h(uint32_t w, uint32_t (&v)[4], const GvConst& k) {
+  const uint32_t t = w >> 8;
+  v[0] = gv_and_or(w, k.m0, k.c);
+  v[1] = gv_and_or(w, k.m1, k.c);
+  v[2] = gv_and_or(t, k.m0, k.c);
+  v[3] = gv_and_or(t, k.m1, k.c);
+}
+__device__ __forceinline__ void gv_mma_h(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1) {
+  asm(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void gv_mma0_h(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                          uint32_t b1) {
+  asm(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+      : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.0f));
+}
+__device__ __forceinline__ uint32_t gv_pack_h2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+__device__ __forceinline__ float gv_h_lo(uint32_t v) { return __half2float(__ushort_as_half((unsigned short)(v & 0xFFFFu))); }
+__device__ __forceinline__ float gv_h_hi(uint32_t v) { return __half2float(__ushort_as_half((unsigned short)(v >> 16))); }
+__device__ __forceinline__ float gv_absmax8(const uint4& x, float m) {
+  const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    m = fmaxf(m, fabsf(__uint_as_float(w[i] << 16)));
+    m = fmaxf(m, fabsf(__uint_as_float(w[i] & 0xFFFF0000u)));
+  }
+  return m;
 }
 
-// Streams NB consecutive groups: all code / scale loads are issued first (constant offsets from the
-// running pointers), then each group is unpacked and multiplied.
-template <int NT, int NB>
-__device__ __forceinline__ void gv_groups(const uint2* __restrict__ c0, const uint2* __restrict__ c1,
-                                          const float* __restrict__ al0, const float* __restrict__ al1,
-                                          const float* __restrict__ be0, const float* __restrict__ be1,
-                                          const uint4* const (&xp)[NT], const bool (&xlive)[NT], float (&y)[NT][4]) {
-  uint2 w0[NB], w1[NB];
-  float a0[NB], a1[NB], b0[NB], b1[NB];
-#pragma unroll
-  for (int u = 0; u < NB; ++u) {
-    w0[u] = __ldg(c0 + u * 4); w1[u] = __ldg(c1 + u * 4);
-    a0[u] = __ldg(al0 + u); a1[u] = __ldg(al1 + u);
-    b0[u] = __ldg(be0 + u); b1[u] = __ldg(be1 + u);
-  }
-  const uint32_t ones = 0x3F803F80u;   // bf16 (1.0, 1.0)
-#pragma unroll
-  for (int u = 0; u < NB; ++u) {
-    uint32_t va[2][4], vb[2][4];      // [word][pair] for rows g (va) and g + 8 (vb)
-    gv_unpack(w0[u].x, va[0]); gv_unpack(w0[u].y, va[1]);
-    gv_unpack(w1[u].x, vb[0]); gv_unpack(w1[u].y, vb[1]);
-    const float s0 = fmaf(-128.0f, a0[u], b0[u]), s1 = fmaf(-128.0f, a1[u], b1[u]);
-#pragma unroll
-    for (int j = 0; j < NT; ++j) {
-      uint4 x0 = make_uint4(0, 0, 0, 0), x1 = make_uint4(0, 0, 0, 0);
-      if (xlive[j]) { x0 = __ldg(xp[j] + u * 8); x1 = __ldg(xp[j] + u * 8 + 1); }
-      float acc[4] = {0.f, 0.f, 0.f, 0.f}, sum[4] = {0.f, 0.f, 0.f, 0.f};
-      const uint32_t xr[2][4] = {{x0.x, x0.y, x0.z, x0.w}, {x1.x, x1.y, x1.z, x1.w}};
-#pragma unroll
-      for (int wd = 0; wd < 2; ++wd) {
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          // codes (2h, 2h+4) and (2h+1, 2h+5) of word wd <-> x at the same positions
-          const uint32_t bx0 = gv_prmt(xr[wd][h], xr[wd][h + 2], 0x5410u);
-          const uint32_t bx1 = gv_prmt(xr[wd][h], xr[wd][h + 2], 0x7632u);
-          gv_mma(acc, va[wd][2 * h], vb[wd][2 * h], va[wd][2 * h + 1], vb[wd][2 * h + 1], bx0, bx1);
-          gv_mma(sum, ones, ones, ones, ones, bx0, bx1);
-        }
-      }
-      y[j][0] = fmaf(a0[u], acc[0], fmaf(s0, sum[0], y[j][0]));
-      y[j][1] = fmaf(a0[u], acc[1], fmaf(s0, sum[1], y[j][1]));
-      y[j][2] = fmaf(a1[u], acc[2], fmaf(s1, sum[2], y[j][2]));
-      y[j][3] = fmaf(a1[u], acc[3], fmaf(s1, sum[3], y[j][3]));
+// shared-memory loads with 32-bit shared-space addresses (immediate offset OFF)
+template <int OFF>
+__device__ __forceinline__ uint2 gv_lds2(uint32_t addr) {
+  uint2 v;
+  asm volatile("ld.shared.v2.u32 {%0, %1}, [%2 + %3];" : "=r"(v.x), "=r"(v.y) : "r"(addr), "n"(OFF));
+  return v;
+}
+template <int OFF>
+__device__ __forceinline__ uint4 gv_lds4(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4 + %5];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr), "n"(OFF));
+  return v;
+}
+template <int OFF>
+__device__ __forceinline__ float gv_ldsf(uint32_t addr) {
+  float v;
+  asm volatile("ld.shared.f32 %0, [%1 + %2];" : "=f"(v) : "r"(addr), "n"(OFF));
+  return v;
+}
+template <int OFF>
+__device__ __forceinline__ float2 gv_ldsf2(uint32_t addr) {
+  float2 v;
+  asm volatile("ld.shared.v2.f32 {%0, %1}, [%2 + %3];" : "=f"(v.x), "=f"(v.y) : "r"(addr), "n"(OFF));
+  return v;
+}
+template <int OFF>
+__device__ __forceinline__ float4 gv_ldsf4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4 + %5];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr), "n"(OFF));
+  return v;
+}
+
+// Waits of this kernel pass a suspend-time hint so that a waiting warp sleeps in hardware until the
+// phase completes instead of polling: polling takes issue slots and ALU cycles from the warps of the
+// same scheduler that still have work.  Still bounded: gives up after the cycle limit.
+__device__ __forceinline__ bool gv_try_wait_hint(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok) : "r"(bar), "r"(parity), "r"(100000u) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool gv_wait(uint32_t bar, uint32_t parity, int* status) {
+  if (gv_try_wait_hint(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (!gv_try_wait_hint(bar, parity)) {
+    if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+      atomicExch(status, (int)QBLORA_ERR_TIMEOUT);
+      return false;
     }
   }
+  return true;
 }
 
-template <int NT>   // NT = number of 8-token tiles (1 or 2)
-__global__ void __launch_bounds__(GV_WARPS * 32, 2) lowbit_gemv_kernel(QwView q, const __nv_bfloat16* __restrict__ X, int T,
-                                                                       void* __restrict__ Y, int y_dtype) {
-  __shared__ float red[GV_WARPS][GV_ROWS][NT * 8];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, tg = lane & 3;
-  const int row_base = blockIdx.x * GV_ROWS;
-  // rows past the end are clamped for loads and dropped at the store
-  const int r0 = min(row_base + g, q.d_out - 1), r1 = min(row_base + g + 8, q.d_out - 1);
-  const int per = (q.G + GV_WARPS - 1) / GV_WARPS;
-  const int g_begin = min(warp * per, q.G), g_end = min(g_begin + per, q.G);
-  // running pointers of this thread, positioned at its first group
-  const uint2* c0 = reinterpret_cast<const uint2*>(q.codes + (int64_t)r0 * (q.d_in >> 1)) + tg + g_begin * 4;
-  const uint2* c1 = reinterpret_cast<const uint2*>(q.codes + (int64_t)r1 * (q.d_in >> 1)) + tg + g_begin * 4;
-  const float* al0 = q.alpha + (int64_t)r0 * q.G + g_begin; const float* al1 = q.alpha + (int64_t)r1 * q.G + g_begin;
-  const float* be0 = q.beta + (int64_t)r0 * q.G + g_begin;  const float* be1 = q.beta + (int64_t)r1 * q.G + g_begin;
-  const uint4* xp[NT];
-  bool xlive[NT];
-#pragma unroll
-  for (int j = 0; j < NT; ++j) {
-    const int t = j * 8 + g;
-    xlive[j] = t < T;
-    xp[j] = reinterpret_cast<const uint4*>(X + (int64_t)(xlive[j] ? t : 0) * q.d_in) + tg * 2 + g_begin * 8;
-  }
-  float y[NT][4];
-#pragma unroll
-  for (int j = 0; j < NT; ++j) { y[j][0] = y[j][1] = y[j][2] = y[j][3] = 0.0f; }
+struct GtParams {
+  int d_in, d_out, G, T;
+  int n_rb, n_kc;            // row blocks of 32 rows, K tiles of 16 groups
+  const __nv_bfloat16* X;
+  void* Y;
+  int y_dtype;
+  int* status;
+};
 
-  constexpr int NB = 4;
-  int left = g_end - g_begin;
-  for (; left >= NB; left -= NB) {
-    gv_groups<NT, NB>(c0, c1, al0, al1, be0, be1, xp, xlive, y);
-    c0 += NB * 4; c1 += NB * 4; al0 += NB; al1 += NB; be0 += NB; be1 += NB;
-#pragma unroll
-    for (int j = 0; j < NT; ++j) xp[j] += NB * 8;
-  }
-  for (; left > 0; --left) {
-    gv_groups<NT, 1>(c0, c1, al0, al1, be0, be1, xp, xlive, y);
-    c0 += 4; c1 += 4; ++al0; ++al1; ++be0; ++be1;
-#pragma unroll
-    for (int j = 0; j < NT; ++j) xp[j] += 8;
-  }
-  // accumulator layout: [0],[1] = row g, tokens 2tg, 2tg+1; [2],[3] = row g + 8
-#pragma unroll
-  for (int j = 0; j < NT; ++j) {
-    red[warp][g][j * 8 + 2 * tg] = y[j][0]; red[warp][g][j * 8 + 2 * tg + 1] = y[j][1];
-    red[warp][g + 8][j * 8 + 2 * tg] = y[j][2]; red[warp][g + 8][j * 8 + 2 * tg + 1] = y[j][3];
+// MODE 0: token fragments rebuilt per group from global x (bf16 MMA), any T <= 8 NT.
+// MODE 1: x converted once per CTA to fp16 fragments in shared memory (T <= 8, small T x D_in).
+// MODE 2: MODE 1 specialised for a single token (only accumulator column 0 is kept).
+template <int NT, int MODE>
+struct GtCfg {
+  static constexpr int STAGES = (MODE != 0 || NT == 2) ? 6 : 8;
+  static constexpr int RED_BYTES = GT_WARPS * GT_ROWS * (NT * 8) * 4;
+  static constexpr int SS_PER_GROUP = MODE == 0 ? NT * 8 : 16;   // floats: S per token, or (P, R) per token
+};
+
+template <int NT, int MODE>   // NT = number of 8-token tiles (1 or 2)
+__global__ void __launch_bounds__(GT_THREADS, 1)
+lowbit_gemv_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_constant__ CUtensorMap tm_a,
+                   const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ GtParams p) {
+  static_assert(MODE == 0 || NT == 1, "shared-memory token operand: one token tile");
+  constexpr int STAGES = GtCfg<NT, MODE>::STAGES;
+  constexpr int NTOK = NT * 8;
+  constexpr int SSG = GtCfg<NT, MODE>::SS_PER_GROUP;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* gbase = smem_raw + (base - raw);
+  const uint32_t red_off = STAGES * GT_STAGE_BYTES;
+  float* red = reinterpret_cast<float*>(gbase + red_off);                 // [16 warps][32 rows][NTOK]
+  const uint32_t bar_off = red_off + GtCfg<NT, MODE>::RED_BYTES;
+  const uint32_t bars = base + bar_off;
+  auto full = [&](int s) { return bars + 8u * s; };
+  auto empty = [&](int s) { return bars + 8u * (STAGES + s); };
+  // MODE 0: ss[G][NTOK] = S (sum of x over the group), 0 beyond T.
+  // MODE 1/2: ss[G][8][2] = (1024 * sum of the fp16 fragment values, sum of the scaled x), then
+  //           xs[G][T][4 tg][8 words] = fp16 fragments
+  float* ss = reinterpret_cast<float*>(gbase + bar_off + 256);
+  const uint32_t ss_off = bar_off + 256;
+  const uint32_t xs_off = ss_off + (uint32_t)p.G * SSG * 4;
+  uint4* xs = reinterpret_cast<uint4*>(gbase + xs_off);
+  const uint32_t zero_off = xs_off + (MODE != 0 ? (uint32_t)p.G * p.T * 128 : 0u);   // 128 zero bytes (MODE 1/2)
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (tid == 0) {
+    if (blockIdx.x == 0) *p.status = 0;   // any give-up below is written at least a wait limit later
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), GT_WARPS); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
-  for (int idx = threadIdx.x; idx < GV_ROWS * NT * 8; idx += GV_WARPS * 32) {
-    const int t = idx / GV_ROWS, r = idx % GV_ROWS;     // consecutive threads -> consecutive output rows
-    const int o = row_base + r;
-    if (t < T && o < q.d_out) {
-      float a = 0.0f;
+
+  if (warp == GT_WARPS) {
+    // ------------------------------------------------------------------ producer (one lane)
+    if (lane == 0) {
+      uint32_t it = 0, ph = 0;
+      int s = 0;
+      bool ok = true;
+      for (int rb = blockIdx.x; rb < p.n_rb && ok; rb += gridDim.x) {
+        for (int kc = 0; kc < p.n_kc; ++kc, ++it) {
+          if (!gv_wait(empty(s), ph ^ 1u, p.status)) { ok = false; break; }
+          const uint32_t st = base + s * GT_STAGE_BYTES;
+          mbar_arrive_expect_tx(full(s), GT_STAGE_BYTES);
 #pragma unroll
-      for (int w = 0; w < GV_WARPS; ++w) a += red[w][r][t];
-      if (y_dtype == QBLORA_BF16) reinterpret_cast<__nv_bfloat16*>(Y)[(int64_t)t * q.d_out + o] = __float2bfloat16_rn(a);
-      else reinterpret_cast<float*>(Y)[(int64_t)t * q.d_out + o] = a;
+          for (int j = 0; j < 4; ++j)   // four groups = 128 bytes = 32 u32 per row and box
+            tma_load_2d(st + j * 4096, &tm_c, full(s), (kc * GT_GROUPS + j * 4) * 8, rb * GT_ROWS);
+          tma_load_2d(st + GT_CODE_BYTES, &tm_a, full(s), kc * GT_GROUPS, rb * GT_ROWS);
+          tma_load_2d(st + GT_CODE_BYTES + GT_SCALE_BYTES, &tm_b, full(s), kc * GT_GROUPS, rb * GT_ROWS);
+          if (++s == STAGES) { s = 0; ph ^= 1u; }
+        }
+      }
+      if (!ok) {   // give copies already in flight a bounded chance to land before the CTA exits
+        const uint32_t lo = it > (uint32_t)STAGES ? it - STAGES : 0;
+        for (uint32_t j = lo; j < it; ++j) gv_wait(full(j % STAGES), (j / STAGES) & 1u, p.status);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ compute warps
+    const int g = lane >> 2, tg = lane & 3;
+    // ---- once per CTA, while the first tiles are in flight: group sums of x and (MODE 1/2) fragments.
+    // Item = (group, token, tg): 16 values of x; the four tg lanes of an item are neighbours.
+    float y_scale = 1.0f;
+    if (MODE == 0) {
+      for (int i = tid; i < p.G * NTOK; i += GT_WARPS * 32)
+        if ((i % NTOK) >= p.T) ss[i] = 0.0f;
+    } else {
+      // fp16 range: one power-of-two prescale for the call so that max |x| stays below 2^15
+      float am = 0.0f;
+      const uint4* xv = reinterpret_cast<const uint4*>(p.X);
+      for (int i = tid; i < p.T * (p.d_in >> 3); i += GT_WARPS * 32) am = gv_absmax8(__ldg(xv + i), am);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) am = fmaxf(am, __shfl_xor_sync(0xFFFFFFFFu, am, o));
+      if (lane == 0) red[warp] = am;
+      for (int i = tid; i < p.G * 16; i += GT_WARPS * 32)
+        if (((i >> 1) & 7) >= p.T) ss[i] = 0.0f;
+      asm volatile("bar.sync 1, 512;" ::: "memory");
+      am = red[0];
+#pragma unroll
+      for (int i = 1; i < GT_WARPS; ++i) am = fmaxf(am, red[i]);
+      int e = (int)((__float_as_uint(am) >> 23) & 0xFFu) - 127 - 14;
+      e = e < 0 ? 0 : (e > 120 ? 120 : e);
+      y_scale = __uint_as_float((uint32_t)(127 + e) << 23);
+      asm volatile("bar.sync 1, 512;" ::: "memory");   // red is free again
+      if (tid < 32) reinterpret_cast<uint32_t*>(gbase + zero_off)[tid] = 0u;
+    }
+    {
+      const float in_scale = 1.0f / y_scale, in_scale16 = in_scale * 0.0625f;
+      const int items = p.G * p.T * 4;
+      for (int i0 = 0; i0 < items; i0 += GT_WARPS * 32) {
+        const int idx = i0 + tid;
+        const bool live = idx < items;
+        const int q = live ? idx : 0;
+        const int t = (q >> 2) % p.T, grp = (q >> 2) / p.T;
+        const uint4* src = reinterpret_cast<const uint4*>(p.X + (int64_t)t * p.d_in + grp * 64 + (q & 3) * 16);
+        const uint4 x0 = __ldg(src), x1 = __ldg(src + 1);
+        if (MODE == 0) {
+          float sum = gv_sum16(x0, x1);
+          sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 1);
+          sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 2);
+          if (live && (q & 3) == 0) ss[grp * NTOK + t] = sum;
+        } else {
+          const uint32_t xw[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+          uint32_t f[8];
+          float ps = 0.0f, rs = 0.0f;   // sum of fragment values; sum of scaled x as the fragments hold it
+#pragma unroll
+          for (int wd = 0; wd < 2; ++wd)
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              // word wd holds x at positions 0..7 as pairs (2j, 2j+1) in xw[4 wd + j]
+              const uint32_t wa = xw[4 * wd + h], wb = xw[4 * wd + h + 2];
+              const uint32_t ev = gv_pack_h2(__uint_as_float(wa << 16) * in_scale, __uint_as_float(wb << 16) * in_scale);
+              const uint32_t od = gv_pack_h2(__uint_as_float(wa & 0xFFFF0000u) * in_scale16,
+                                             __uint_as_float(wb & 0xFFFF0000u) * in_scale16);
+              f[2 * (2 * wd + h)] = ev;
+              f[2 * (2 * wd + h) + 1] = od;
+              const float se = gv_h_lo(ev) + gv_h_hi(ev), so = gv_h_lo(od) + gv_h_hi(od);
+              ps += se + so;
+              rs += se + 16.0f * so;
+            }
+          ps += __shfl_xor_sync(0xFFFFFFFFu, ps, 1); rs += __shfl_xor_sync(0xFFFFFFFFu, rs, 1);
+          ps += __shfl_xor_sync(0xFFFFFFFFu, ps, 2); rs += __shfl_xor_sync(0xFFFFFFFFu, rs, 2);
+          if (live) {
+            if ((q & 3) == 0) *reinterpret_cast<float2*>(ss + (grp * 8 + t) * 2) = make_float2(1024.0f * ps, rs);
+            xs[q * 2] = make_uint4(f[0], f[1], f[2], f[3]);
+            xs[q * 2 + 1] = make_uint4(f[4], f[5], f[6], f[7]);
+          }
+        }
+      }
+    }
+    asm volatile("bar.sync 1, 512;" ::: "memory");
+
+    // byte offsets inside a stage that do not depend on the stage: the thread's 8 bytes of codes of the
+    // warp's group in row g (rows g + 8 q: + 1024 q, same swizzle phase) and its scale entries (rows g + 8 q: + 512 q)
+    const uint32_t code_off = ((uint32_t)warp >> 2) * 4096u + (uint32_t)g * 128u +
+                              ((((((uint32_t)warp & 3u) << 1) | ((uint32_t)tg >> 1)) ^ (uint32_t)g) << 4) +
+                              (((uint32_t)tg & 1u) << 3);
+    // alpha / beta tiles are [32 rows][16 groups] fp32 with the 64-byte swizzle (16-byte chunk index
+    // xor (row / 2) % 4), which spreads the eight rows a warp reads at once over eight banks
+    const uint32_t scale_off = GT_CODE_BYTES + (uint32_t)g * 64u +
+                               ((((uint32_t)warp >> 2) ^ (((uint32_t)g >> 1) & 3u)) << 4) + ((uint32_t)warp & 3u) * 4u;
+    const uint4* xrow[NT];
+    bool xlive[NT];
+#pragma unroll
+    for (int j = 0; j < NT; ++j) {
+      const int t = j * 8 + g;
+      xlive[j] = t < p.T;
+      xrow[j] = reinterpret_cast<const uint4*>(p.X + (int64_t)(xlive[j] ? t : 0) * p.d_in) + tg * 2;
+    }
+    // MODE 1/2: lanes whose token does not exist read the zero block (stride 0) instead of selecting zeros
+    const uint32_t xs_addr = base + (xlive[0] ? xs_off + (uint32_t)(g * 4 + tg) * 32u : zero_off + (uint32_t)tg * 32u);
+    const uint32_t xs_stride = xlive[0] ? (uint32_t)p.T * 128u : 0u;
+    const uint32_t ss_addr = base + ss_off + (MODE == 0 ? 8u * tg : (MODE == 1 ? 16u * tg : 0u));
+    float* my_red = red + warp * GT_ROWS * NTOK;
+    const GvConst kc_(0x000F000Fu, 0x00F000F0u, MODE == 0 ? 0x43004300u : 0x64006400u);
+    bool ok = true;        // after a timed-out wait the warp keeps walking its loops (so the CTA
+                           // barriers still match) but no longer waits or computes
+    int s = 0;
+    uint32_t ph = 0;
+    for (int rb = blockIdx.x; rb < p.n_rb; rb += gridDim.x) {
+      float y[NT][2][4];
+#pragma unroll
+      for (int j = 0; j < NT; ++j)
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) { y[j][mt][0] = y[j][mt][1] = y[j][mt][2] = y[j][mt][3] = 0.0f; }
+      for (int kc = 0; kc < p.n_kc; ++kc) {
+        if (ok && !gv_wait(full(s), ph, p.status)) ok = false;
+        const int grp = kc * GT_GROUPS + warp;
+        if (ok) {
+          if (grp < p.G) {                                   // warp-uniform
+            const uint32_t sb = base + (uint32_t)s * GT_STAGE_BYTES;
+            const uint32_t ca = sb + code_off, sa = sb + scale_off;
+            uint32_t f[NT][8];
+            float4 sg[NT];   // MODE 0: (S[2tg], S[2tg+1], -, -); MODE 1: (P, R)[2tg], (P, R)[2tg+1]; MODE 2: (P, R)[0]
+            if (MODE == 0) {
+#pragma unroll
+              for (int j = 0; j < NT; ++j) {
+                const float2 v = j == 0 ? gv_ldsf2<0>(ss_addr + (uint32_t)grp * (NTOK * 4)) : gv_ldsf2<32>(ss_addr + (uint32_t)grp * (NTOK * 4));
+                sg[j] = make_float4(v.x, v.y, 0.0f, 0.0f);
+                uint4 x0 = make_uint4(0, 0, 0, 0), x1 = make_uint4(0, 0, 0, 0);
+                if (xlive[j]) { x0 = __ldg(xrow[j] + grp * 8); x1 = __ldg(xrow[j] + grp * 8 + 1); }
+                gv_permute_x(x0, x1, f[j]);
+              }
+            } else {
+              if (MODE == 1) sg[0] = gv_ldsf4<0>(ss_addr + (uint32_t)grp * 64u);
+              else { const float2 v = gv_ldsf2<0>(ss_addr + (uint32_t)grp * 64u); sg[0] = make_float4(v.x, v.y, 0.0f, 0.0f); }
+              const uint32_t xa = xs_addr + (uint32_t)grp * xs_stride;
+              const uint4 x0 = gv_lds4<0>(xa), x1 = gv_lds4<16>(xa);
+              f[0][0] = x0.x; f[0][1] = x0.y; f[0][2] = x0.z; f[0][3] = x0.w;
+              f[0][4] = x1.x; f[0][5] = x1.y; f[0][6] = x1.z; f[0][7] = x1.w;
+            }
+            // all shared-memory loads of the group first (they stay in program order), then the math
+            uint2 w0[2], w1[2];
+            float a0[2], a1[2], b0[2], b1[2];
+            w0[0] = gv_lds2<0>(ca); w1[0] = gv_lds2<1024>(ca); w0[1] = gv_lds2<2048>(ca); w1[1] = gv_lds2<3072>(ca);
+            a0[0] = gv_ldsf<0>(sa); a1[0] = gv_ldsf<512>(sa); a0[1] = gv_ldsf<1024>(sa); a1[1] = gv_ldsf<1536>(sa);
+            b0[0] = gv_ldsf<GT_SCALE_BYTES>(sa); b1[0] = gv_ldsf<GT_SCALE_BYTES + 512>(sa);
+            b0[1] = gv_ldsf<GT_SCALE_BYTES + 1024>(sa); b1[1] = gv_ldsf<GT_SCALE_BYTES + 1536>(sa);
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt) {
+              uint32_t va[2][4], vb[2][4];      // [word][pair] for rows g + 16 mt (va) and g + 16 mt + 8 (vb)
+              if (MODE == 0) {
+                gv_unpack(w0[mt].x, va[0], kc_); gv_unpack(w0[mt].y, va[1], kc_);
+                gv_unpack(w1[mt].x, vb[0], kc_); gv_unpack(w1[mt].y, vb[1], kc_);
+                const float s0 = fmaf(-128.0f, a0[mt], b0[mt]), s1 = fmaf(-128.0f, a1[mt], b1[mt]);
+#pragma unroll
+                for (int j = 0; j < NT; ++j) {
+                  float acc[4];
+                  gv_mma0(acc, va[0][0], vb[0][0], va[0][1], vb[0][1], f[j][0], f[j][1]);
+                  gv_mma(acc, va[0][2], vb[0][2], va[0][3], vb[0][3], f[j][2], f[j][3]);
+                  gv_mma(acc, va[1][0], vb[1][0], va[1][1], vb[1][1], f[j][4], f[j][5]);
+                  gv_mma(acc, va[1][2], vb[1][2], va[1][3], vb[1][3], f[j][6], f[j][7]);
+                  y[j][mt][0] = fmaf(a0[mt], acc[0], fmaf(s0, sg[j].x, y[j][mt][0]));
+                  y[j][mt][1] = fmaf(a0[mt], acc[1], fmaf(s0, sg[j].y, y[j][mt][1]));
+                  y[j][mt][2] = fmaf(a1[mt], acc[2], fmaf(s1, sg[j].x, y[j][mt][2]));
+                  y[j][mt][3] = fmaf(a1[mt], acc[3], fmaf(s1, sg[j].y, y[j][mt][3]));
+                }
+              } else {
+                gv_unpack_h(w0[mt].x, va[0], kc_); gv_unpack_h(w0[mt].y, va[1], kc_);
+                gv_unpack_h(w1[mt].x, vb[0], kc_); gv_unpack_h(w1[mt].y, vb[1], kc_);
+                float acc[4];
+                gv_mma0_h(acc, va[0][0], vb[0][0], va[0][1], vb[0][1], f[0][0], f[0][1]);
+                gv_mma_h(acc, va[0][2], vb[0][2], va[0][3], vb[0][3], f[0][2], f[0][3]);
+                gv_mma_h(acc, va[1][0], vb[1][0], va[1][1], vb[1][1], f[0][4], f[0][5]);
+                gv_mma_h(acc, va[1][2], vb[1][2], va[1][3], vb[1][3], f[0][6], f[0][7]);
+                // alpha (acc - 1024 P) + beta R
+                if (MODE == 1) {
+                  y[0][mt][0] = fmaf(a0[mt], acc[0] - sg[0].x, fmaf(b0[mt], sg[0].y, y[0][mt][0]));
+                  y[0][mt][1] = fmaf(a0[mt], acc[1] - sg[0].z, fmaf(b0[mt], sg[0].w, y[0][mt][1]));
+                  y[0][mt][2] = fmaf(a1[mt], acc[2] - sg[0].x, fmaf(b1[mt], sg[0].y, y[0][mt][2]));
+                  y[0][mt][3] = fmaf(a1[mt], acc[3] - sg[0].z, fmaf(b1[mt], sg[0].w, y[0][mt][3]));
+                } else {   // single token: column 0 of the accumulator tile (held by the tg == 0 lanes)
+                  y[0][mt][0] = fmaf(a0[mt], acc[0] - sg[0].x, fmaf(b0[mt], sg[0].y, y[0][mt][0]));
+                  y[0][mt][2] = fmaf(a1[mt], acc[2] - sg[0].x, fmaf(b1[mt], sg[0].y, y[0][mt][2]));
+                }
+              }
+            }
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(empty(s));   // this warp is done reading the stage
+        }
+        if (++s == STAGES) { s = 0; ph ^= 1u; }
+      }
+      // end of the row block: sum the sixteen warps in warp order and store
+      // accumulator layout: [0],[1] = row g, tokens 2tg, 2tg+1; [2],[3] = row g + 8
+#pragma unroll
+      for (int j = 0; j < NT; ++j)
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+          float* r0 = my_red + (mt * 16 + g) * NTOK + j * 8 + 2 * tg;
+          *reinterpret_cast<float2*>(r0) = make_float2(y[j][mt][0], y[j][mt][1]);
+          *reinterpret_cast<float2*>(r0 + 8 * NTOK) = make_float2(y[j][mt][2], y[j][mt][3]);
+        }
+      asm volatile("bar.sync 1, 512;" ::: "memory");
+      for (int idx = tid; idx < GT_ROWS * NTOK; idx += GT_WARPS * 32) {
+        const int t = idx >> 5, r = idx & 31;               // consecutive threads -> consecutive output rows
+        const int o = rb * GT_ROWS + r;
+        if (t < p.T && o < p.d_out) {
+          float a = 0.0f;
+#pragma unroll
+          for (int ww = 0; ww < GT_WARPS; ++ww) a += red[(ww * GT_ROWS + r) * NTOK + t];
+          a *= y_scale;
+          if (p.y_dtype == QBLORA_BF16) reinterpret_cast<__nv_bfloat16*>(p.Y)[(int64_t)t * p.d_out + o] = __float2bfloat16_rn(a);
+          else reinterpret_cast<float*>(p.Y)[(int64_t)t * p.d_out + o] = a;
+        }
+      }
+      asm volatile("bar.sync 1, 512;" ::: "memory");   // red is reused by the next block
     }
   }
+  __syncthreads();
+}
+
+// dynamic shared memory: alignment slack, stage ring, reduction buffer, barriers, group sums, (MODE 1/2) fragments
+template <int NT, int MODE>
+size_t gt_smem_bytes(int G, int T) {
+  size_t n = 1024 + (size_t)GtCfg<NT, MODE>::STAGES * GT_STAGE_BYTES + GtCfg<NT, MODE>::RED_BYTES + 256 +
+             (size_t)G * GtCfg<NT, MODE>::SS_PER_GROUP * 4;
+  if (MODE != 0) n += (size_t)G * T * 128 + 128;
+  return n;
+}
+
+template <int NT, int MODE>
+int gt_launch(const CUtensorMap& tm_c, const CUtensorMap& tm_a, const CUtensorMap& tm_b, const GtParams& p, int grid,
+              cudaStream_t st) {
+  const size_t smem = gt_smem_bytes<NT, MODE>(p.G, p.T);
+  if (smem > 227 * 1024) return QBLORA_ERR_UNSUPPORTED;
+  QB_CUDA(cudaFuncSetAttribute(lowbit_gemv_kernel<NT, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  lowbit_gemv_kernel<NT, MODE><<<grid, GT_THREADS, smem, st>>>(tm_c, tm_a, tm_b, p);
+  return QBLORA_OK;
 }
 
 }  // namespace
 
 bool gemv_supported(const QwView& qw, int64_t T) {
-  return qw.block_in == 64 && qw.block_out == 1 && qw.qfmt == QBLORA_FMT_AFFINE_MINMAX && T <= 16;
+  // TMA over alpha / beta rows needs a 16-byte row pitch: G % 4 == 0
+  return qw.block_in == 64 && qw.block_out == 1 && qw.qfmt == QBLORA_FMT_AFFINE_MINMAX && T <= 16 && qw.G % 4 == 0 && qw.G <= 1024;
 }
 
-int launch_lowbit_gemv(const QwView& qw, const __nv_bfloat16* X, int64_t T, void* Y, int y_dtype,
+int launch_lowbit_gemv(const QwView& qw, const __nv_bfloat16* X, int64_t T, void* Y, int y_dtype, int* status,
                        cudaStream_t st) {
-  DominantKernelTimer timer(st);
-  count_launch();
-  const int grid = (qw.d_out + GV_ROWS - 1) / GV_ROWS;
-  if (T <= 8) lowbit_gemv_kernel<1><<<grid, GV_WARPS * 32, 0, st>>>(qw, X, (int)T, Y, y_dtype);
-  else lowbit_gemv_kernel<2><<<grid, GV_WARPS * 32, 0, st>>>(qw, X, (int)T, Y, y_dtype);
+  const int NT = T <= 8 ? 1 : 2;
+  GtParams p{};
+  p.d_in = qw.d_in; p.d_out = qw.d_out; p.G = qw.G; p.T = (int)T;
+  p.n_rb = (qw.d_out + GT_ROWS - 1) / GT_ROWS;
+  p.n_kc = (qw.G + GT_GROUPS - 1) / GT_GROUPS;
+  p.X = X; p.Y = Y; p.y_dtype = y_dtype; p.status = status;
+  CUtensorMap tm_c, tm_a, tm_b;
+  // codes as 32-bit words: [d_out][d_in / 8], boxes of 32 words (four groups) x 32 rows, 128-byte swizzle
+  int rc = make_tensor_map_2d_typed(&tm_c, TM_U32, qw.codes, (uint64_t)qw.d_in / 8, (uint64_t)qw.d_out,
+                                    (uint64_t)qw.d_in / 2, 32, GT_ROWS, 128);
+  if (rc) return rc;
+  rc = make_tensor_map_2d_typed(&tm_a, TM_F32, qw.alpha, (uint64_t)qw.G, (uint64_t)qw.d_out, (uint64_t)qw.G * 4,
+                                GT_GROUPS, GT_ROWS, 64);
+  if (rc) return rc;
+  rc = make_tensor_map_2d_typed(&tm_b, TM_F32, qw.beta, (uint64_t)qw.G, (uint64_t)qw.d_out, (uint64_t)qw.G * 4,
+                                GT_GROUPS, GT_ROWS, 64);
+  if (rc) return rc;
+  int sms = 148;
+  { int dev = 0; if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); }
+  const int grid = p.n_rb < sms ? p.n_rb : sms;
+  // fp16 fragments of x fit in shared memory next to a six-stage ring?
+  const bool xs = NT == 1 && gt_smem_bytes<1, 1>(p.G, p.T) <= 225 * 1024;
+  {
+    DominantKernelTimer timer(st);
+    count_launch();
+    if (xs && T == 1) rc = gt_launch<1, 2>(tm_c, tm_a, tm_b, p, grid, st);
+    else if (xs) rc = gt_launch<1, 1>(tm_c, tm_a, tm_b, p, grid, st);
+    else if (NT == 1) rc = gt_launch<1, 0>(tm_c, tm_a, tm_b, p, grid, st);
+    else rc = gt_launch<2, 0>(tm_c, tm_a, tm_b, p, grid, st);
+    if (rc) return rc;
+  }
   QB_CUDA(cudaGetLastError());
   return QBLORA_OK;
 }

@@ -37,4 +37,9 @@ int small_gemm_splits(int M, int N, int K);
 int make_tensor_map_2d(void* tm, bool is_u8, const void* ptr, uint64_t inner, uint64_t rows, uint64_t pitch_bytes,
                        uint32_t box_inner, uint32_t box_rows, bool swizzle128);
 
+// Same with an explicit element type and shared-memory swizzle span (0, 64 or 128 bytes).
+enum { TM_BF16 = 0, TM_U8 = 1, TM_U32 = 2, TM_F32 = 3 };
+int make_tensor_map_2d_typed(void* tm, int elem, const void* ptr, uint64_t inner, uint64_t rows, uint64_t pitch_bytes,
+                             uint32_t box_inner, uint32_t box_rows, int swizzle_bytes);
+
 }  // namespace qb

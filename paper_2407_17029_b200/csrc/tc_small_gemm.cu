@@ -233,15 +233,24 @@ int operand_map(CUtensorMap* tm, const SgOperand& op, int MN, int K, int box_row
 
 int make_tensor_map_2d(void* tm, bool is_u8, const void* ptr, uint64_t inner, uint64_t rows, uint64_t pitch_bytes,
                        uint32_t box_inner, uint32_t box_rows, bool swizzle128) {
+  return make_tensor_map_2d_typed(tm, is_u8 ? TM_U8 : TM_BF16, ptr, inner, rows, pitch_bytes, box_inner, box_rows, swizzle128 ? 128 : 0);
+}
+
+int make_tensor_map_2d_typed(void* tm, int elem, const void* ptr, uint64_t inner, uint64_t rows, uint64_t pitch_bytes,
+                             uint32_t box_inner, uint32_t box_rows, int swizzle_bytes) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return QBLORA_ERR_CUDA;
   cuuint64_t dims[2] = {inner, rows};
   cuuint64_t strides[1] = {pitch_bytes};
   cuuint32_t box[2] = {box_inner, box_rows};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn(static_cast<CUtensorMap*>(tm), is_u8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+  const CUtensorMapDataType dt = elem == TM_U8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8
+                                 : elem == TM_U32 ? CU_TENSOR_MAP_DATA_TYPE_UINT32
+                                 : elem == TM_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+  CUresult r = fn(static_cast<CUtensorMap*>(tm), dt,
                   2, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                  swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                  swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                  : swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE,
                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? QBLORA_OK : QBLORA_ERR_CUDA;
 }
