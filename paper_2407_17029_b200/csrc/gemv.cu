@@ -198,6 +198,7 @@ __device__ __forceinline__ bool gv_wait(uint32_t bar, uint32_t parity, int* stat
 struct GtParams {
   int d_in, d_out, G, T;
   int n_rb, n_kc;            // row blocks of 32 rows, K tiles of 16 groups
+  int stages;                // depth of the shared-memory ring (as many as fit)
   const __nv_bfloat16* X;
   void* Y;
   int y_dtype;
@@ -209,9 +210,10 @@ struct GtParams {
 // MODE 2: MODE 1 specialised for a single token (only accumulator column 0 is kept).
 template <int NT, int MODE>
 struct GtCfg {
-  static constexpr int STAGES = (MODE != 0 || NT == 2) ? 6 : 8;
-  static constexpr int RED_BYTES = GT_WARPS * GT_ROWS * (NT * 8) * 4;
-  static constexpr int SS_PER_GROUP = MODE == 0 ? NT * 8 : 16;   // floats: S per token, or (P, R) per token
+  static constexpr int RED_TOKENS = MODE == 2 ? 1 : NT * 8;                     // tokens kept per row in the reduction
+  static constexpr int RED_BYTES = GT_WARPS * GT_ROWS * RED_TOKENS * 4;
+  static constexpr int SS_PER_GROUP = MODE == 0 ? NT * 8 : (MODE == 1 ? 16 : 2);  // floats: S, or (P, R), per token
+  static constexpr int MAX_STAGES = 10;
 };
 
 template <int NT, int MODE>   // NT = number of 8-token tiles (1 or 2)
@@ -219,19 +221,22 @@ __global__ void __launch_bounds__(GT_THREADS, 1)
 lowbit_gemv_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_constant__ CUtensorMap tm_a,
                    const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ GtParams p) {
   static_assert(MODE == 0 || NT == 1, "shared-memory token operand: one token tile");
-  constexpr int STAGES = GtCfg<NT, MODE>::STAGES;
+  const int STAGES = p.stages;
   constexpr int NTOK = NT * 8;
+  constexpr int RT = GtCfg<NT, MODE>::RED_TOKENS;
   constexpr int SSG = GtCfg<NT, MODE>::SS_PER_GROUP;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* gbase = smem_raw + (base - raw);
   const uint32_t red_off = STAGES * GT_STAGE_BYTES;
-  float* red = reinterpret_cast<float*>(gbase + red_off);                 // [16 warps][32 rows][NTOK]
+  float* red = reinterpret_cast<float*>(gbase + red_off);                 // [16 warps][32 rows][RT]
   const uint32_t bar_off = red_off + GtCfg<NT, MODE>::RED_BYTES;
   const uint32_t bars = base + bar_off;
   auto full = [&](int s) { return bars + 8u * s; };
   auto empty = [&](int s) { return bars + 8u * (STAGES + s); };
+  const uint32_t red_done = bars + 8u * (2 * STAGES);       // all 16 warps have written their sums of the row block
+  const uint32_t red_free = bars + 8u * (2 * STAGES + 1);   // the summing warps have read them
   // MODE 0: ss[G][NTOK] = S (sum of x over the group), 0 beyond T.
   // MODE 1/2: ss[G][8][2] = (1024 * sum of the fp16 fragment values, sum of the scaled x), then
   //           xs[G][T][4 tg][8 words] = fp16 fragments
@@ -245,6 +250,8 @@ lowbit_gemv_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_consta
   if (tid == 0) {
     if (blockIdx.x == 0) *p.status = 0;   // any give-up below is written at least a wait limit later
     for (int s = 0; s < STAGES; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), GT_WARPS); }
+    mbar_init(red_done, GT_WARPS);
+    mbar_init(red_free, p.T);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -279,19 +286,33 @@ lowbit_gemv_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_consta
     // ---- once per CTA, while the first tiles are in flight: group sums of x and (MODE 1/2) fragments.
     // Item = (group, token, tg): 16 values of x; the four tg lanes of an item are neighbours.
     float y_scale = 1.0f;
+    const int items = p.G * p.T * 4;
+    const bool one_round = items <= GT_WARPS * 32;
+    uint4 c0, c1;     // this thread's item of the first round (x is read from global once when one round covers it)
+    {
+      const int q = tid < items ? tid : 0;
+      const int t = (q >> 2) % p.T, grp = (q >> 2) / p.T;
+      const uint4* src = reinterpret_cast<const uint4*>(p.X + (int64_t)t * p.d_in + grp * 64 + (q & 3) * 16);
+      c0 = __ldg(src); c1 = __ldg(src + 1);
+    }
     if (MODE == 0) {
       for (int i = tid; i < p.G * NTOK; i += GT_WARPS * 32)
         if ((i % NTOK) >= p.T) ss[i] = 0.0f;
     } else {
       // fp16 range: one power-of-two prescale for the call so that max |x| stays below 2^15
       float am = 0.0f;
-      const uint4* xv = reinterpret_cast<const uint4*>(p.X);
-      for (int i = tid; i < p.T * (p.d_in >> 3); i += GT_WARPS * 32) am = gv_absmax8(__ldg(xv + i), am);
+      if (one_round) {
+        am = gv_absmax8(c1, gv_absmax8(c0, am));
+      } else {
+        const uint4* xv = reinterpret_cast<const uint4*>(p.X);
+        for (int i = tid; i < p.T * (p.d_in >> 3); i += GT_WARPS * 32) am = gv_absmax8(__ldg(xv + i), am);
+      }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) am = fmaxf(am, __shfl_xor_sync(0xFFFFFFFFu, am, o));
       if (lane == 0) red[warp] = am;
-      for (int i = tid; i < p.G * 16; i += GT_WARPS * 32)
-        if (((i >> 1) & 7) >= p.T) ss[i] = 0.0f;
+      if (MODE == 1)
+        for (int i = tid; i < p.G * 16; i += GT_WARPS * 32)
+          if (((i >> 1) & 7) >= p.T) ss[i] = 0.0f;
       asm volatile("bar.sync 1, 512;" ::: "memory");
       am = red[0];
 #pragma unroll
@@ -302,16 +323,41 @@ lowbit_gemv_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_consta
       asm volatile("bar.sync 1, 512;" ::: "memory");   // red is free again
       if (tid < 32) reinterpret_cast<uint32_t*>(gbase + zero_off)[tid] = 0u;
     }
-    {
+    if (MODE == 0) {
+      // group sums only; eight rounds of loads are in flight at a time (the rounds are L2 round trips).
+      // All CTAs walk x in the same order: starting each at its own offset measured slower.
+      constexpr int DEPTH = 8;
+      for (int i0 = 0; i0 < items; i0 += DEPTH * GT_WARPS * 32) {
+        uint4 xa[DEPTH], xb[DEPTH];
+#pragma unroll
+        for (int u = 0; u < DEPTH; ++u) {
+          const int idx = i0 + u * GT_WARPS * 32 + tid;
+          const int q = idx < items ? idx : 0;
+          const int t = (q >> 2) % p.T, grp = (q >> 2) / p.T;
+          const uint4* src = reinterpret_cast<const uint4*>(p.X + (int64_t)t * p.d_in + grp * 64 + (q & 3) * 16);
+          xa[u] = __ldg(src); xb[u] = __ldg(src + 1);
+        }
+#pragma unroll
+        for (int u = 0; u < DEPTH; ++u) {
+          const int idx = i0 + u * GT_WARPS * 32 + tid;
+          const bool live = idx < items;
+          const int q = live ? idx : 0;
+          const int t = (q >> 2) % p.T, grp = (q >> 2) / p.T;
+          float sum = gv_sum16(xa[u], xb[u]);
+          sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 1);
+          sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 2);
+          if (live && (q & 3) == 0) ss[grp * NTOK + t] = sum;
+        }
+      }
+    } else {
       const float in_scale = 1.0f / y_scale, in_scale16 = in_scale * 0.0625f;
-      const int items = p.G * p.T * 4;
       for (int i0 = 0; i0 < items; i0 += GT_WARPS * 32) {
         const int idx = i0 + tid;
         const bool live = idx < items;
         const int q = live ? idx : 0;
         const int t = (q >> 2) % p.T, grp = (q >> 2) / p.T;
         const uint4* src = reinterpret_cast<const uint4*>(p.X + (int64_t)t * p.d_in + grp * 64 + (q & 3) * 16);
-        const uint4 x0 = __ldg(src), x1 = __ldg(src + 1);
+        const uint4 x0 = i0 == 0 ? c0 : __ldg(src), x1 = i0 == 0 ? c1 : __ldg(src + 1);
         if (MODE == 0) {
           float sum = gv_sum16(x0, x1);
           sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 1);
@@ -339,7 +385,7 @@ lowbit_gemv_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_consta
           ps += __shfl_xor_sync(0xFFFFFFFFu, ps, 1); rs += __shfl_xor_sync(0xFFFFFFFFu, rs, 1);
           ps += __shfl_xor_sync(0xFFFFFFFFu, ps, 2); rs += __shfl_xor_sync(0xFFFFFFFFu, rs, 2);
           if (live) {
-            if ((q & 3) == 0) *reinterpret_cast<float2*>(ss + (grp * 8 + t) * 2) = make_float2(1024.0f * ps, rs);
+            if ((q & 3) == 0) *reinterpret_cast<float2*>(ss + grp * SSG + t * 2) = make_float2(1024.0f * ps, rs);
             xs[q * 2] = make_uint4(f[0], f[1], f[2], f[3]);
             xs[q * 2 + 1] = make_uint4(f[4], f[5], f[6], f[7]);
           }
@@ -369,7 +415,7 @@ lowbit_gemv_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_consta
     const uint32_t xs_addr = base + (xlive[0] ? xs_off + (uint32_t)(g * 4 + tg) * 32u : zero_off + (uint32_t)tg * 32u);
     const uint32_t xs_stride = xlive[0] ? (uint32_t)p.T * 128u : 0u;
     const uint32_t ss_addr = base + ss_off + (MODE == 0 ? 8u * tg : (MODE == 1 ? 16u * tg : 0u));
-    float* my_red = red + warp * GT_ROWS * NTOK;
+    uint32_t rph = 0, rcount = 0;   // phase of the reduction barriers; row blocks done
     const GvConst kc_(0x000F000Fu, 0x00F000F0u, MODE == 0 ? 0x43004300u : 0x64006400u);
     bool ok = true;        // after a timed-out wait the warp keeps walking its loops (so the CTA
                            // barriers still match) but no longer waits or computes
@@ -401,7 +447,7 @@ lowbit_gemv_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_consta
               }
             } else {
               if (MODE == 1) sg[0] = gv_ldsf4<0>(ss_addr + (uint32_t)grp * 64u);
-              else { const float2 v = gv_ldsf2<0>(ss_addr + (uint32_t)grp * 64u); sg[0] = make_float4(v.x, v.y, 0.0f, 0.0f); }
+              else { const float2 v = gv_ldsf2<0>(ss_addr + (uint32_t)grp * 8u); sg[0] = make_float4(v.x, v.y, 0.0f, 0.0f); }
               const uint32_t xa = xs_addr + (uint32_t)grp * xs_stride;
               const uint4 x0 = gv_lds4<0>(xa), x1 = gv_lds4<16>(xa);
               f[0][0] = x0.x; f[0][1] = x0.y; f[0][2] = x0.z; f[0][3] = x0.w;
@@ -459,49 +505,77 @@ lowbit_gemv_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_consta
         }
         if (++s == STAGES) { s = 0; ph ^= 1u; }
       }
-      // end of the row block: sum the sixteen warps in warp order and store
+      // End of the row block, without a CTA-wide barrier.  Every warp writes its partial sums into its
+      // slot (once the warps that summed the previous row block have let go of the buffer) and arrives
+      // on red_done; token t is then summed over the sixteen slots in slot order (deterministic) and
+      // stored by warp (t + row block count) % 16, which is the only warp that waits for the others.
       // accumulator layout: [0],[1] = row g, tokens 2tg, 2tg+1; [2],[3] = row g + 8
+      if (ok && !gv_wait(red_free, rph ^ 1u, p.status)) ok = false;
+      float* my_red = red + warp * GT_ROWS * RT;
+      if (MODE == 2) {
+        if (tg == 0) {
 #pragma unroll
-      for (int j = 0; j < NT; ++j)
-#pragma unroll
-        for (int mt = 0; mt < 2; ++mt) {
-          float* r0 = my_red + (mt * 16 + g) * NTOK + j * 8 + 2 * tg;
-          *reinterpret_cast<float2*>(r0) = make_float2(y[j][mt][0], y[j][mt][1]);
-          *reinterpret_cast<float2*>(r0 + 8 * NTOK) = make_float2(y[j][mt][2], y[j][mt][3]);
+          for (int mt = 0; mt < 2; ++mt) { my_red[mt * 16 + g] = y[0][mt][0]; my_red[mt * 16 + g + 8] = y[0][mt][2]; }
         }
-      asm volatile("bar.sync 1, 512;" ::: "memory");
-      for (int idx = tid; idx < GT_ROWS * NTOK; idx += GT_WARPS * 32) {
-        const int t = idx >> 5, r = idx & 31;               // consecutive threads -> consecutive output rows
-        const int o = rb * GT_ROWS + r;
-        if (t < p.T && o < p.d_out) {
+      } else {
+#pragma unroll
+        for (int j = 0; j < NT; ++j)
+#pragma unroll
+          for (int mt = 0; mt < 2; ++mt) {
+            float* r0 = my_red + (mt * 16 + g) * RT + j * 8 + 2 * tg;
+            *reinterpret_cast<float2*>(r0) = make_float2(y[j][mt][0], y[j][mt][1]);
+            *reinterpret_cast<float2*>(r0 + 8 * RT) = make_float2(y[j][mt][2], y[j][mt][3]);
+          }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(red_done);
+      {
+        const int t = (warp - (int)(rcount & 15u)) & 15;    // the token this warp sums (if it exists)
+        if (t < p.T) {
+          if (ok && !gv_wait(red_done, rph, p.status)) ok = false;
           float a = 0.0f;
 #pragma unroll
-          for (int ww = 0; ww < GT_WARPS; ++ww) a += red[(ww * GT_ROWS + r) * NTOK + t];
+          for (int ww = 0; ww < GT_WARPS; ++ww) a += red[(ww * GT_ROWS + lane) * RT + t];
+          __syncwarp();
+          if (lane == 0) mbar_arrive(red_free);
           a *= y_scale;
-          if (p.y_dtype == QBLORA_BF16) reinterpret_cast<__nv_bfloat16*>(p.Y)[(int64_t)t * p.d_out + o] = __float2bfloat16_rn(a);
-          else reinterpret_cast<float*>(p.Y)[(int64_t)t * p.d_out + o] = a;
+          const int o = rb * GT_ROWS + lane;                // lane = row of the block
+          if (o < p.d_out) {
+            if (p.y_dtype == QBLORA_BF16) reinterpret_cast<__nv_bfloat16*>(p.Y)[(int64_t)t * p.d_out + o] = __float2bfloat16_rn(a);
+            else reinterpret_cast<float*>(p.Y)[(int64_t)t * p.d_out + o] = a;
+          }
         }
       }
-      asm volatile("bar.sync 1, 512;" ::: "memory");   // red is reused by the next block
+      ++rcount;
+      rph ^= 1u;
     }
   }
   __syncthreads();
 }
 
-// dynamic shared memory: alignment slack, stage ring, reduction buffer, barriers, group sums, (MODE 1/2) fragments
+// dynamic shared memory besides the stage ring: alignment slack, reduction buffer, barriers, group
+// sums, (MODE 1/2) fragments and the zero block
 template <int NT, int MODE>
-size_t gt_smem_bytes(int G, int T) {
-  size_t n = 1024 + (size_t)GtCfg<NT, MODE>::STAGES * GT_STAGE_BYTES + GtCfg<NT, MODE>::RED_BYTES + 256 +
-             (size_t)G * GtCfg<NT, MODE>::SS_PER_GROUP * 4;
+size_t gt_fixed_smem(int G, int T) {
+  size_t n = 1024 + GtCfg<NT, MODE>::RED_BYTES + 256 + (size_t)G * GtCfg<NT, MODE>::SS_PER_GROUP * 4;
   if (MODE != 0) n += (size_t)G * T * 128 + 128;
   return n;
 }
+constexpr size_t GT_SMEM_MAX = 227 * 1024;
+template <int NT, int MODE>
+int gt_stages(int G, int T) {   // ring depth that fits; < 4 means this mode does not fit
+  const size_t fixed = gt_fixed_smem<NT, MODE>(G, T);
+  if (fixed + 4 * (size_t)GT_STAGE_BYTES > GT_SMEM_MAX) return 0;
+  const int n = (int)((GT_SMEM_MAX - fixed) / GT_STAGE_BYTES);
+  return n < GtCfg<NT, MODE>::MAX_STAGES ? n : GtCfg<NT, MODE>::MAX_STAGES;
+}
 
 template <int NT, int MODE>
-int gt_launch(const CUtensorMap& tm_c, const CUtensorMap& tm_a, const CUtensorMap& tm_b, const GtParams& p, int grid,
+int gt_launch(const CUtensorMap& tm_c, const CUtensorMap& tm_a, const CUtensorMap& tm_b, GtParams p, int grid,
               cudaStream_t st) {
-  const size_t smem = gt_smem_bytes<NT, MODE>(p.G, p.T);
-  if (smem > 227 * 1024) return QBLORA_ERR_UNSUPPORTED;
+  p.stages = gt_stages<NT, MODE>(p.G, p.T);
+  if (p.stages < 4) return QBLORA_ERR_UNSUPPORTED;
+  const size_t smem = gt_fixed_smem<NT, MODE>(p.G, p.T) + (size_t)p.stages * GT_STAGE_BYTES;
   QB_CUDA(cudaFuncSetAttribute(lowbit_gemv_kernel<NT, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   lowbit_gemv_kernel<NT, MODE><<<grid, GT_THREADS, smem, st>>>(tm_c, tm_a, tm_b, p);
   return QBLORA_OK;
@@ -537,7 +611,7 @@ int launch_lowbit_gemv(const QwView& qw, const __nv_bfloat16* X, int64_t T, void
   { int dev = 0; if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); }
   const int grid = p.n_rb < sms ? p.n_rb : sms;
   // fp16 fragments of x fit in shared memory next to a six-stage ring?
-  const bool xs = NT == 1 && gt_smem_bytes<1, 1>(p.G, p.T) <= 225 * 1024;
+  const bool xs = NT == 1 && (T == 1 ? gt_stages<1, 2>(p.G, p.T) : gt_stages<1, 1>(p.G, p.T)) >= 6;
   {
     DominantKernelTimer timer(st);
     count_launch();

@@ -92,9 +92,12 @@ struct BlockTable {
     o23 = prmt(lo, hi, 0x7362u);
   }
   // eight codes (code e in bits 4e..4e+3 of w) -> eight bf16 values in element order
-  __device__ __forceinline__ void lookup8(uint32_t w, uint32_t (&o)[4]) const {
+  // m4 = 0x44444444 and c3210 = 0x32103210 come in registers: (x & literal) | literal compiles to
+  // two logic ops, the explicit three-input form to one
+  __device__ __forceinline__ void lookup8(uint32_t w, uint32_t (&o)[4], uint32_t m4, uint32_t c3210) const {
     const uint32_t a = w & 0x77777777u;                               // index within an 8-entry half
-    const uint32_t s2 = ((w >> 1) & 0x44444444u) | 0x32103210u;       // byte j: j + 4 * (code >> 3)
+    uint32_t s2;                                                      // byte j: j + 4 * (code >> 3)
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(s2) : "r"(w >> 1), "r"(m4), "r"(c3210));
     half(a, s2, o[0], o[1]);
     half(a >> 16, s2 >> 16, o[2], o[3]);
   }
@@ -220,6 +223,8 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
     const int g = (warp - 2) >> 2;
     const int d = tid - 64 - 128 * g;
     const uint32_t leader_peer = map_to_cta(peer(0), 0);
+    uint32_t k_m4 = 0x44444444u, k_c3210 = 0x32103210u;   // constants of lookup8, pinned to registers
+    asm volatile("" : "+r"(k_m4), "+r"(k_c3210));
     bool ok = true;
     uint32_t it = 0;
     for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
@@ -260,7 +265,7 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             uint32_t o4[4];
-            tab.lookup8(w[j], o4);
+            tab.lookup8(w[j], o4, k_m4, k_c3210);
             st_shared_v4(dst + (((uint32_t)j ^ xr) << 4), o4[0], o4[1], o4[2], o4[3]);
           }
         } else {
