@@ -29,7 +29,7 @@ from paper_2407_17029_b200 import synth  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, per launch, from the ncu
 # capture summarised in profiles/ncu_full_tc_dq_gemm_C2.md (set to None when that kernel changes)
-MEASURED_DRAM_TRAFFIC = {("C2", "GA"): 27.6e6 + 0.27e6}
+MEASURED_DRAM_TRAFFIC = {("C2", "GA"): 27.6e6 + 0.06e6}
 
 METRIC = "fused 4-bit+BLoRA linear fwd+bwd TFLOP/s & low-bit GEMM GB/s, % of roofline"
 
@@ -309,7 +309,8 @@ def run_gpu(args, wl, geom):
             "step_flops": flops_step}
 
     if rank == 0 and not args.no_extras:
-        line["lowbit"] = lowbit_extras(qb, torch, dev, peaks, l2_bytes)
+        line["lowbit"] = lowbit_extras(qb, torch, dev, peaks, l2_bytes, args.lowbit_shapes.split(","),
+                                       [int(t) for t in args.lowbit_tokens.split(",")])
     if rank == 0 and not args.no_cpu_baseline and world == 1:
         rows = args.ref_rows
         cache = oracle_cache(wl, geom, rows)
@@ -323,7 +324,7 @@ def run_gpu(args, wl, geom):
         dist.destroy_process_group()
 
 
-def lowbit_extras(qb, torch, dev, peaks, l2_bytes):
+def lowbit_extras(qb, torch, dev, peaks, l2_bytes, shapes=("q", "up"), tokens=(1, 16)):
     """Deploy path of the QA-BLoRA config: merge, then the low-bit product at 1 and 16 tokens on the
     attention and MLP shapes; GB/s = packed-weight bytes streamed once / kernel time."""
     wl = synth.WORKLOADS["C5"]
@@ -332,7 +333,7 @@ def lowbit_extras(qb, torch, dev, peaks, l2_bytes):
     def bf(a):
         return torch.from_numpy(synth.bf16_bits(a).view(np.int16).copy()).to(dev).view(torch.bfloat16)
 
-    for spec in wl.linears[:2]:
+    for spec in [sp for sp in wl.linears if sp.name in shapes]:
         li = synth.make_linear_inputs(wl, spec, synth.GEOM_A, seed=0, tokens=16)
         dq = qb.quantize_blockwise(torch.from_numpy(li.W).to(dev), 64, 1, qb.FMT_AFFINE_MINMAX)
         li.W = None
@@ -354,7 +355,7 @@ def lowbit_extras(qb, torch, dev, peaks, l2_bytes):
         e.record(); torch.cuda.synchronize()
         out[f"{spec.name}/merge_us"] = s.elapsed_time(e) / 10 * 1e3
         X = bf(li.X)
-        for T in (1, 16):
+        for T in tokens:
             Xt = X[:T].contiguous()
             Y = torch.empty((T, spec.d_out), dtype=torch.bfloat16, device=dev)
             ws = qb.alloc_workspace(qb.OP_LOWBIT_GEMM, copies[0], None, T)
@@ -372,10 +373,33 @@ def lowbit_extras(qb, torch, dev, peaks, l2_bytes):
                 qb.lowbit_gemm(copies[i % ncopies], Xt, ws=ws, out=Y)
             e.record(); torch.cuda.synchronize()
             call_us = s.elapsed_time(e) / reps * 1e3
-            us = statistics.mean(a.elapsed_time(b) for a, b in evs) * 1e3
+            single_us = statistics.mean(a.elapsed_time(b) for a, b in evs) * 1e3
+            # chain time: 2 * ncopies launches over the rotating copies replayed as one CUDA graph, the way a
+            # decode step issues its products back to back; per-launch time = graph time / launches.  An
+            # event pair around ONE launch also counts about 6 us of launch latency that a chain hides.
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            n_chain = 2 * ncopies
+            with torch.cuda.stream(side):
+                qb.lowbit_gemm(copies[0], Xt, ws=ws, out=Y)
+            side.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                for i in range(n_chain):
+                    qb.lowbit_gemm(copies[i % ncopies], Xt, ws=ws, out=Y)
+            for _ in range(3):
+                graph.replay()
+            torch.cuda.synchronize()
+            chain = []
+            for _ in range(10):
+                s.record(); graph.replay(); e.record(); torch.cuda.synchronize()
+                chain.append(s.elapsed_time(e) / n_chain * 1e3)
+            us = statistics.median(chain)
             gbs = nbytes / (us * 1e-6) / 1e9
-            out[f"{spec.name}/T{T}"] = {"kernel_us": us, "GB/s": gbs, "frac_hbm": gbs / peaks["hbm_gbs"],
-                                        "bytes": nbytes, "copies": ncopies, "call_us_back_to_back": call_us}
+            out[f"{spec.name}/T{T}"] = {"kernel_us": us, "timing": f"CUDA-graph chain of {n_chain} launches over {ncopies} weight copies",
+                                        "GB/s": gbs, "frac_hbm": gbs / peaks["hbm_gbs"], "bytes": nbytes, "copies": ncopies,
+                                        "single_launch_event_pair_us": single_us, "call_us_back_to_back": call_us,
+                                        "status": qb.device_status(ws)}
     out["peak_hbm_gbs"] = peaks["hbm_gbs"]
     out["peak_kind"] = peaks["source"]
     return out
@@ -393,6 +417,8 @@ def main():
     ap.add_argument("--ref-max-steps", type=int, default=3)
     ap.add_argument("--no-extras", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--lowbit-shapes", default="q,up", help="linears of C5 timed in the lowbit extras")
+    ap.add_argument("--lowbit-tokens", default="1,16", help="token counts timed in the lowbit extras")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "gpu" else args.warmup
     wl = synth.WORKLOADS[args.workload]
