@@ -299,7 +299,7 @@ lowbit_gemv_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_consta
       for (int i = tid; i < p.G * NTOK; i += GT_WARPS * 32)
         if ((i % NTOK) >= p.T) ss[i] = 0.0f;
     } else {
-      // fp16 range: one power-of-two prescale for the call so that max |x| stays below 2^15
+      // fp16 range: one power-of-two prescale for the call brings max |x| just below 2^15 (up or down)
       float am = 0.0f;
       if (one_round) {
         am = gv_absmax8(c1, gv_absmax8(c0, am));
@@ -317,8 +317,8 @@ lowbit_gemv_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_consta
       am = red[0];
 #pragma unroll
       for (int i = 1; i < GT_WARPS; ++i) am = fmaxf(am, red[i]);
-      int e = (int)((__float_as_uint(am) >> 23) & 0xFFu) - 127 - 14;
-      e = e < 0 ? 0 : (e > 120 ? 120 : e);
+      int e = (int)((__float_as_uint(am) >> 23) & 0xFFu) - 127 - 14;   // max |x| * 2^-e in [2^14, 2^15)
+      e = e < -100 ? -100 : (e > 120 ? 120 : e);
       y_scale = __uint_as_float((uint32_t)(127 + e) << 23);
       asm volatile("bar.sync 1, 512;" ::: "memory");   // red is free again
       if (tid < 32) reinterpret_cast<uint32_t*>(gbase + zero_off)[tid] = 0u;

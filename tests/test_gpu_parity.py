@@ -211,3 +211,18 @@ def test_lowbit_gemm_parity(qb, path, T):
     dq, Xd = qweight_to_dev(qw), to_bf16_dev(X)
     gate_strict(to_np64(qb.lowbit_gemm(dq, Xd, torch.float32)), ref, f"lowbit T={T} f32")
     gate_bf16(to_np64(qb.lowbit_gemm(dq, Xd, torch.bfloat16)), ref, f"lowbit T={T} bf16")
+
+
+@pytest.mark.parametrize("T", [1, 3, 16])
+@pytest.mark.parametrize("log2_gain", [-40, 0, 22])
+def test_lowbit_decode_token_range(qb, T, log2_gain):
+    # The small-T path holds x in fp16 after a power-of-two prescale: tokens far above fp16's
+    # largest value and far below its smallest normal must come out as exactly as ordinary ones.
+    # One token carries a single huge outlier so that most of its elements sit 2^17 below its maximum.
+    qw, _, X, _ = make_case(57, T, 328, 448, 64, 8, 16, qfmt=1)
+    X = X.copy()
+    X[0, 5] *= np.float32(2.0 ** 17)
+    X = synth.round_to_bf16(X * np.float32(2.0 ** log2_gain))
+    ref = oracle.lowbit_gemm(qw, X)
+    dq, Xd = qweight_to_dev(qw), to_bf16_dev(X)
+    gate_strict(to_np64(qb.lowbit_gemm(dq, Xd, torch.float32)), ref, f"lowbit range T={T} gain=2^{log2_gain}")
