@@ -324,7 +324,7 @@ def run_gpu(args, wl, geom):
         dist.destroy_process_group()
 
 
-def lowbit_extras(qb, torch, dev, peaks, l2_bytes, shapes=("q", "up"), tokens=(1, 16)):
+def lowbit_extras(qb, torch, dev, peaks, l2_bytes, shapes=("q", "up"), tokens=(1, 16, 2048)):
     """Deploy path of the QA-BLoRA config: merge, then the low-bit product at 1 and 16 tokens on the
     attention and MLP shapes; GB/s = packed-weight bytes streamed once / kernel time."""
     wl = synth.WORKLOADS["C5"]
@@ -335,8 +335,20 @@ def lowbit_extras(qb, torch, dev, peaks, l2_bytes, shapes=("q", "up"), tokens=(1
 
     for spec in [sp for sp in wl.linears if sp.name in shapes]:
         li = synth.make_linear_inputs(wl, spec, synth.GEOM_A, seed=0, tokens=16)
-        dq = qb.quantize_blockwise(torch.from_numpy(li.W).to(dev), 64, 1, qb.FMT_AFFINE_MINMAX)
+        Wd = torch.from_numpy(li.W).to(dev)
+        dq = qb.quantize_blockwise(Wd, 64, 1, qb.FMT_AFFINE_MINMAX)
         li.W = None
+        # quantizer: reads the fp32 weight once (larger than L2), writes codes + alpha + beta
+        s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s.record()
+        for _ in range(3):
+            qb.quantize_blockwise(Wd, 64, 1, qb.FMT_AFFINE_MINMAX)
+        e.record(); torch.cuda.synchronize()
+        q_us = s.elapsed_time(e) / 3 * 1e3
+        q_bytes = Wd.numel() * 4 + packed_bytes(spec.d_out, spec.d_in)
+        out[f"{spec.name}/quantize"] = {"us": q_us, "GB/s": q_bytes / q_us / 1e3, "frac_hbm": q_bytes / q_us / 1e3 / peaks["hbm_gbs"],
+                                        "bytes": q_bytes, "note": "includes the binding's output allocation"}
+        del Wd
         ad = qb.Adapter(64, 8, wl.rank, 1.0, bf(li.A), bf(li.B))
         nbytes = packed_bytes(spec.d_out, spec.d_in)
         ncopies = int(np.ceil(2.0 * l2_bytes / nbytes)) + 1
@@ -346,7 +358,6 @@ def lowbit_extras(qb, torch, dev, peaks, l2_bytes, shapes=("q", "up"), tokens=(1
             copies.append(qb.QWeight(m.d_out, m.d_in, 64, 1, m.qfmt, m.code, m.codes.clone(), m.alpha.clone(), m.beta.clone()))
         # merge timing
         wsm = qb.alloc_workspace(qb.OP_MERGE, dq, ad, 0)
-        s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         for _ in range(3):
             qb.merge(dq, ad, ws=wsm)
         s.record()
@@ -356,6 +367,23 @@ def lowbit_extras(qb, torch, dev, peaks, l2_bytes, shapes=("q", "up"), tokens=(1
         out[f"{spec.name}/merge_us"] = s.elapsed_time(e) / 10 * 1e3
         X = bf(li.X)
         for T in tokens:
+            if T > 16:
+                # prefill-shaped product: the fused dequant GEMM with the min-max table; tensor-bound
+                Xl = bf(synth.make_activations(0, f"C5/{spec.name}/Xl", T, spec.d_in)[0])
+                Yl = torch.empty((T, spec.d_out), dtype=torch.bfloat16, device=dev)
+                wsl = qb.alloc_workspace(qb.OP_LOWBIT_GEMM, copies[0], None, T)
+                for i in range(3):
+                    qb.lowbit_gemm(copies[i % ncopies], Xl, ws=wsl, out=Yl)
+                s.record()
+                for i in range(10):
+                    qb.lowbit_gemm(copies[i % ncopies], Xl, ws=wsl, out=Yl)
+                e.record(); torch.cuda.synchronize()
+                us = s.elapsed_time(e) / 10 * 1e3
+                tf = 2.0 * T * spec.d_in * spec.d_out / us / 1e6
+                out[f"{spec.name}/T{T}"] = {"us": us, "TFLOP/s": tf, "frac_bf16_sustained": tf / peaks["bf16_tflops_sustained"],
+                                            "status": qb.device_status(wsl)}
+                del Xl, Yl
+                continue
             Xt = X[:T].contiguous()
             Y = torch.empty((T, spec.d_out), dtype=torch.bfloat16, device=dev)
             ws = qb.alloc_workspace(qb.OP_LOWBIT_GEMM, copies[0], None, T)
@@ -418,7 +446,7 @@ def main():
     ap.add_argument("--no-extras", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--lowbit-shapes", default="q,up", help="linears of C5 timed in the lowbit extras")
-    ap.add_argument("--lowbit-tokens", default="1,16", help="token counts timed in the lowbit extras")
+    ap.add_argument("--lowbit-tokens", default="1,16,2048", help="token counts timed in the lowbit extras")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "gpu" else args.warmup
     wl = synth.WORKLOADS[args.workload]
