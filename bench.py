@@ -238,6 +238,7 @@ def run_gpu(args, wl, geom):
         a.record(); b.record()
     launches0 = qb.kernel_launches()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # ---- eager pass: every call launched from the host; the library brackets the dominant kernel
     barrier()
     e0.record()
     for i in range(args.steps):
@@ -245,9 +246,32 @@ def run_gpu(args, wl, geom):
     e1.record()
     barrier()
     launches = qb.kernel_launches() - launches0
-    ms = e0.elapsed_time(e1)
-    clocks = sampler.stop()
+    eager_ms = e0.elapsed_time(e1)
     dom_ms = statistics.mean(a.elapsed_time(b) for a, b, _ in kev)
+    ms = eager_ms
+    mode = "eager launches"
+    if not args.no_graph:
+        # ---- the same steps replayed as CUDA graphs (one graph per buffer set, one step each): the small
+        # adapter-side kernels are launch-bound when issued from the host one by one
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        graphs = []
+        for si in range(nsets):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                step(si)
+            graphs.append(g)
+        for i in range(args.warmup):
+            graphs[i % nsets].replay()
+        barrier()
+        e0.record()
+        for i in range(args.steps):
+            graphs[(args.warmup + i) % nsets].replay()
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        mode = "CUDA-graph replay, one graph per buffer set"
+    clocks = sampler.stop()
     for spec, q2, ad, X, dY, Y, dX, dA, dB, wsf, wsb in sets[0]:
         assert qb.device_status(wsf) == qb.OK and qb.device_status(wsb) == qb.OK
     if dist is not None:
@@ -297,6 +321,7 @@ def run_gpu(args, wl, geom):
                        "tokens": T, "linears": [f"{s.name}[{s.d_out},{s.d_in}]" for s in wl.linears], "rank": r,
                        "quant": "4-bit, block 64 along input, " + ("min-max" if wl.qfmt else "level table + absmax"),
                        "parallelism": "replicas only" if world > 1 else "single GPU",
+                       "launch": mode,
                        "l2": f"rotating over {nsets} distinct buffer sets ({nsets * step_bytes / 2**20:.0f} MiB > 2x L2)"},
             "clocks": clocks, "gpu_launches": int(launches),
             "e2e": {"value": e2e_val, "unit": "TFLOP/s", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
@@ -306,7 +331,9 @@ def run_gpu(args, wl, geom):
                          "peak_kind": f"bf16 dense, sustained, {peaks['source']}", "unit": "TFLOP/s",
                          "frac": dom_flops / (dom_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
                          "traffic": MEASURED_DRAM_TRAFFIC.get((wl.name, geom.name)), "ms_per_launch": dom_ms},
-            "step_flops": flops_step}
+            "step_flops": flops_step,
+            "eager": {"ms_per_step": eager_ms / args.steps, "value": flops_step * args.steps / (eager_ms * 1e-3) / 1e12,
+                      "unit": "TFLOP/s", "note": "this rank, every call launched from the host"}}
 
     if rank == 0 and not args.no_extras:
         line["lowbit"] = lowbit_extras(qb, torch, dev, peaks, l2_bytes, args.lowbit_shapes.split(","),
@@ -445,6 +472,7 @@ def main():
     ap.add_argument("--ref-max-steps", type=int, default=3)
     ap.add_argument("--no-extras", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of graph replay")
     ap.add_argument("--lowbit-shapes", default="q,up", help="linears of C5 timed in the lowbit extras")
     ap.add_argument("--lowbit-tokens", default="1,16,2048", help="token counts timed in the lowbit extras")
     args = ap.parse_args()

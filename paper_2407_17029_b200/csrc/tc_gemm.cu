@@ -24,6 +24,7 @@
 
 #include "common.cuh"
 #include "simt_gemm.cuh"
+#include <cstdlib>
 #include "tc_ptx.cuh"
 #include "tc_small.cuh"
 
@@ -613,12 +614,50 @@ int tc_linear_fwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, in
   return launch_main(0, qw, ad, X, w.u16, w.ldr, T, Y, y_dtype, status, st);
 }
 
+namespace {
+// Second stream for the backward's adapter-gradient chain, so that it runs beside the dX contraction
+// (whose last wave leaves SMs idle) instead of in front of it.  Created on first use, per host thread
+// and device; the events only order work (no timing).
+struct SideLane {
+  cudaStream_t stream = nullptr;
+  cudaEvent_t fork = nullptr, du_done = nullptr, join = nullptr;
+  bool ok = false, tried = false;
+};
+SideLane* side_lane() {
+  static thread_local SideLane lanes[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  SideLane& l = lanes[dev];
+  if (!l.tried) {
+    l.tried = true;
+    const char* off = getenv("QBLORA_NO_OVERLAP");
+    if (!(off && off[0] == '1') &&
+        cudaStreamCreateWithFlags(&l.stream, cudaStreamNonBlocking) == cudaSuccess &&
+        cudaEventCreateWithFlags(&l.fork, cudaEventDisableTiming) == cudaSuccess &&
+        cudaEventCreateWithFlags(&l.du_done, cudaEventDisableTiming) == cudaSuccess &&
+        cudaEventCreateWithFlags(&l.join, cudaEventDisableTiming) == cudaSuccess)
+      l.ok = true;
+  }
+  return l.ok ? &l : nullptr;
+}
+}  // namespace
+
 int tc_linear_bwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, const __nv_bfloat16* dY, int64_t T,
                   void* dX, int dx_dtype, float* dA, float* dB, char* ws, cudaStream_t st) {
   TcWs w = carve(QBLORA_OP_LINEAR_BWD, ad, T, ws);
   int* status = reinterpret_cast<int*>(ws);
   int rc;
   if (ad) {
+    // Two chains: (a) dv -> du, which the dX contraction needs; (b) pooled x -> u -> dB, dA, which
+    // nothing else needs.  With a side lane (b) runs on it: it starts together with (a), waits for du
+    // before the gradient products, and is joined at the end; the caller's stream goes straight from
+    // (a) to the dX contraction.
+    SideLane* lane = (dX && (dA || dB)) ? side_lane() : nullptr;
+    cudaStream_t sb = lane ? lane->stream : st;
+    if (lane) {
+      QB_CUDA(cudaEventRecord(lane->fork, st));
+      QB_CUDA(cudaStreamWaitEvent(lane->stream, lane->fork, 0));
+    }
     const int64_t n = T * ad->Q;
     if (segsum_fast_ok(qw.d_out, ad->l2)) {
       const int64_t chunks = T * (qw.d_out / 8);
@@ -636,21 +675,25 @@ int tc_linear_bwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, co
       rc = small_gemm((int)T, ad->r, segs, 2, out, status, st);
       if (rc) return rc;
     }
+    if (lane) QB_CUDA(cudaEventRecord(lane->du_done, st));
     if (dA || dB) {
-      rc = launch_pool(qw, *ad, X, T, w, st);
+      rc = launch_pool(qw, *ad, X, T, w, sb);
       if (rc) return rc;
     }
     if (dB) {
       SgOut uo{};
       uo.hi = w.uh; uo.lo = w.ul; uo.ld16 = w.ldr;
-      rc = launch_u_gemm(*ad, T, w, uo, status, st);
+      rc = launch_u_gemm(*ad, T, w, uo, status, sb);
       if (rc) return rc;
+    }
+    if (lane) QB_CUDA(cudaStreamWaitEvent(lane->stream, lane->du_done, 0));   // dv and du are complete
+    if (dB) {
       // dB[k][q] = sum_t u[t][k] dv[t][q]: both operands token-major, i.e. MN-contiguous
       const SgOperand uh{w.uh, w.ldr, false}, ul{w.ul, w.ldr, false}, dh{w.dvh, w.ldq, false}, dl{w.dvl, w.ldq, false};
       SgSegment segs[3] = {{uh, dh, (int)T}, {ul, dh, (int)T}, {uh, dl, (int)T}};
       SgOut out{};
       out.f32 = dB; out.ld32 = ad->Q;
-      rc = small_gemm(ad->r, ad->Q, segs, 3, out, status, st, w.partial);
+      rc = small_gemm(ad->r, ad->Q, segs, 3, out, status, sb, w.partial);
       if (rc) return rc;
     }
     if (dA) {
@@ -659,8 +702,14 @@ int tc_linear_bwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, co
       SgSegment segs[3] = {{xh, dh, (int)T}, {xl, dh, (int)T}, {xh, dl, (int)T}};
       SgOut out{};
       out.f32 = dA; out.ld32 = ad->r;
-      rc = small_gemm(ad->P, ad->r, segs, 3, out, status, st, w.partial);
+      rc = small_gemm(ad->P, ad->r, segs, 3, out, status, sb, w.partial);
       if (rc) return rc;
+    }
+    if (lane) {
+      QB_CUDA(cudaEventRecord(lane->join, lane->stream));
+      rc = dX ? launch_main(1, qw, ad, dY, w.du16, w.ldr, T, dX, dx_dtype, status, st) : QBLORA_OK;
+      QB_CUDA(cudaStreamWaitEvent(st, lane->join, 0));   // the call's work is complete when st is
+      return rc;
     }
   }
   if (!dX) return QBLORA_OK;
