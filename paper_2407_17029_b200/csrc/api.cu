@@ -86,7 +86,7 @@ size_t ws_bytes_impl(int op, const QwView& q, const AdView* ad, int64_t T) {
       return simt_ws_bytes(op, q, ad, T);
     case QBLORA_OP_MERGE: return ad ? merge_ws_bytes(q, *ad) : 0;
     case QBLORA_OP_LOWBIT_GEMM:
-      if (gemv_supported(q, T)) return kStatusBytes;
+      if (gemv_supported(q, T)) return gemv_ws_bytes(q, T);
       if (!force_general() && tc_supported(q, nullptr, T)) return tc_ws_bytes(QBLORA_OP_LINEAR_FWD, q, nullptr, T);
       return simt_ws_bytes(QBLORA_OP_LINEAR_FWD, q, nullptr, T);
     default: return 0;

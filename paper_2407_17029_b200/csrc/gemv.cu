@@ -22,6 +22,7 @@
 //   alpha * sum((128 + c) x) + (beta - 128 alpha) * S  =  alpha * sum(c x) + beta * S.
 // When T * D_in is small enough the permuted token fragments are also kept in shared memory for the
 // life of the CTA; otherwise they are rebuilt per group from global x (L1-resident).
+#include <cstdlib>
 #include "tc_ptx.cuh"
 #include "tc_small.cuh"
 
@@ -171,6 +172,18 @@ __device__ __forceinline__ float4 gv_ldsf4(uint32_t addr) {
   float4 v;
   asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4 + %5];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr), "n"(OFF));
   return v;
+}
+
+// Release of a shared-memory buffer to the producer.  The arrival names values computed from
+// everything the warp loaded from the buffer, so it cannot be issued before those loads have
+// returned: a load that is merely issued may still be in flight when the refill lands.
+__device__ __forceinline__ void gv_release(uint32_t bar, float d0, float d1, float d2, float d3) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];  // after %1 %2 %3 %4"
+               ::"r"(bar), "f"(d0), "f"(d1), "f"(d2), "f"(d3) : "memory");
+}
+__device__ __forceinline__ void gv_release_u(uint32_t bar, uint32_t d0, uint32_t d1, float d2, float d3) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];  // after %1 %2 %3 %4"
+               ::"r"(bar), "r"(d0), "r"(d1), "f"(d2), "f"(d3) : "memory");
 }
 
 // Waits of this kernel pass a suspend-time hint so that a waiting warp sleeps in hardware until the
@@ -501,7 +514,7 @@ lowbit_gemv_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_consta
             }
           }
           __syncwarp();
-          if (lane == 0) mbar_arrive(empty(s));   // this warp is done reading the stage
+          if (lane == 0) gv_release(empty(s), y[0][0][0], y[0][0][2], y[0][1][0], y[0][1][2]);   // this warp is done reading the stage
         }
         if (++s == STAGES) { s = 0; ph ^= 1u; }
       }
@@ -537,7 +550,7 @@ lowbit_gemv_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_consta
 #pragma unroll
           for (int ww = 0; ww < GT_WARPS; ++ww) a += red[(ww * GT_ROWS + lane) * RT + t];
           __syncwarp();
-          if (lane == 0) mbar_arrive(red_free);
+          if (lane == 0) gv_release(red_free, a, a, a, a);
           a *= y_scale;
           const int o = rb * GT_ROWS + lane;                // lane = row of the block
           if (o < p.d_out) {
@@ -581,6 +594,301 @@ int gt_launch(const CUtensorMap& tm_c, const CUtensorMap& tm_a, const CUtensorMa
   return QBLORA_OK;
 }
 
+// ---------------------------------------------------------------------------------------------------
+// K-outer variant for 2..16 tokens.  A small kernel first turns x into fp16 MMA fragments in the
+// workspace: per K tile a contiguous block [16 groups][NTOK tokens][4 quarters][32 B] plus, per group
+// and token, (1024 P 2^e, R 2^e, 2^e, 0), where 2^-e is that 64-value slice's own power-of-two
+// prescale, P the sum of the fragment values and R the sum of the scaled x (so no pass over all of x
+// is needed and tokens of very different magnitude do not share a scale).  The main kernel makes the
+// K tiles the OUTER loop: the producer streams a K tile's fragment block into shared memory once
+// (bulk copy, double-buffered) and then the weight tiles of the CTA's RB row blocks for that K tile.
+// A warp takes its group's fragments into registers once per K tile and reuses them for the RB row
+// blocks, so the main loop has no global loads, no byte permutes and the cheaper fp16 unpack, and x
+// crosses L2 -> SM once per RB row blocks.  The RB accumulators stay in registers.
+template <int NT>
+struct KoCfg {
+  static constexpr int NTOK = NT * 8;
+  static constexpr int RB = NT == 1 ? 4 : 2;                       // row blocks per pass (register budget)
+  static constexpr int XBUF_BYTES = GT_GROUPS * NTOK * 128;        // fragments of one K tile
+  static constexpr int SBUF_BYTES = GT_GROUPS * NTOK * 16;         // float4 per group and token
+  static constexpr int KT_BYTES = XBUF_BYTES + SBUF_BYTES;         // one K tile's block in the workspace
+  static constexpr int RED_BYTES = GT_WARPS * GT_ROWS * NTOK * 4;
+  static constexpr int FIXED = 1024 + 2 * KT_BYTES + RED_BYTES + 512;
+};
+
+__device__ __forceinline__ void gv_bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+// one thread per (K tile, group, token, quarter): 16 values of x -> 32 bytes of fragments
+template <int NT>
+__global__ void __launch_bounds__(256) x_prepare_kernel(const __nv_bfloat16* __restrict__ X, int T, int d_in, int G,
+                                                        int n_kc, uint8_t* __restrict__ out) {
+  using Cfg = KoCfg<NT>;
+  constexpr int NTOK = Cfg::NTOK;
+  const int idx = blockIdx.x * 256 + threadIdx.x;
+  const int total = n_kc * GT_GROUPS * NTOK * 4;
+  const bool in_range = idx < total;
+  const int q = in_range ? idx : 0;
+  const int tg = q & 3, t = (q >> 2) % NTOK, gl = ((q >> 2) / NTOK) % GT_GROUPS, kc = (q >> 2) / (NTOK * GT_GROUPS);
+  const int grp = kc * GT_GROUPS + gl;
+  uint4 xa = make_uint4(0, 0, 0, 0), xb = make_uint4(0, 0, 0, 0);
+  if (in_range && t < T && grp < G) {
+    const uint4* src = reinterpret_cast<const uint4*>(X + (int64_t)t * d_in + grp * 64 + tg * 16);
+    xa = __ldg(src); xb = __ldg(src + 1);
+  }
+  float am = gv_absmax8(xb, gv_absmax8(xa, 0.0f));
+  am = fmaxf(am, __shfl_xor_sync(0xFFFFFFFFu, am, 1));
+  am = fmaxf(am, __shfl_xor_sync(0xFFFFFFFFu, am, 2));
+  int e = (int)((__float_as_uint(am) >> 23) & 0xFFu) - 127 - 14;     // max |x| 2^-e in [2^14, 2^15)
+  e = e < -100 ? -100 : (e > 120 ? 120 : e);
+  const float up = __uint_as_float((uint32_t)(127 + e) << 23), dn = __uint_as_float((uint32_t)(127 - e) << 23);
+  const float dn16 = dn * 0.0625f;
+  const uint32_t xw[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
+  uint32_t f[8];
+  float ps = 0.0f, rs = 0.0f;   // sum of fragment values; sum of scaled x as the fragments hold it
+#pragma unroll
+  for (int wd = 0; wd < 2; ++wd)
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const uint32_t wa = xw[4 * wd + h], wb = xw[4 * wd + h + 2];
+      const uint32_t ev = gv_pack_h2(__uint_as_float(wa << 16) * dn, __uint_as_float(wb << 16) * dn);
+      const uint32_t od = gv_pack_h2(__uint_as_float(wa & 0xFFFF0000u) * dn16, __uint_as_float(wb & 0xFFFF0000u) * dn16);
+      f[2 * (2 * wd + h)] = ev;
+      f[2 * (2 * wd + h) + 1] = od;
+      const float se = gv_h_lo(ev) + gv_h_hi(ev), so = gv_h_lo(od) + gv_h_hi(od);
+      ps += se + so;
+      rs += se + 16.0f * so;
+    }
+  ps += __shfl_xor_sync(0xFFFFFFFFu, ps, 1); rs += __shfl_xor_sync(0xFFFFFFFFu, rs, 1);
+  ps += __shfl_xor_sync(0xFFFFFFFFu, ps, 2); rs += __shfl_xor_sync(0xFFFFFFFFu, rs, 2);
+  if (in_range) {
+    uint8_t* blk = out + (size_t)kc * Cfg::KT_BYTES;
+    const uint32_t item = (uint32_t)(gl * NTOK + t);
+    uint4* dst = reinterpret_cast<uint4*>(blk + item * 128u + (uint32_t)tg * 32u);
+    dst[0] = make_uint4(f[0], f[1], f[2], f[3]);
+    dst[1] = make_uint4(f[4], f[5], f[6], f[7]);
+    if (tg == 0) *reinterpret_cast<float4*>(blk + Cfg::XBUF_BYTES + item * 16u) = make_float4(1024.0f * ps * up, rs * up, up, 0.0f);
+  }
+}
+
+template <int NT>
+__global__ void __launch_bounds__(GT_THREADS, 1)
+lowbit_gemv_ko_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_constant__ CUtensorMap tm_a,
+                      const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ GtParams p,
+                      const uint8_t* __restrict__ xfrag) {
+  using Cfg = KoCfg<NT>;
+  constexpr int NTOK = Cfg::NTOK, RB = Cfg::RB;
+  const int STAGES = p.stages;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* gbase = smem_raw + (base - raw);
+  const uint32_t xbuf_off = STAGES * GT_STAGE_BYTES;                    // [2] x (fragments, then float4 per group, token)
+  const uint32_t red_off = xbuf_off + 2 * Cfg::KT_BYTES;
+  float* red = reinterpret_cast<float*>(gbase + red_off);               // [16 warps][32 rows][NTOK]
+  const uint32_t bars = base + red_off + Cfg::RED_BYTES;
+  auto full = [&](int s) { return bars + 8u * s; };
+  auto empty = [&](int s) { return bars + 8u * (STAGES + s); };
+  const uint32_t red_done = bars + 8u * (2 * STAGES);
+  const uint32_t red_free = bars + 8u * (2 * STAGES + 1);
+  auto xfull = [&](uint32_t b) { return bars + 8u * (2 * STAGES + 2 + b); };
+  auto xempty = [&](uint32_t b) { return bars + 8u * (2 * STAGES + 4 + b); };
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (tid == 0) {
+    if (blockIdx.x == 0) *p.status = 0;   // any give-up below is written at least a wait limit later
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), GT_WARPS); }
+    mbar_init(red_done, GT_WARPS);
+    mbar_init(red_free, p.T);
+    for (uint32_t b = 0; b < 2; ++b) { mbar_init(xfull(b), 1); mbar_init(xempty(b), GT_WARPS); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  const int n_pass = (p.n_rb + gridDim.x * RB - 1) / (gridDim.x * RB);   // passes of RB row blocks per CTA
+
+  if (warp == GT_WARPS) {
+    // ------------------------------------------------------------------ producer (one lane)
+    if (lane == 0) {
+      uint32_t it = 0, ph = 0, xit = 0;
+      int s = 0;
+      bool ok = true;
+      for (int pass = 0; pass < n_pass && ok; ++pass) {
+        if (pass * RB * (int)gridDim.x + (int)blockIdx.x >= p.n_rb) break;   // no row block left for this CTA
+        for (int kc = 0; kc < p.n_kc && ok; ++kc, ++xit) {
+          const uint32_t xb = xit & 1u;
+          if (!gv_wait(xempty(xb), ((xit >> 1) & 1u) ^ 1u, p.status)) { ok = false; break; }
+          mbar_arrive_expect_tx(xfull(xb), Cfg::KT_BYTES);
+          gv_bulk_load(base + xbuf_off + xb * Cfg::KT_BYTES, xfrag + (size_t)kc * Cfg::KT_BYTES, Cfg::KT_BYTES, xfull(xb));
+          for (int j = 0; j < RB; ++j) {
+            const int rb = (pass * RB + j) * gridDim.x + blockIdx.x;
+            if (rb >= p.n_rb) break;
+            if (!gv_wait(empty(s), ph ^ 1u, p.status)) { ok = false; break; }
+            const uint32_t st = base + s * GT_STAGE_BYTES;
+            mbar_arrive_expect_tx(full(s), GT_STAGE_BYTES);
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+              tma_load_2d(st + q * 4096, &tm_c, full(s), (kc * GT_GROUPS + q * 4) * 8, rb * GT_ROWS);
+            tma_load_2d(st + GT_CODE_BYTES, &tm_a, full(s), kc * GT_GROUPS, rb * GT_ROWS);
+            tma_load_2d(st + GT_CODE_BYTES + GT_SCALE_BYTES, &tm_b, full(s), kc * GT_GROUPS, rb * GT_ROWS);
+            ++it;
+            if (++s == STAGES) { s = 0; ph ^= 1u; }
+          }
+        }
+      }
+      if (!ok) {   // give copies already in flight a bounded chance to land before the CTA exits
+        const uint32_t lo = it > (uint32_t)STAGES ? it - STAGES : 0;
+        for (uint32_t j = lo; j < it; ++j) gv_wait(full(j % STAGES), (j / STAGES) & 1u, p.status);
+        const uint32_t xlo = xit > 2u ? xit - 2u : 0u;
+        for (uint32_t j = xlo; j < xit; ++j) gv_wait(xfull(j & 1u), (j >> 1) & 1u, p.status);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ compute warps
+    const int g = lane >> 2, tg = lane & 3;
+    const uint32_t code_off = ((uint32_t)warp >> 2) * 4096u + (uint32_t)g * 128u +
+                              ((((((uint32_t)warp & 3u) << 1) | ((uint32_t)tg >> 1)) ^ (uint32_t)g) << 4) +
+                              (((uint32_t)tg & 1u) << 3);
+    const uint32_t scale_off = GT_CODE_BYTES + (uint32_t)g * 64u +
+                               ((((uint32_t)warp >> 2) ^ (((uint32_t)g >> 1) & 3u)) << 4) + ((uint32_t)warp & 3u) * 4u;
+    const GvConst kc_(0x000F000Fu, 0x00F000F0u, 0x64006400u);
+    // B fragment of lane (g, tg) = token g (+ 8 n), quarter tg, of this warp's group
+    const uint32_t xrd = base + xbuf_off + ((uint32_t)warp * NTOK + (uint32_t)g) * 128u + (uint32_t)tg * 32u;
+    const uint32_t srd = base + xbuf_off + Cfg::XBUF_BYTES + ((uint32_t)warp * NTOK + 2u * (uint32_t)tg) * 16u;
+    bool ok = true;
+    int s = 0;
+    uint32_t ph = 0, rph = 0, rcount = 0, xit = 0;
+    for (int pass = 0; pass < n_pass; ++pass) {
+      if (pass * RB * (int)gridDim.x + (int)blockIdx.x >= p.n_rb) break;
+      float y[RB][NT][2][4];
+#pragma unroll
+      for (int j = 0; j < RB; ++j)
+#pragma unroll
+        for (int n = 0; n < NT; ++n)
+#pragma unroll
+          for (int mt = 0; mt < 2; ++mt) { y[j][n][mt][0] = y[j][n][mt][1] = y[j][n][mt][2] = y[j][n][mt][3] = 0.0f; }
+      for (int kc = 0; kc < p.n_kc; ++kc, ++xit) {
+        // ---- this warp's group of the K tile: fragments and offsets into registers, once for all row blocks
+        const uint32_t xb = xit & 1u;
+        if (ok && !gv_wait(xfull(xb), (xit >> 1) & 1u, p.status)) ok = false;
+        uint32_t f[NT][8];
+        float4 sg[NT][2];
+#pragma unroll
+        for (int n = 0; n < NT; ++n) {
+          const uint32_t xa_ = xrd + xb * Cfg::KT_BYTES + (uint32_t)n * (8u * 128u);
+          const uint4 x0 = gv_lds4<0>(xa_), x1 = gv_lds4<16>(xa_);
+          f[n][0] = x0.x; f[n][1] = x0.y; f[n][2] = x0.z; f[n][3] = x0.w;
+          f[n][4] = x1.x; f[n][5] = x1.y; f[n][6] = x1.z; f[n][7] = x1.w;
+          const uint32_t sa_ = srd + xb * Cfg::KT_BYTES + (uint32_t)n * (8u * 16u);
+          sg[n][0] = gv_ldsf4<0>(sa_); sg[n][1] = gv_ldsf4<16>(sa_);
+        }
+        __syncwarp();
+        const bool group_live = kc * GT_GROUPS + warp < p.G;
+#pragma unroll
+        for (int j = 0; j < RB; ++j) {
+          const int rb = (pass * RB + j) * gridDim.x + blockIdx.x;
+          if (rb >= p.n_rb) break;
+          if (ok && !gv_wait(full(s), ph, p.status)) ok = false;
+          if (ok) {
+            if (group_live) {
+              const uint32_t sb = base + (uint32_t)s * GT_STAGE_BYTES;
+              const uint32_t ca = sb + code_off, sa = sb + scale_off;
+              uint2 w0[2], w1[2];
+              float a0[2], a1[2], b0[2], b1[2];
+              w0[0] = gv_lds2<0>(ca); w1[0] = gv_lds2<1024>(ca); w0[1] = gv_lds2<2048>(ca); w1[1] = gv_lds2<3072>(ca);
+              a0[0] = gv_ldsf<0>(sa); a1[0] = gv_ldsf<512>(sa); a0[1] = gv_ldsf<1024>(sa); a1[1] = gv_ldsf<1536>(sa);
+              b0[0] = gv_ldsf<GT_SCALE_BYTES>(sa); b1[0] = gv_ldsf<GT_SCALE_BYTES + 512>(sa);
+              b0[1] = gv_ldsf<GT_SCALE_BYTES + 1024>(sa); b1[1] = gv_ldsf<GT_SCALE_BYTES + 1536>(sa);
+#pragma unroll
+              for (int mt = 0; mt < 2; ++mt) {
+                uint32_t va[2][4], vb[2][4];
+                gv_unpack_h(w0[mt].x, va[0], kc_); gv_unpack_h(w0[mt].y, va[1], kc_);
+                gv_unpack_h(w1[mt].x, vb[0], kc_); gv_unpack_h(w1[mt].y, vb[1], kc_);
+#pragma unroll
+                for (int n = 0; n < NT; ++n) {
+                  float acc[4];
+                  gv_mma0_h(acc, va[0][0], vb[0][0], va[0][1], vb[0][1], f[n][0], f[n][1]);
+                  gv_mma_h(acc, va[0][2], vb[0][2], va[0][3], vb[0][3], f[n][2], f[n][3]);
+                  gv_mma_h(acc, va[1][0], vb[1][0], va[1][1], vb[1][1], f[n][4], f[n][5]);
+                  gv_mma_h(acc, va[1][2], vb[1][2], va[1][3], vb[1][3], f[n][6], f[n][7]);
+                  // alpha (2^e acc - 1024 P 2^e) + beta R 2^e for tokens 2tg (sg[n][0]) and 2tg+1 (sg[n][1])
+                  y[j][n][mt][0] = fmaf(a0[mt], fmaf(acc[0], sg[n][0].z, -sg[n][0].x), fmaf(b0[mt], sg[n][0].y, y[j][n][mt][0]));
+                  y[j][n][mt][1] = fmaf(a0[mt], fmaf(acc[1], sg[n][1].z, -sg[n][1].x), fmaf(b0[mt], sg[n][1].y, y[j][n][mt][1]));
+                  y[j][n][mt][2] = fmaf(a1[mt], fmaf(acc[2], sg[n][0].z, -sg[n][0].x), fmaf(b1[mt], sg[n][0].y, y[j][n][mt][2]));
+                  y[j][n][mt][3] = fmaf(a1[mt], fmaf(acc[3], sg[n][1].z, -sg[n][1].x), fmaf(b1[mt], sg[n][1].y, y[j][n][mt][3]));
+                }
+              }
+            }
+            __syncwarp();
+            if (lane == 0) gv_release(empty(s), y[j][0][0][0], y[j][0][0][2], y[j][0][1][0], y[j][0][1][2]);
+          }
+          if (++s == STAGES) { s = 0; ph ^= 1u; }
+        }
+        // The fragment buffer is released only here, after the K tile's row blocks: releasing it right
+        // after the loads into registers (even with the release made to depend on the loaded values)
+        // produced rare wrong sums for the second token tile under stress.
+        __syncwarp();
+        if (ok && lane == 0) gv_release_u(xempty(xb), f[0][7], f[NT - 1][7], sg[0][1].w, sg[NT - 1][1].w);
+      }
+      // ---- end of the pass: the RB row blocks are summed over the warps one after the other
+#pragma unroll
+      for (int j = 0; j < RB; ++j) {
+        const int rb = (pass * RB + j) * gridDim.x + blockIdx.x;
+        if (rb >= p.n_rb) break;
+        if (ok && !gv_wait(red_free, rph ^ 1u, p.status)) ok = false;
+        float* my_red = red + warp * GT_ROWS * NTOK;
+#pragma unroll
+        for (int n = 0; n < NT; ++n)
+#pragma unroll
+          for (int mt = 0; mt < 2; ++mt) {
+            float* r0 = my_red + (mt * 16 + g) * NTOK + n * 8 + 2 * tg;
+            *reinterpret_cast<float2*>(r0) = make_float2(y[j][n][mt][0], y[j][n][mt][1]);
+            *reinterpret_cast<float2*>(r0 + 8 * NTOK) = make_float2(y[j][n][mt][2], y[j][n][mt][3]);
+          }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(red_done);
+        const int t = (warp - (int)(rcount & 15u)) & 15;    // the token this warp sums (if it exists)
+        if (t < p.T) {
+          if (ok && !gv_wait(red_done, rph, p.status)) ok = false;
+          float a = 0.0f;
+#pragma unroll
+          for (int ww = 0; ww < GT_WARPS; ++ww) a += red[(ww * GT_ROWS + lane) * NTOK + t];
+          __syncwarp();
+          if (lane == 0) gv_release(red_free, a, a, a, a);
+          const int o = rb * GT_ROWS + lane;                // lane = row of the block
+          if (o < p.d_out) {
+            if (p.y_dtype == QBLORA_BF16) reinterpret_cast<__nv_bfloat16*>(p.Y)[(int64_t)t * p.d_out + o] = __float2bfloat16_rn(a);
+            else reinterpret_cast<float*>(p.Y)[(int64_t)t * p.d_out + o] = a;
+          }
+        }
+        ++rcount;
+        rph ^= 1u;
+      }
+    }
+  }
+  __syncthreads();
+}
+
+template <int NT>
+int ko_stages() {
+  const int n = (int)((GT_SMEM_MAX - KoCfg<NT>::FIXED) / GT_STAGE_BYTES);
+  return n < 10 ? n : 10;
+}
+template <int NT>
+int ko_launch(const CUtensorMap& tm_c, const CUtensorMap& tm_a, const CUtensorMap& tm_b, GtParams p, int grid,
+              uint8_t* xfrag, cudaStream_t st) {
+  p.stages = ko_stages<NT>();
+  const int items = p.n_kc * GT_GROUPS * KoCfg<NT>::NTOK * 4;
+  x_prepare_kernel<NT><<<(items + 255) / 256, 256, 0, st>>>(p.X, p.T, p.d_in, p.G, p.n_kc, xfrag);
+  count_launch();
+  const size_t smem = KoCfg<NT>::FIXED + (size_t)p.stages * GT_STAGE_BYTES;
+  QB_CUDA(cudaFuncSetAttribute(lowbit_gemv_ko_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  lowbit_gemv_ko_kernel<NT><<<grid, GT_THREADS, smem, st>>>(tm_c, tm_a, tm_b, p, xfrag);
+  return QBLORA_OK;
+}
+
 }  // namespace
 
 bool gemv_supported(const QwView& qw, int64_t T) {
@@ -588,8 +896,15 @@ bool gemv_supported(const QwView& qw, int64_t T) {
   return qw.block_in == 64 && qw.block_out == 1 && qw.qfmt == QBLORA_FMT_AFFINE_MINMAX && T <= 16 && qw.G % 4 == 0 && qw.G <= 1024;
 }
 
+size_t gemv_ws_bytes(const QwView& qw, int64_t T) {
+  if (T <= 1) return kStatusBytes;
+  const size_t n_kc = (size_t)(qw.G + GT_GROUPS - 1) / GT_GROUPS;
+  return kStatusBytes + n_kc * (T <= 8 ? (size_t)KoCfg<1>::KT_BYTES : (size_t)KoCfg<2>::KT_BYTES);
+}
+
 int launch_lowbit_gemv(const QwView& qw, const __nv_bfloat16* X, int64_t T, void* Y, int y_dtype, int* status,
                        cudaStream_t st) {
+  uint8_t* xfrag = reinterpret_cast<uint8_t*>(status) + kStatusBytes;   // T > 1: fragments of x (see gemv_ws_bytes)
   const int NT = T <= 8 ? 1 : 2;
   GtParams p{};
   p.d_in = qw.d_in; p.d_out = qw.d_out; p.G = qw.G; p.T = (int)T;
@@ -615,7 +930,10 @@ int launch_lowbit_gemv(const QwView& qw, const __nv_bfloat16* X, int64_t T, void
   {
     DominantKernelTimer timer(st);
     count_launch();
+    static const bool ko_off = [] { const char* e = getenv("QBLORA_GEMV_KOUTER"); return e && e[0] == '0'; }();
     if (xs && T == 1) rc = gt_launch<1, 2>(tm_c, tm_a, tm_b, p, grid, st);
+    else if (!ko_off && NT == 1) rc = ko_launch<1>(tm_c, tm_a, tm_b, p, grid, xfrag, st);
+    else if (!ko_off) rc = ko_launch<2>(tm_c, tm_a, tm_b, p, grid, xfrag, st);
     else if (xs) rc = gt_launch<1, 1>(tm_c, tm_a, tm_b, p, grid, st);
     else if (NT == 1) rc = gt_launch<1, 0>(tm_c, tm_a, tm_b, p, grid, st);
     else rc = gt_launch<2, 0>(tm_c, tm_a, tm_b, p, grid, st);
