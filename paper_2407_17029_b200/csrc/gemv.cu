@@ -6,22 +6,24 @@
 // quantization groups (16 KB of codes as four 128-byte-swizzled TMA boxes, plus the 32 x 16 alpha
 // and beta values) through a shared-memory ring guarded by mbarriers, so no compute warp ever waits
 // on DRAM latency or does global address arithmetic for the weight.  Each of the sixteen compute
-// warps owns one of the tile's 16 groups and all 32 rows (two MMA row tiles), so the token operand
-// of a group is fetched once per warp and tile.  Partial sums stay in registers across the K tiles
-// of a row block and are summed through shared memory in warp order at the end of the block
+// warps owns one of the tile's 16 groups and all 32 rows (two MMA row tiles).  Partial sums stay in
+// registers across the K tiles and are summed through shared memory in warp order at the end
 // (deterministic).
 //
-// Arithmetic.  The work of a warp is shaped for mma.sync.m16n8k16 (bf16, fp32 accumulate): 16 rows
-// are the M side, up to 8 tokens per N tile.  A thread (g = lane / 4, tg = lane % 4) reads, for rows
-// g + 8 q (q = 0..3), the 8 bytes holding codes 16 tg .. 16 tg + 15 of the group and turns each
-// 32-bit word into four bf16 pairs (128 + c) with one logic op per pair (the nibbles land in the
-// mantissa of 128.0).  Because the order of the k index inside an MMA is free as long as both
-// operands agree, nibble pairs (e, e + 4) are used as they fall out of the word and the token operand
-// is permuted to match with byte permutes.  With S = sum of x over the group (computed once per CTA
-// into shared memory), the group contributes
-//   alpha * sum((128 + c) x) + (beta - 128 alpha) * S  =  alpha * sum(c x) + beta * S.
-// When T * D_in is small enough the permuted token fragments are also kept in shared memory for the
-// life of the CTA; otherwise they are rebuilt per group from global x (L1-resident).
+// Arithmetic.  The work of a warp is shaped for mma.sync.m16n8k16 (fp16 operands, fp32 accumulate):
+// 16 rows are the M side, up to 8 tokens per N tile.  A thread (g = lane / 4, tg = lane % 4) reads,
+// for rows g + 8 q (q = 0..3), the 8 bytes holding codes 16 tg .. 16 tg + 15 of the group and turns
+// each 32-bit word into four fp16 pairs with one three-input logic op per pair: the nibbles are OR-ed
+// into the mantissa of 1024.0, and because fp16's mantissa holds two neighbouring nibbles a word
+// needs one shift only; odd nibbles come out as 1024 + 16 c and the token operand carries 1/16 at
+// those positions.  The order of the k index inside an MMA is free as long as both operands agree,
+// so nibble pairs (e, e + 4) are used as they fall out of the word and the token fragments are laid
+// out to match.  x (bf16) is converted to fp16 after a power-of-two prescale 2^-e (per call for one
+// token, per 64-value slice otherwise).  With P = sum of the fragment values and R = sum of the
+// scaled x over a group, the group contributes  2^e (alpha (acc - 1024 P) + beta R).
+//
+// Two kernels: one token (fragments of x resident in shared memory, row blocks outer) and 2..16
+// tokens (K tiles outer, fragments prepared once in the workspace and streamed per K tile).
 #include <cstdlib>
 #include "tc_ptx.cuh"
 #include "tc_small.cuh"
@@ -38,26 +40,6 @@ constexpr int GT_CODE_BYTES = GT_ROWS * GT_GROUPS * 32;   // 16 KB = four boxes 
 constexpr int GT_SCALE_BYTES = GT_ROWS * GT_GROUPS * 4;   // 2 KB each for alpha and beta
 constexpr int GT_STAGE_BYTES = GT_CODE_BYTES + 2 * GT_SCALE_BYTES;
 
-__device__ __forceinline__ uint32_t gv_prmt(uint32_t a, uint32_t b, uint32_t sel) {
-  uint32_t r;
-  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
-  return r;
-}
-__device__ __forceinline__ void gv_mma(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                       uint32_t b1) {
-  asm(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-// first MMA of a chain: accumulator input is zero
-__device__ __forceinline__ void gv_mma0(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                        uint32_t b1) {
-  asm(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
-      : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.0f));
-}
 // (w & m) | c as ONE three-input logic op.  Mask and magic are passed in registers: written with two
 // literals the compiler emits two logic ops (one literal each), which costs a third of the kernel.
 __device__ __forceinline__ uint32_t gv_and_or(uint32_t w, uint32_t m, uint32_t c) {
@@ -72,33 +54,6 @@ struct GvConst {
     asm volatile("" : "+r"(m0), "+r"(m1), "+r"(c));
   }
 };
-// word of 8 codes -> (128 + c) bf16 pairs: v[e] = (code e, code e + 4), e = 0..3
-// (k.m0 = 0x000F000F, k.c = 0x43004300)
-__device__ __forceinline__ void gv_unpack(uint32_t w, uint32_t (&v)[4], const GvConst& k) {
-  v[0] = gv_and_or(w, k.m0, k.c);
-  v[1] = gv_and_or(w >> 4, k.m0, k.c);
-  v[2] = gv_and_or(w >> 8, k.m0, k.c);
-  v[3] = gv_and_or(w >> 12, k.m0, k.c);
-}
-// 16 consecutive x values (two 16-byte words) -> the eight B registers of the four MMAs of a thread:
-// f[2 (2 wd + h)] / f[2 (2 wd + h) + 1] pair x at positions (2h, 2h+4) / (2h+1, 2h+5) of word wd
-__device__ __forceinline__ void gv_permute_x(const uint4& x0, const uint4& x1, uint32_t (&f)[8]) {
-  const uint32_t xr[2][4] = {{x0.x, x0.y, x0.z, x0.w}, {x1.x, x1.y, x1.z, x1.w}};
-#pragma unroll
-  for (int wd = 0; wd < 2; ++wd)
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      f[2 * (2 * wd + h)] = gv_prmt(xr[wd][h], xr[wd][h + 2], 0x5410u);
-      f[2 * (2 * wd + h) + 1] = gv_prmt(xr[wd][h], xr[wd][h + 2], 0x7632u);
-    }
-}
-__device__ __forceinline__ float gv_sum16(const uint4& x0, const uint4& x1) {
-  const uint32_t w[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
-  float a = 0.0f;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) a += __uint_as_float(w[i] << 16) + __uint_as_float(w[i] & 0xFFFF0000u);
-  return a;
-}
 // ---- fp16 variants (shared-memory token operand only) --------------------------------------------
 // With a 10-bit mantissa two neighbouring nibbles fit below the magic exponent, so a word needs one
 // shift instead of three: v[0], v[2] = 1024 + c for codes (0,4), (2,6); v[1], v[3] = 1024 + 16 c for
@@ -218,53 +173,43 @@ struct GtParams {
   int* status;
 };
 
-// MODE 0: token fragments rebuilt per group from global x (bf16 MMA), any T <= 8 NT.
-// MODE 1: x converted once per CTA to fp16 fragments in shared memory (T <= 8, small T x D_in).
-// MODE 2: MODE 1 specialised for a single token (only accumulator column 0 is kept).
-template <int NT, int MODE>
-struct GtCfg {
-  static constexpr int RED_TOKENS = MODE == 2 ? 1 : NT * 8;                     // tokens kept per row in the reduction
-  static constexpr int RED_BYTES = GT_WARPS * GT_ROWS * RED_TOKENS * 4;
-  static constexpr int SS_PER_GROUP = MODE == 0 ? NT * 8 : (MODE == 1 ? 16 : 2);  // floats: S, or (P, R), per token
-  static constexpr int MAX_STAGES = 10;
-};
+// ---------------------------------------------------------------------------------------------------
+// One token.  x is converted once per CTA into fp16 fragments in shared memory (with ONE power-of-two
+// prescale 2^-e for the call, undone on the output), the row blocks are the outer loop and only
+// column 0 of the accumulator tile is kept.
+constexpr int T1_RED_BYTES = GT_WARPS * GT_ROWS * 4;        // [16 warps][32 rows]
+constexpr int T1_MAX_STAGES = 10;
 
-template <int NT, int MODE>   // NT = number of 8-token tiles (1 or 2)
 __global__ void __launch_bounds__(GT_THREADS, 1)
-lowbit_gemv_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_constant__ CUtensorMap tm_a,
-                   const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ GtParams p) {
-  static_assert(MODE == 0 || NT == 1, "shared-memory token operand: one token tile");
+lowbit_gemv_t1_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_constant__ CUtensorMap tm_a,
+                      const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ GtParams p) {
   const int STAGES = p.stages;
-  constexpr int NTOK = NT * 8;
-  constexpr int RT = GtCfg<NT, MODE>::RED_TOKENS;
-  constexpr int SSG = GtCfg<NT, MODE>::SS_PER_GROUP;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* gbase = smem_raw + (base - raw);
   const uint32_t red_off = STAGES * GT_STAGE_BYTES;
-  float* red = reinterpret_cast<float*>(gbase + red_off);                 // [16 warps][32 rows][RT]
-  const uint32_t bar_off = red_off + GtCfg<NT, MODE>::RED_BYTES;
+  float* red = reinterpret_cast<float*>(gbase + red_off);                 // [16 warps][32 rows]
+  const uint32_t bar_off = red_off + T1_RED_BYTES;
   const uint32_t bars = base + bar_off;
   auto full = [&](int s) { return bars + 8u * s; };
   auto empty = [&](int s) { return bars + 8u * (STAGES + s); };
   const uint32_t red_done = bars + 8u * (2 * STAGES);       // all 16 warps have written their sums of the row block
-  const uint32_t red_free = bars + 8u * (2 * STAGES + 1);   // the summing warps have read them
-  // MODE 0: ss[G][NTOK] = S (sum of x over the group), 0 beyond T.
-  // MODE 1/2: ss[G][8][2] = (1024 * sum of the fp16 fragment values, sum of the scaled x), then
-  //           xs[G][T][4 tg][8 words] = fp16 fragments
-  float* ss = reinterpret_cast<float*>(gbase + bar_off + 256);
+  const uint32_t red_free = bars + 8u * (2 * STAGES + 1);   // the summing warp has read them
+  // ss[G] = (1024 * sum of the fp16 fragment values, sum of the scaled x) per group, then
+  // xs[G][4 tg][8 words] = fp16 fragments, then 128 zero bytes
   const uint32_t ss_off = bar_off + 256;
-  const uint32_t xs_off = ss_off + (uint32_t)p.G * SSG * 4;
+  float* ss = reinterpret_cast<float*>(gbase + ss_off);
+  const uint32_t xs_off = ss_off + (uint32_t)p.G * 8;
   uint4* xs = reinterpret_cast<uint4*>(gbase + xs_off);
-  const uint32_t zero_off = xs_off + (MODE != 0 ? (uint32_t)p.G * p.T * 128 : 0u);   // 128 zero bytes (MODE 1/2)
+  const uint32_t zero_off = xs_off + (uint32_t)p.G * 128;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
     if (blockIdx.x == 0) *p.status = 0;   // any give-up below is written at least a wait limit later
     for (int s = 0; s < STAGES; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), GT_WARPS); }
     mbar_init(red_done, GT_WARPS);
-    mbar_init(red_free, p.T);
+    mbar_init(red_free, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -296,112 +241,68 @@ lowbit_gemv_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_consta
   } else {
     // ------------------------------------------------------------------ compute warps
     const int g = lane >> 2, tg = lane & 3;
-    // ---- once per CTA, while the first tiles are in flight: group sums of x and (MODE 1/2) fragments.
-    // Item = (group, token, tg): 16 values of x; the four tg lanes of an item are neighbours.
-    float y_scale = 1.0f;
-    const int items = p.G * p.T * 4;
+    // ---- once per CTA, while the first tiles are in flight: fragments and group sums of x.
+    // Item = (group, tg): 16 values of x; the four tg lanes of an item are neighbours.
+    const int items = p.G * 4;
     const bool one_round = items <= GT_WARPS * 32;
     uint4 c0, c1;     // this thread's item of the first round (x is read from global once when one round covers it)
     {
       const int q = tid < items ? tid : 0;
-      const int t = (q >> 2) % p.T, grp = (q >> 2) / p.T;
-      const uint4* src = reinterpret_cast<const uint4*>(p.X + (int64_t)t * p.d_in + grp * 64 + (q & 3) * 16);
+      const uint4* src = reinterpret_cast<const uint4*>(p.X + q * 16);
       c0 = __ldg(src); c1 = __ldg(src + 1);
     }
-    if (MODE == 0) {
-      for (int i = tid; i < p.G * NTOK; i += GT_WARPS * 32)
-        if ((i % NTOK) >= p.T) ss[i] = 0.0f;
+    float am = 0.0f;
+    if (one_round) {
+      am = gv_absmax8(c1, gv_absmax8(c0, am));
     } else {
-      // fp16 range: one power-of-two prescale for the call brings max |x| just below 2^15 (up or down)
-      float am = 0.0f;
-      if (one_round) {
-        am = gv_absmax8(c1, gv_absmax8(c0, am));
-      } else {
-        const uint4* xv = reinterpret_cast<const uint4*>(p.X);
-        for (int i = tid; i < p.T * (p.d_in >> 3); i += GT_WARPS * 32) am = gv_absmax8(__ldg(xv + i), am);
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) am = fmaxf(am, __shfl_xor_sync(0xFFFFFFFFu, am, o));
-      if (lane == 0) red[warp] = am;
-      if (MODE == 1)
-        for (int i = tid; i < p.G * 16; i += GT_WARPS * 32)
-          if (((i >> 1) & 7) >= p.T) ss[i] = 0.0f;
-      asm volatile("bar.sync 1, 512;" ::: "memory");
-      am = red[0];
-#pragma unroll
-      for (int i = 1; i < GT_WARPS; ++i) am = fmaxf(am, red[i]);
-      int e = (int)((__float_as_uint(am) >> 23) & 0xFFu) - 127 - 14;   // max |x| * 2^-e in [2^14, 2^15)
-      e = e < -100 ? -100 : (e > 120 ? 120 : e);
-      y_scale = __uint_as_float((uint32_t)(127 + e) << 23);
-      asm volatile("bar.sync 1, 512;" ::: "memory");   // red is free again
-      if (tid < 32) reinterpret_cast<uint32_t*>(gbase + zero_off)[tid] = 0u;
+      const uint4* xv = reinterpret_cast<const uint4*>(p.X);
+      for (int i = tid; i < (p.d_in >> 3); i += GT_WARPS * 32) am = gv_absmax8(__ldg(xv + i), am);
     }
-    if (MODE == 0) {
-      // group sums only; eight rounds of loads are in flight at a time (the rounds are L2 round trips).
-      // All CTAs walk x in the same order: starting each at its own offset measured slower.
-      constexpr int DEPTH = 8;
-      for (int i0 = 0; i0 < items; i0 += DEPTH * GT_WARPS * 32) {
-        uint4 xa[DEPTH], xb[DEPTH];
 #pragma unroll
-        for (int u = 0; u < DEPTH; ++u) {
-          const int idx = i0 + u * GT_WARPS * 32 + tid;
-          const int q = idx < items ? idx : 0;
-          const int t = (q >> 2) % p.T, grp = (q >> 2) / p.T;
-          const uint4* src = reinterpret_cast<const uint4*>(p.X + (int64_t)t * p.d_in + grp * 64 + (q & 3) * 16);
-          xa[u] = __ldg(src); xb[u] = __ldg(src + 1);
-        }
+    for (int o = 16; o > 0; o >>= 1) am = fmaxf(am, __shfl_xor_sync(0xFFFFFFFFu, am, o));
+    if (lane == 0) red[warp] = am;
+    asm volatile("bar.sync 1, 512;" ::: "memory");
+    am = red[0];
 #pragma unroll
-        for (int u = 0; u < DEPTH; ++u) {
-          const int idx = i0 + u * GT_WARPS * 32 + tid;
-          const bool live = idx < items;
-          const int q = live ? idx : 0;
-          const int t = (q >> 2) % p.T, grp = (q >> 2) / p.T;
-          float sum = gv_sum16(xa[u], xb[u]);
-          sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 1);
-          sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 2);
-          if (live && (q & 3) == 0) ss[grp * NTOK + t] = sum;
-        }
-      }
-    } else {
-      const float in_scale = 1.0f / y_scale, in_scale16 = in_scale * 0.0625f;
+    for (int i = 1; i < GT_WARPS; ++i) am = fmaxf(am, red[i]);
+    int e = (int)((__float_as_uint(am) >> 23) & 0xFFu) - 127 - 14;   // max |x| * 2^-e in [2^14, 2^15)
+    e = e < -100 ? -100 : (e > 120 ? 120 : e);
+    const float y_scale = __uint_as_float((uint32_t)(127 + e) << 23);
+    asm volatile("bar.sync 1, 512;" ::: "memory");   // red is free again
+    if (tid < 32) reinterpret_cast<uint32_t*>(gbase + zero_off)[tid] = 0u;
+    {
+      const float in_scale = __uint_as_float((uint32_t)(127 - e) << 23), in_scale16 = in_scale * 0.0625f;
       for (int i0 = 0; i0 < items; i0 += GT_WARPS * 32) {
         const int idx = i0 + tid;
         const bool live = idx < items;
         const int q = live ? idx : 0;
-        const int t = (q >> 2) % p.T, grp = (q >> 2) / p.T;
-        const uint4* src = reinterpret_cast<const uint4*>(p.X + (int64_t)t * p.d_in + grp * 64 + (q & 3) * 16);
+        const uint4* src = reinterpret_cast<const uint4*>(p.X + q * 16);
         const uint4 x0 = i0 == 0 ? c0 : __ldg(src), x1 = i0 == 0 ? c1 : __ldg(src + 1);
-        if (MODE == 0) {
-          float sum = gv_sum16(x0, x1);
-          sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 1);
-          sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 2);
-          if (live && (q & 3) == 0) ss[grp * NTOK + t] = sum;
-        } else {
-          const uint32_t xw[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
-          uint32_t f[8];
-          float ps = 0.0f, rs = 0.0f;   // sum of fragment values; sum of scaled x as the fragments hold it
+        const uint32_t xw[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+        uint32_t f[8];
+        float ps = 0.0f, rs = 0.0f;   // sum of fragment values; sum of scaled x as the fragments hold it
 #pragma unroll
-          for (int wd = 0; wd < 2; ++wd)
+        for (int wd = 0; wd < 2; ++wd)
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-              // word wd holds x at positions 0..7 as pairs (2j, 2j+1) in xw[4 wd + j]
-              const uint32_t wa = xw[4 * wd + h], wb = xw[4 * wd + h + 2];
-              const uint32_t ev = gv_pack_h2(__uint_as_float(wa << 16) * in_scale, __uint_as_float(wb << 16) * in_scale);
-              const uint32_t od = gv_pack_h2(__uint_as_float(wa & 0xFFFF0000u) * in_scale16,
-                                             __uint_as_float(wb & 0xFFFF0000u) * in_scale16);
-              f[2 * (2 * wd + h)] = ev;
-              f[2 * (2 * wd + h) + 1] = od;
-              const float se = gv_h_lo(ev) + gv_h_hi(ev), so = gv_h_lo(od) + gv_h_hi(od);
-              ps += se + so;
-              rs += se + 16.0f * so;
-            }
-          ps += __shfl_xor_sync(0xFFFFFFFFu, ps, 1); rs += __shfl_xor_sync(0xFFFFFFFFu, rs, 1);
-          ps += __shfl_xor_sync(0xFFFFFFFFu, ps, 2); rs += __shfl_xor_sync(0xFFFFFFFFu, rs, 2);
-          if (live) {
-            if ((q & 3) == 0) *reinterpret_cast<float2*>(ss + grp * SSG + t * 2) = make_float2(1024.0f * ps, rs);
-            xs[q * 2] = make_uint4(f[0], f[1], f[2], f[3]);
-            xs[q * 2 + 1] = make_uint4(f[4], f[5], f[6], f[7]);
+          for (int h = 0; h < 2; ++h) {
+            // word wd holds x at positions 0..7 as pairs (2j, 2j+1) in xw[4 wd + j]; fragment register
+            // 2 (2 wd + h) pairs positions (2h, 2h+4), the next one (2h+1, 2h+5) scaled by 1/16
+            const uint32_t wa = xw[4 * wd + h], wb = xw[4 * wd + h + 2];
+            const uint32_t ev = gv_pack_h2(__uint_as_float(wa << 16) * in_scale, __uint_as_float(wb << 16) * in_scale);
+            const uint32_t od = gv_pack_h2(__uint_as_float(wa & 0xFFFF0000u) * in_scale16,
+                                           __uint_as_float(wb & 0xFFFF0000u) * in_scale16);
+            f[2 * (2 * wd + h)] = ev;
+            f[2 * (2 * wd + h) + 1] = od;
+            const float se = gv_h_lo(ev) + gv_h_hi(ev), so = gv_h_lo(od) + gv_h_hi(od);
+            ps += se + so;
+            rs += se + 16.0f * so;
           }
+        ps += __shfl_xor_sync(0xFFFFFFFFu, ps, 1); rs += __shfl_xor_sync(0xFFFFFFFFu, rs, 1);
+        ps += __shfl_xor_sync(0xFFFFFFFFu, ps, 2); rs += __shfl_xor_sync(0xFFFFFFFFu, rs, 2);
+        if (live) {
+          if ((q & 3) == 0) *reinterpret_cast<float2*>(ss + (q >> 2) * 2) = make_float2(1024.0f * ps, rs);
+          xs[q * 2] = make_uint4(f[0], f[1], f[2], f[3]);
+          xs[q * 2 + 1] = make_uint4(f[4], f[5], f[6], f[7]);
         }
       }
     }
@@ -416,30 +317,19 @@ lowbit_gemv_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_consta
     // xor (row / 2) % 4), which spreads the eight rows a warp reads at once over eight banks
     const uint32_t scale_off = GT_CODE_BYTES + (uint32_t)g * 64u +
                                ((((uint32_t)warp >> 2) ^ (((uint32_t)g >> 1) & 3u)) << 4) + ((uint32_t)warp & 3u) * 4u;
-    const uint4* xrow[NT];
-    bool xlive[NT];
-#pragma unroll
-    for (int j = 0; j < NT; ++j) {
-      const int t = j * 8 + g;
-      xlive[j] = t < p.T;
-      xrow[j] = reinterpret_cast<const uint4*>(p.X + (int64_t)(xlive[j] ? t : 0) * p.d_in) + tg * 2;
-    }
-    // MODE 1/2: lanes whose token does not exist read the zero block (stride 0) instead of selecting zeros
-    const uint32_t xs_addr = base + (xlive[0] ? xs_off + (uint32_t)(g * 4 + tg) * 32u : zero_off + (uint32_t)tg * 32u);
-    const uint32_t xs_stride = xlive[0] ? (uint32_t)p.T * 128u : 0u;
-    const uint32_t ss_addr = base + ss_off + (MODE == 0 ? 8u * tg : (MODE == 1 ? 16u * tg : 0u));
+    // B fragment column = token: only the lanes with g == 0 hold the token, the others read the zero
+    // block (stride 0) instead of selecting zeros
+    const uint32_t xs_addr = base + (g == 0 ? xs_off : zero_off) + (uint32_t)tg * 32u;
+    const uint32_t xs_stride = g == 0 ? 128u : 0u;
+    const uint32_t ss_addr = base + ss_off;
     uint32_t rph = 0, rcount = 0;   // phase of the reduction barriers; row blocks done
-    const GvConst kc_(0x000F000Fu, 0x00F000F0u, MODE == 0 ? 0x43004300u : 0x64006400u);
+    const GvConst kc_(0x000F000Fu, 0x00F000F0u, 0x64006400u);
     bool ok = true;        // after a timed-out wait the warp keeps walking its loops (so the CTA
                            // barriers still match) but no longer waits or computes
     int s = 0;
     uint32_t ph = 0;
     for (int rb = blockIdx.x; rb < p.n_rb; rb += gridDim.x) {
-      float y[NT][2][4];
-#pragma unroll
-      for (int j = 0; j < NT; ++j)
-#pragma unroll
-        for (int mt = 0; mt < 2; ++mt) { y[j][mt][0] = y[j][mt][1] = y[j][mt][2] = y[j][mt][3] = 0.0f; }
+      float y[2][2] = {{0.0f, 0.0f}, {0.0f, 0.0f}};    // [row tile][row g, row g + 8], token 0 (lanes tg == 0)
       for (int kc = 0; kc < p.n_kc; ++kc) {
         if (ok && !gv_wait(full(s), ph, p.status)) ok = false;
         const int grp = kc * GT_GROUPS + warp;
@@ -447,25 +337,9 @@ lowbit_gemv_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_consta
           if (grp < p.G) {                                   // warp-uniform
             const uint32_t sb = base + (uint32_t)s * GT_STAGE_BYTES;
             const uint32_t ca = sb + code_off, sa = sb + scale_off;
-            uint32_t f[NT][8];
-            float4 sg[NT];   // MODE 0: (S[2tg], S[2tg+1], -, -); MODE 1: (P, R)[2tg], (P, R)[2tg+1]; MODE 2: (P, R)[0]
-            if (MODE == 0) {
-#pragma unroll
-              for (int j = 0; j < NT; ++j) {
-                const float2 v = j == 0 ? gv_ldsf2<0>(ss_addr + (uint32_t)grp * (NTOK * 4)) : gv_ldsf2<32>(ss_addr + (uint32_t)grp * (NTOK * 4));
-                sg[j] = make_float4(v.x, v.y, 0.0f, 0.0f);
-                uint4 x0 = make_uint4(0, 0, 0, 0), x1 = make_uint4(0, 0, 0, 0);
-                if (xlive[j]) { x0 = __ldg(xrow[j] + grp * 8); x1 = __ldg(xrow[j] + grp * 8 + 1); }
-                gv_permute_x(x0, x1, f[j]);
-              }
-            } else {
-              if (MODE == 1) sg[0] = gv_ldsf4<0>(ss_addr + (uint32_t)grp * 64u);
-              else { const float2 v = gv_ldsf2<0>(ss_addr + (uint32_t)grp * 8u); sg[0] = make_float4(v.x, v.y, 0.0f, 0.0f); }
-              const uint32_t xa = xs_addr + (uint32_t)grp * xs_stride;
-              const uint4 x0 = gv_lds4<0>(xa), x1 = gv_lds4<16>(xa);
-              f[0][0] = x0.x; f[0][1] = x0.y; f[0][2] = x0.z; f[0][3] = x0.w;
-              f[0][4] = x1.x; f[0][5] = x1.y; f[0][6] = x1.z; f[0][7] = x1.w;
-            }
+            const float2 sg = gv_ldsf2<0>(ss_addr + (uint32_t)grp * 8u);      // (1024 P, R) of the group
+            const uint32_t xa = xs_addr + (uint32_t)grp * xs_stride;
+            const uint4 x0 = gv_lds4<0>(xa), x1 = gv_lds4<16>(xa);
             // all shared-memory loads of the group first (they stay in program order), then the math
             uint2 w0[2], w1[2];
             float a0[2], a1[2], b0[2], b1[2];
@@ -476,87 +350,47 @@ lowbit_gemv_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_consta
 #pragma unroll
             for (int mt = 0; mt < 2; ++mt) {
               uint32_t va[2][4], vb[2][4];      // [word][pair] for rows g + 16 mt (va) and g + 16 mt + 8 (vb)
-              if (MODE == 0) {
-                gv_unpack(w0[mt].x, va[0], kc_); gv_unpack(w0[mt].y, va[1], kc_);
-                gv_unpack(w1[mt].x, vb[0], kc_); gv_unpack(w1[mt].y, vb[1], kc_);
-                const float s0 = fmaf(-128.0f, a0[mt], b0[mt]), s1 = fmaf(-128.0f, a1[mt], b1[mt]);
-#pragma unroll
-                for (int j = 0; j < NT; ++j) {
-                  float acc[4];
-                  gv_mma0(acc, va[0][0], vb[0][0], va[0][1], vb[0][1], f[j][0], f[j][1]);
-                  gv_mma(acc, va[0][2], vb[0][2], va[0][3], vb[0][3], f[j][2], f[j][3]);
-                  gv_mma(acc, va[1][0], vb[1][0], va[1][1], vb[1][1], f[j][4], f[j][5]);
-                  gv_mma(acc, va[1][2], vb[1][2], va[1][3], vb[1][3], f[j][6], f[j][7]);
-                  y[j][mt][0] = fmaf(a0[mt], acc[0], fmaf(s0, sg[j].x, y[j][mt][0]));
-                  y[j][mt][1] = fmaf(a0[mt], acc[1], fmaf(s0, sg[j].y, y[j][mt][1]));
-                  y[j][mt][2] = fmaf(a1[mt], acc[2], fmaf(s1, sg[j].x, y[j][mt][2]));
-                  y[j][mt][3] = fmaf(a1[mt], acc[3], fmaf(s1, sg[j].y, y[j][mt][3]));
-                }
-              } else {
-                gv_unpack_h(w0[mt].x, va[0], kc_); gv_unpack_h(w0[mt].y, va[1], kc_);
-                gv_unpack_h(w1[mt].x, vb[0], kc_); gv_unpack_h(w1[mt].y, vb[1], kc_);
-                float acc[4];
-                gv_mma0_h(acc, va[0][0], vb[0][0], va[0][1], vb[0][1], f[0][0], f[0][1]);
-                gv_mma_h(acc, va[0][2], vb[0][2], va[0][3], vb[0][3], f[0][2], f[0][3]);
-                gv_mma_h(acc, va[1][0], vb[1][0], va[1][1], vb[1][1], f[0][4], f[0][5]);
-                gv_mma_h(acc, va[1][2], vb[1][2], va[1][3], vb[1][3], f[0][6], f[0][7]);
-                // alpha (acc - 1024 P) + beta R
-                if (MODE == 1) {
-                  y[0][mt][0] = fmaf(a0[mt], acc[0] - sg[0].x, fmaf(b0[mt], sg[0].y, y[0][mt][0]));
-                  y[0][mt][1] = fmaf(a0[mt], acc[1] - sg[0].z, fmaf(b0[mt], sg[0].w, y[0][mt][1]));
-                  y[0][mt][2] = fmaf(a1[mt], acc[2] - sg[0].x, fmaf(b1[mt], sg[0].y, y[0][mt][2]));
-                  y[0][mt][3] = fmaf(a1[mt], acc[3] - sg[0].z, fmaf(b1[mt], sg[0].w, y[0][mt][3]));
-                } else {   // single token: column 0 of the accumulator tile (held by the tg == 0 lanes)
-                  y[0][mt][0] = fmaf(a0[mt], acc[0] - sg[0].x, fmaf(b0[mt], sg[0].y, y[0][mt][0]));
-                  y[0][mt][2] = fmaf(a1[mt], acc[2] - sg[0].x, fmaf(b1[mt], sg[0].y, y[0][mt][2]));
-                }
-              }
+              gv_unpack_h(w0[mt].x, va[0], kc_); gv_unpack_h(w0[mt].y, va[1], kc_);
+              gv_unpack_h(w1[mt].x, vb[0], kc_); gv_unpack_h(w1[mt].y, vb[1], kc_);
+              float acc[4];
+              gv_mma0_h(acc, va[0][0], vb[0][0], va[0][1], vb[0][1], x0.x, x0.y);
+              gv_mma_h(acc, va[0][2], vb[0][2], va[0][3], vb[0][3], x0.z, x0.w);
+              gv_mma_h(acc, va[1][0], vb[1][0], va[1][1], vb[1][1], x1.x, x1.y);
+              gv_mma_h(acc, va[1][2], vb[1][2], va[1][3], vb[1][3], x1.z, x1.w);
+              // alpha (acc - 1024 P) + beta R; column 0 of the accumulator tile is held by the tg == 0 lanes
+              y[mt][0] = fmaf(a0[mt], acc[0] - sg.x, fmaf(b0[mt], sg.y, y[mt][0]));
+              y[mt][1] = fmaf(a1[mt], acc[2] - sg.x, fmaf(b1[mt], sg.y, y[mt][1]));
             }
           }
           __syncwarp();
-          if (lane == 0) gv_release(empty(s), y[0][0][0], y[0][0][2], y[0][1][0], y[0][1][2]);   // this warp is done reading the stage
+          if (lane == 0) gv_release(empty(s), y[0][0], y[0][1], y[1][0], y[1][1]);   // this warp is done reading the stage
         }
         if (++s == STAGES) { s = 0; ph ^= 1u; }
       }
       // End of the row block, without a CTA-wide barrier.  Every warp writes its partial sums into its
-      // slot (once the warps that summed the previous row block have let go of the buffer) and arrives
-      // on red_done; token t is then summed over the sixteen slots in slot order (deterministic) and
-      // stored by warp (t + row block count) % 16, which is the only warp that waits for the others.
-      // accumulator layout: [0],[1] = row g, tokens 2tg, 2tg+1; [2],[3] = row g + 8
+      // slot (once the warp that summed the previous row block has let go of the buffer) and arrives
+      // on red_done; the sixteen slots are then summed in slot order (deterministic) and stored by
+      // warp (row block count) % 16, which is the only warp that waits for the others.
       if (ok && !gv_wait(red_free, rph ^ 1u, p.status)) ok = false;
-      float* my_red = red + warp * GT_ROWS * RT;
-      if (MODE == 2) {
-        if (tg == 0) {
+      float* my_red = red + warp * GT_ROWS;
+      if (tg == 0) {
 #pragma unroll
-          for (int mt = 0; mt < 2; ++mt) { my_red[mt * 16 + g] = y[0][mt][0]; my_red[mt * 16 + g + 8] = y[0][mt][2]; }
-        }
-      } else {
-#pragma unroll
-        for (int j = 0; j < NT; ++j)
-#pragma unroll
-          for (int mt = 0; mt < 2; ++mt) {
-            float* r0 = my_red + (mt * 16 + g) * RT + j * 8 + 2 * tg;
-            *reinterpret_cast<float2*>(r0) = make_float2(y[j][mt][0], y[j][mt][1]);
-            *reinterpret_cast<float2*>(r0 + 8 * RT) = make_float2(y[j][mt][2], y[j][mt][3]);
-          }
+        for (int mt = 0; mt < 2; ++mt) { my_red[mt * 16 + g] = y[mt][0]; my_red[mt * 16 + g + 8] = y[mt][1]; }
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(red_done);
-      {
-        const int t = (warp - (int)(rcount & 15u)) & 15;    // the token this warp sums (if it exists)
-        if (t < p.T) {
-          if (ok && !gv_wait(red_done, rph, p.status)) ok = false;
-          float a = 0.0f;
+      if (warp == (int)(rcount & 15u)) {
+        if (ok && !gv_wait(red_done, rph, p.status)) ok = false;
+        float a = 0.0f;
 #pragma unroll
-          for (int ww = 0; ww < GT_WARPS; ++ww) a += red[(ww * GT_ROWS + lane) * RT + t];
-          __syncwarp();
-          if (lane == 0) gv_release(red_free, a, a, a, a);
-          a *= y_scale;
-          const int o = rb * GT_ROWS + lane;                // lane = row of the block
-          if (o < p.d_out) {
-            if (p.y_dtype == QBLORA_BF16) reinterpret_cast<__nv_bfloat16*>(p.Y)[(int64_t)t * p.d_out + o] = __float2bfloat16_rn(a);
-            else reinterpret_cast<float*>(p.Y)[(int64_t)t * p.d_out + o] = a;
-          }
+        for (int ww = 0; ww < GT_WARPS; ++ww) a += red[ww * GT_ROWS + lane];
+        __syncwarp();
+        if (lane == 0) gv_release(red_free, a, a, a, a);
+        a *= y_scale;
+        const int o = rb * GT_ROWS + lane;                // lane = row of the block
+        if (o < p.d_out) {
+          if (p.y_dtype == QBLORA_BF16) reinterpret_cast<__nv_bfloat16*>(p.Y)[o] = __float2bfloat16_rn(a);
+          else reinterpret_cast<float*>(p.Y)[o] = a;
         }
       }
       ++rcount;
@@ -566,36 +400,27 @@ lowbit_gemv_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_consta
   __syncthreads();
 }
 
-// dynamic shared memory besides the stage ring: alignment slack, reduction buffer, barriers, group
-// sums, (MODE 1/2) fragments and the zero block
-template <int NT, int MODE>
-size_t gt_fixed_smem(int G, int T) {
-  size_t n = 1024 + GtCfg<NT, MODE>::RED_BYTES + 256 + (size_t)G * GtCfg<NT, MODE>::SS_PER_GROUP * 4;
-  if (MODE != 0) n += (size_t)G * T * 128 + 128;
-  return n;
-}
 constexpr size_t GT_SMEM_MAX = 227 * 1024;
-template <int NT, int MODE>
-int gt_stages(int G, int T) {   // ring depth that fits; < 4 means this mode does not fit
-  const size_t fixed = gt_fixed_smem<NT, MODE>(G, T);
-  if (fixed + 4 * (size_t)GT_STAGE_BYTES > GT_SMEM_MAX) return 0;
+// dynamic shared memory besides the stage ring: alignment slack, reduction buffer, barriers, group
+// sums, fragments, zero block
+size_t t1_fixed_smem(int G) { return 1024 + T1_RED_BYTES + 256 + (size_t)G * 8 + (size_t)G * 128 + 128; }
+int t1_stages(int G) {   // ring depth that fits; 0 if fewer than six stages would be left
+  const size_t fixed = t1_fixed_smem(G);
+  if (fixed + 6 * (size_t)GT_STAGE_BYTES > GT_SMEM_MAX) return 0;
   const int n = (int)((GT_SMEM_MAX - fixed) / GT_STAGE_BYTES);
-  return n < GtCfg<NT, MODE>::MAX_STAGES ? n : GtCfg<NT, MODE>::MAX_STAGES;
+  return n < T1_MAX_STAGES ? n : T1_MAX_STAGES;
 }
-
-template <int NT, int MODE>
-int gt_launch(const CUtensorMap& tm_c, const CUtensorMap& tm_a, const CUtensorMap& tm_b, GtParams p, int grid,
+int t1_launch(const CUtensorMap& tm_c, const CUtensorMap& tm_a, const CUtensorMap& tm_b, GtParams p, int grid,
               cudaStream_t st) {
-  p.stages = gt_stages<NT, MODE>(p.G, p.T);
-  if (p.stages < 4) return QBLORA_ERR_UNSUPPORTED;
-  const size_t smem = gt_fixed_smem<NT, MODE>(p.G, p.T) + (size_t)p.stages * GT_STAGE_BYTES;
-  QB_CUDA(cudaFuncSetAttribute(lowbit_gemv_kernel<NT, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  lowbit_gemv_kernel<NT, MODE><<<grid, GT_THREADS, smem, st>>>(tm_c, tm_a, tm_b, p);
+  p.stages = t1_stages(p.G);
+  const size_t smem = t1_fixed_smem(p.G) + (size_t)p.stages * GT_STAGE_BYTES;
+  QB_CUDA(cudaFuncSetAttribute(lowbit_gemv_t1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  lowbit_gemv_t1_kernel<<<grid, GT_THREADS, smem, st>>>(tm_c, tm_a, tm_b, p);
   return QBLORA_OK;
 }
 
 // ---------------------------------------------------------------------------------------------------
-// K-outer variant for 2..16 tokens.  A small kernel first turns x into fp16 MMA fragments in the
+// K-outer variant for 2..16 tokens (and for one token when its fragments do not fit shared memory).  A small kernel first turns x into fp16 MMA fragments in the
 // workspace: per K tile a contiguous block [16 groups][NTOK tokens][4 quarters][32 B] plus, per group
 // and token, (1024 P 2^e, R 2^e, 2^e, 0), where 2^-e is that 64-value slice's own power-of-two
 // prescale, P the sum of the fragment values and R the sum of the scaled x (so no pass over all of x
@@ -897,15 +722,14 @@ bool gemv_supported(const QwView& qw, int64_t T) {
 }
 
 size_t gemv_ws_bytes(const QwView& qw, int64_t T) {
-  if (T <= 1) return kStatusBytes;
+  // status word, then the token fragments of the K-outer kernel (one K tile after the other)
   const size_t n_kc = (size_t)(qw.G + GT_GROUPS - 1) / GT_GROUPS;
   return kStatusBytes + n_kc * (T <= 8 ? (size_t)KoCfg<1>::KT_BYTES : (size_t)KoCfg<2>::KT_BYTES);
 }
 
 int launch_lowbit_gemv(const QwView& qw, const __nv_bfloat16* X, int64_t T, void* Y, int y_dtype, int* status,
                        cudaStream_t st) {
-  uint8_t* xfrag = reinterpret_cast<uint8_t*>(status) + kStatusBytes;   // T > 1: fragments of x (see gemv_ws_bytes)
-  const int NT = T <= 8 ? 1 : 2;
+  uint8_t* xfrag = reinterpret_cast<uint8_t*>(status) + kStatusBytes;   // fragments of x (see gemv_ws_bytes)
   GtParams p{};
   p.d_in = qw.d_in; p.d_out = qw.d_out; p.G = qw.G; p.T = (int)T;
   p.n_rb = (qw.d_out + GT_ROWS - 1) / GT_ROWS;
@@ -925,18 +749,12 @@ int launch_lowbit_gemv(const QwView& qw, const __nv_bfloat16* X, int64_t T, void
   int sms = 148;
   { int dev = 0; if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); }
   const int grid = p.n_rb < sms ? p.n_rb : sms;
-  // fp16 fragments of x fit in shared memory next to a six-stage ring?
-  const bool xs = NT == 1 && (T == 1 ? gt_stages<1, 2>(p.G, p.T) : gt_stages<1, 1>(p.G, p.T)) >= 6;
   {
     DominantKernelTimer timer(st);
     count_launch();
-    static const bool ko_off = [] { const char* e = getenv("QBLORA_GEMV_KOUTER"); return e && e[0] == '0'; }();
-    if (xs && T == 1) rc = gt_launch<1, 2>(tm_c, tm_a, tm_b, p, grid, st);
-    else if (!ko_off && NT == 1) rc = ko_launch<1>(tm_c, tm_a, tm_b, p, grid, xfrag, st);
-    else if (!ko_off) rc = ko_launch<2>(tm_c, tm_a, tm_b, p, grid, xfrag, st);
-    else if (xs) rc = gt_launch<1, 1>(tm_c, tm_a, tm_b, p, grid, st);
-    else if (NT == 1) rc = gt_launch<1, 0>(tm_c, tm_a, tm_b, p, grid, st);
-    else rc = gt_launch<2, 0>(tm_c, tm_a, tm_b, p, grid, st);
+    if (T == 1 && t1_stages(p.G) > 0) rc = t1_launch(tm_c, tm_a, tm_b, p, grid, st);
+    else if (T <= 8) rc = ko_launch<1>(tm_c, tm_a, tm_b, p, grid, xfrag, st);
+    else rc = ko_launch<2>(tm_c, tm_a, tm_b, p, grid, xfrag, st);
     if (rc) return rc;
   }
   QB_CUDA(cudaGetLastError());

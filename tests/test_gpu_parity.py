@@ -226,3 +226,14 @@ def test_lowbit_decode_token_range(qb, T, log2_gain):
     ref = oracle.lowbit_gemm(qw, X)
     dq, Xd = qweight_to_dev(qw), to_bf16_dev(X)
     gate_strict(to_np64(qb.lowbit_gemm(dq, Xd, torch.float32)), ref, f"lowbit range T={T} gain=2^{log2_gain}")
+
+
+@pytest.mark.parametrize("T", [1, 5])
+def test_lowbit_decode_wide_input(qb, T):
+    # 896 groups per row: the one-token kernel's resident token fragments no longer fit beside its tile
+    # ring, so T = 1 takes the kernel that streams them (the one T = 5 uses anyway); 72 rows = two
+    # full row blocks and a ragged one.
+    qw, _, X, _ = make_case(58, T, 72, 896 * 64, 64, 8, 16, qfmt=1)
+    ref = oracle.lowbit_gemm(qw, X)
+    dq, Xd = qweight_to_dev(qw), to_bf16_dev(X)
+    gate_strict(to_np64(qb.lowbit_gemm(dq, Xd, torch.float32)), ref, f"lowbit wide T={T}")
