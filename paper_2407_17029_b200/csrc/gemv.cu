@@ -452,6 +452,9 @@ __global__ void __launch_bounds__(256) x_prepare_kernel(const __nv_bfloat16* __r
                                                         int n_kc, uint8_t* __restrict__ out) {
   using Cfg = KoCfg<NT>;
   constexpr int NTOK = Cfg::NTOK;
+  // the main kernel is launched as a programmatic dependent: it may start (set up, stream weights) now and
+  // waits for this grid's completion only before it reads the fragments
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int idx = blockIdx.x * 256 + threadIdx.x;
   const int total = n_kc * GT_GROUPS * NTOK * 4;
   const bool in_range = idx < total;
@@ -544,9 +547,14 @@ lowbit_gemv_ko_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
         if (pass * RB * (int)gridDim.x + (int)blockIdx.x >= p.n_rb) break;   // no row block left for this CTA
         for (int kc = 0; kc < p.n_kc && ok; ++kc, ++xit) {
           const uint32_t xb = xit & 1u;
-          if (!gv_wait(xempty(xb), ((xit >> 1) & 1u) ^ 1u, p.status)) { ok = false; break; }
-          mbar_arrive_expect_tx(xfull(xb), Cfg::KT_BYTES);
-          gv_bulk_load(base + xbuf_off + xb * Cfg::KT_BYTES, xfrag + (size_t)kc * Cfg::KT_BYTES, Cfg::KT_BYTES, xfull(xb));
+          // The very first fragment block is requested AFTER the first weight tiles: the weights do not
+          // depend on the kernel that prepares the fragments, whose completion is awaited just before.
+          const bool first = xit == 0;
+          if (!first) {
+            if (!gv_wait(xempty(xb), ((xit >> 1) & 1u) ^ 1u, p.status)) { ok = false; break; }
+            mbar_arrive_expect_tx(xfull(xb), Cfg::KT_BYTES);
+            gv_bulk_load(base + xbuf_off + xb * Cfg::KT_BYTES, xfrag + (size_t)kc * Cfg::KT_BYTES, Cfg::KT_BYTES, xfull(xb));
+          }
           for (int j = 0; j < RB; ++j) {
             const int rb = (pass * RB + j) * gridDim.x + blockIdx.x;
             if (rb >= p.n_rb) break;
@@ -560,6 +568,11 @@ lowbit_gemv_ko_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
             tma_load_2d(st + GT_CODE_BYTES + GT_SCALE_BYTES, &tm_b, full(s), kc * GT_GROUPS, rb * GT_ROWS);
             ++it;
             if (++s == STAGES) { s = 0; ph ^= 1u; }
+          }
+          if (first) {
+            asm volatile("griddepcontrol.wait;" ::: "memory");   // the fragments are complete and visible
+            mbar_arrive_expect_tx(xfull(xb), Cfg::KT_BYTES);
+            gv_bulk_load(base + xbuf_off + xb * Cfg::KT_BYTES, xfrag + (size_t)kc * Cfg::KT_BYTES, Cfg::KT_BYTES, xfull(xb));
           }
         }
       }
@@ -710,7 +723,14 @@ int ko_launch(const CUtensorMap& tm_c, const CUtensorMap& tm_a, const CUtensorMa
   count_launch();
   const size_t smem = KoCfg<NT>::FIXED + (size_t)p.stages * GT_STAGE_BYTES;
   QB_CUDA(cudaFuncSetAttribute(lowbit_gemv_ko_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  lowbit_gemv_ko_kernel<NT><<<grid, GT_THREADS, smem, st>>>(tm_c, tm_a, tm_b, p, xfrag);
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(GT_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  const uint8_t* xf = xfrag;
+  QB_CUDA(cudaLaunchKernelEx(&cfg, lowbit_gemv_ko_kernel<NT>, tm_c, tm_a, tm_b, p, xf));
   return QBLORA_OK;
 }
 
