@@ -184,14 +184,20 @@ def device_status(ws: torch.Tensor, stream=None) -> int:
 
 def quantize_blockwise(W: torch.Tensor, block_in: int = 64, block_out: int = 1,
                        qfmt: int = FMT_CODEBOOK_ABSMAX, code: Optional[List[float]] = None,
-                       stream=None) -> QWeight:
+                       stream=None, out: Optional[QWeight] = None) -> QWeight:
+    """Quantizes W [d_out][d_in] (fp32 or bf16).  `out`: a QWeight of the same geometry whose tensors are
+    overwritten (no allocation in the call)."""
     assert W.is_cuda and W.is_contiguous() and W.dim() == 2
     d_out, d_in = W.shape
     if qfmt == FMT_CODEBOOK_ABSMAX and code is None:
         code = default_code_table()
-    codes = torch.empty((d_out, d_in // 2), dtype=torch.uint8, device=W.device)
-    alpha = torch.empty((max(d_out // block_out, 1), max(d_in // block_in, 1)), dtype=torch.float32, device=W.device)
-    beta = torch.empty_like(alpha) if qfmt == FMT_AFFINE_MINMAX else None
+    if out is not None:
+        assert (out.d_out, out.d_in, out.block_in, out.block_out, out.qfmt) == (d_out, d_in, block_in, block_out, qfmt)
+        codes, alpha, beta = out.codes, out.alpha, out.beta
+    else:
+        codes = torch.empty((d_out, d_in // 2), dtype=torch.uint8, device=W.device)
+        alpha = torch.empty((max(d_out // block_out, 1), max(d_in // block_in, 1)), dtype=torch.float32, device=W.device)
+        beta = torch.empty_like(alpha) if qfmt == FMT_AFFINE_MINMAX else None
     ctab = (ctypes.c_float * 16)(*code) if code is not None else None
     st = _lib.qblora_quantize_blockwise(W.data_ptr(), _dt(W.dtype), d_out, d_in, block_in, block_out, qfmt,
                                         ctab, codes.data_ptr(), alpha.data_ptr(),

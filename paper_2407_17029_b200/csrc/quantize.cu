@@ -30,59 +30,70 @@ __device__ __forceinline__ int code_of_affine(float w, float beta, float alpha) 
   return (int)rq;
 }
 
-// One warp per block of 64 consecutive elements of a row (block_in == 64, block_out == 1).
-// Because d_in is a multiple of 64, block b is the flat element range [64 b, 64 b + 64) and its
-// packed codes are bytes [32 b, 32 b + 32).  Lane l owns elements 2l, 2l+1 = byte l.
+// block_in == 64, block_out == 1.  Because d_in is a multiple of 64, block b is the flat element range
+// [64 b, 64 b + 64) and its packed codes are bytes [32 b, 32 b + 32).  A warp takes four consecutive
+// blocks per step: lane l owns elements 8 (l % 8) .. + 7 of block 4 w + l / 8 (one or two 16-byte loads,
+// 1 KB / 512 B per warp and step, contiguous), the block's min / max / absmax come from three shuffle
+// rounds inside its eight lanes, and the lane's eight codes leave as one 32-bit store.
 template <typename TIn>
 __global__ void __launch_bounds__(256) quantize_b64_kernel(const TIn* __restrict__ W, int64_t nblocks,
                                                            int qfmt, QuantTable tab,
                                                            uint8_t* __restrict__ codes,
                                                            float* __restrict__ alpha,
                                                            float* __restrict__ beta) {
-  const int lane = threadIdx.x & 31;
+  const int lane = threadIdx.x & 31, sub = lane >> 3, part = lane & 7;
   const int64_t warps_per_grid = (int64_t)gridDim.x * (blockDim.x >> 5);
-  for (int64_t b = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); b < nblocks;
-       b += warps_per_grid) {
-    float w0, w1;
-    if constexpr (sizeof(TIn) == 4) {
-      float2 v = reinterpret_cast<const float2*>(W)[b * 32 + lane];
-      w0 = v.x; w1 = v.y;
-    } else {
-      __nv_bfloat162 v = reinterpret_cast<const __nv_bfloat162*>(W)[b * 32 + lane];
-      w0 = __low2float(v); w1 = __high2float(v);
-    }
-    float mn = fminf(w0, w1), mx = fmaxf(w0, w1), am = fmaxf(fabsf(w0), fabsf(w1));
+  const int64_t steps = (nblocks + 3) >> 2;
+  for (int64_t w = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); w < steps; w += warps_per_grid) {
+    const int64_t b = 4 * w + sub;
+    const bool live = b < nblocks;
+    float v[8];
 #pragma unroll
-    for (int s = 16; s > 0; s >>= 1) {
+    for (int e = 0; e < 8; ++e) v[e] = 0.0f;
+    if (live) {
+      if constexpr (sizeof(TIn) == 4) {
+        const float4* src = reinterpret_cast<const float4*>(W) + (b * 16 + part * 2);
+        const float4 x0 = src[0], x1 = src[1];
+        v[0] = x0.x; v[1] = x0.y; v[2] = x0.z; v[3] = x0.w; v[4] = x1.x; v[5] = x1.y; v[6] = x1.z; v[7] = x1.w;
+      } else {
+        const uint4 x = reinterpret_cast<const uint4*>(W)[b * 8 + part];
+        const uint32_t xw[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) { v[2 * e] = __uint_as_float(xw[e] << 16); v[2 * e + 1] = __uint_as_float(xw[e] & 0xffff0000u); }
+      }
+    }
+    float mn = v[0], mx = v[0], am = fabsf(v[0]);
+#pragma unroll
+    for (int e = 1; e < 8; ++e) { mn = fminf(mn, v[e]); mx = fmaxf(mx, v[e]); am = fmaxf(am, fabsf(v[e])); }
+#pragma unroll
+    for (int s = 4; s > 0; s >>= 1) {
       mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, s));
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, s));
       am = fmaxf(am, __shfl_xor_sync(0xffffffffu, am, s));
     }
-    int c0, c1;
+    uint32_t packed = 0;
     if (qfmt == QBLORA_FMT_CODEBOOK_ABSMAX) {
-      if (am != 0.0f) {
-        c0 = code_of_level(__fdiv_rn(w0, am), tab);
-        c1 = code_of_level(__fdiv_rn(w1, am), tab);
-      } else {
-        c0 = c1 = tab.zero_idx;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const int c = am != 0.0f ? code_of_level(__fdiv_rn(v[e], am), tab) : tab.zero_idx;
+        packed |= (uint32_t)c << (4 * e);
       }
-      if (lane == 0) alpha[b] = am;
+      if (live && part == 0) alpha[b] = am;
     } else {
-      float d = __fsub_rn(mx, mn);
-      float a = __fdiv_rn(d, 15.0f);
-      bool degenerate = (d == 0.0f) || (a == 0.0f);
-      if (!degenerate) {
-        c0 = code_of_affine(w0, mn, a);
-        c1 = code_of_affine(w1, mn, a);
-      } else {
-        c0 = c1 = 0;
+      const float d = __fsub_rn(mx, mn);
+      const float a = __fdiv_rn(d, 15.0f);
+      const bool degenerate = (d == 0.0f) || (a == 0.0f);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const int c = degenerate ? 0 : code_of_affine(v[e], mn, a);
+        packed |= (uint32_t)c << (4 * e);
       }
-      if (lane == 0) {
+      if (live && part == 0) {
         alpha[b] = degenerate ? 0.0f : a;
         beta[b] = mn;
       }
     }
-    codes[b * 32 + lane] = (uint8_t)(c0 | (c1 << 4));
+    if (live) reinterpret_cast<uint32_t*>(codes)[b * 8 + part] = packed;   // element 2k in the low nibble of byte k
   }
 }
 
@@ -146,7 +157,7 @@ int launch_quantize(const void* W, int w_dtype, int d_out, int d_in, int block_i
   }
   if (block_in == 64 && block_out == 1) {
     int64_t nblocks = (int64_t)d_out * (d_in / 64);
-    int64_t ctas = (nblocks + 7) / 8;
+    int64_t ctas = ((nblocks + 3) / 4 + 7) / 8;      // four blocks per warp and step, eight warps per CTA
     int grid = (int)(ctas < 148 * 16 ? ctas : 148 * 16);
     if (grid < 1) grid = 1;
     if (w_dtype == QBLORA_F32)
