@@ -82,7 +82,7 @@ typedef struct {
   float scaling;                 /* s; multiplies the adapter term only */
   const void* A;                 /* DEVICE bf16 [P][r] */
   const void* B;                 /* DEVICE bf16 [r][Q]; NULL => A is the single matrix H, bf16 [P][Q],
-                                    of Sec. 3.3 / Algorithm 2 (accepted by qablora_merge only) */
+                                    of Sec. 3.3 / Algorithm 2 (rank is then ignored) */
 } qblora_adapter;
 
 /* Writes the built-in 16-level table (HOST out): nine non-negative levels
@@ -152,6 +152,9 @@ int qblora_linear_fwd(const qblora_qweight* qw, const qblora_adapter* adapter, c
  *   dY DEVICE bf16 [tokens][d_out];  dX DEVICE out [tokens][d_in] (dx_dtype BF16 or F32);
  *   dA DEVICE out fp32 [P][r];  dB DEVICE out fp32 [r][Q].  Any of dX, dA, dB may be NULL (skipped).
  *   adapter may be NULL (then dA and dB must be NULL).
+ *   Single-matrix adapter (adapter->B == NULL, Sec. 3.3): the adapter term of the forward is
+ *   s * (x' H)[t][o / lambda_out]; dA receives dH = x'^T dv as fp32 [P][Q], dB must be NULL, and the
+ *   pooled-input gradient is dv H^T.
  */
 int qblora_linear_bwd(const qblora_qweight* qw, const qblora_adapter* adapter, const void* X,
                       const void* dY, int64_t tokens, void* dX, int dx_dtype, float* dA, float* dB,

@@ -77,6 +77,25 @@ int reset_status(void* ws, cudaStream_t st) {
   return QBLORA_OK;
 }
 
+// Single-matrix adapters (B == NULL, A is H [P][Q]; Sec. 3.3 / Algorithm 2) train through the same
+// kernels as the two-factor form with A := I_P, B := H, r := P: then u = x' I = x' exactly, the adapter
+// output is s * repeat(x' H), dB of the factored form is dH = x'^T dv, and du I^T = dv H^T is the
+// pooled-input gradient.  The identity lives at the end of the workspace and is written per call.
+size_t single_identity_bytes(const AdView& ad) { return align_up((size_t)ad.P * ad.P * 2, 256); }
+AdView single_as_factored(const AdView& ad, const __nv_bfloat16* identity) {
+  AdView f = ad;
+  f.r = ad.P;
+  f.B = ad.A;          // H
+  f.A = identity;
+  return f;
+}
+
+size_t ws_bytes_impl(int op, const QwView& q, const AdView* ad, int64_t T);
+size_t ws_bytes_single(int op, const QwView& q, const AdView& ad, int64_t T) {
+  const AdView f = single_as_factored(ad, nullptr);
+  return align_up(ws_bytes_impl(op, q, &f, T), 256) + single_identity_bytes(ad);
+}
+
 size_t ws_bytes_impl(int op, const QwView& q, const AdView* ad, int64_t T) {
   switch (op) {
     case QBLORA_OP_QUANTIZE: return 0;
@@ -131,6 +150,8 @@ size_t qblora_workspace_bytes(int op, const qblora_qweight* qw, const qblora_ada
     adp = &ad;
   }
   if (op != QBLORA_OP_MERGE && op != QBLORA_OP_QUANTIZE && tokens < 1) return 0;
+  if (adp && !adapter->B && (op == QBLORA_OP_LINEAR_FWD || op == QBLORA_OP_LINEAR_BWD))
+    return ws_bytes_single(op, q, ad, tokens);
   return ws_bytes_impl(op, q, adp, tokens);
 }
 
@@ -171,14 +192,21 @@ int qblora_linear_fwd(const qblora_qweight* qw, const qblora_adapter* adapter, c
   if (adapter) {
     rc = make_ad(adapter, q, true, &ad);
     if (rc) return rc;
-    if (!adapter->B) return QBLORA_ERR_UNSUPPORTED;  // single-matrix adapters: merge only
     adp = &ad;
   }
-  const size_t need = ws_bytes_impl(QBLORA_OP_LINEAR_FWD, q, adp, tokens);
+  const bool single = adapter && !adapter->B;
+  const size_t need = single ? ws_bytes_single(QBLORA_OP_LINEAR_FWD, q, ad, tokens)
+                             : ws_bytes_impl(QBLORA_OP_LINEAR_FWD, q, adp, tokens);
   if (!ws || !aligned16(ws) || ws_bytes < need) return QBLORA_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   rc = reset_status(ws, st);
   if (rc) return rc;
+  if (single) {
+    __nv_bfloat16* eye = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(ws) + need - single_identity_bytes(ad));
+    rc = launch_identity(eye, ad.P, st);
+    if (rc) return rc;
+    ad = single_as_factored(ad, eye);
+  }
   const __nv_bfloat16* Xb = static_cast<const __nv_bfloat16*>(X);
   if (!force_general() && tc_supported(q, adp, tokens))
     return tc_linear_fwd(q, adp, Xb, tokens, Y, y_dtype, static_cast<char*>(ws), st);
@@ -197,18 +225,28 @@ int qblora_linear_bwd(const qblora_qweight* qw, const qblora_adapter* adapter, c
   if (adapter) {
     rc = make_ad(adapter, q, true, &ad);
     if (rc) return rc;
-    if (!adapter->B) return QBLORA_ERR_UNSUPPORTED;
+    if (!adapter->B && dB) return QBLORA_ERR_INVALID_ARG;   // single matrix: its gradient dH goes to dA
     if (!X || !aligned16(X)) return QBLORA_ERR_INVALID_ARG;
     adp = &ad;
   } else if (dA || dB) {
     return QBLORA_ERR_INVALID_ARG;
   }
   if (!dX && !dA && !dB) return QBLORA_OK;
-  const size_t need = ws_bytes_impl(QBLORA_OP_LINEAR_BWD, q, adp, tokens);
+  const bool single = adapter && !adapter->B;
+  const size_t need = single ? ws_bytes_single(QBLORA_OP_LINEAR_BWD, q, ad, tokens)
+                             : ws_bytes_impl(QBLORA_OP_LINEAR_BWD, q, adp, tokens);
   if (!ws || !aligned16(ws) || ws_bytes < need) return QBLORA_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   rc = reset_status(ws, st);
   if (rc) return rc;
+  if (single) {
+    __nv_bfloat16* eye = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(ws) + need - single_identity_bytes(ad));
+    rc = launch_identity(eye, ad.P, st);
+    if (rc) return rc;
+    ad = single_as_factored(ad, eye);
+    dB = dA;          // dH = x'^T dv is the factored form's dB
+    dA = nullptr;     // the identity is not trained
+  }
   const __nv_bfloat16* Xb = static_cast<const __nv_bfloat16*>(X);
   const __nv_bfloat16* dYb = static_cast<const __nv_bfloat16*>(dY);
   if (!force_general() && tc_supported(q, adp, tokens))

@@ -112,4 +112,19 @@ int simt_linear_bwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X,
   return QBLORA_OK;
 }
 
+namespace {
+__global__ void identity_kernel(__nv_bfloat16* out, int n) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx < (int64_t)n * n) out[idx] = __float2bfloat16_rn((idx / n) == (idx % n) ? 1.0f : 0.0f);
+}
+}  // namespace
+
+int launch_identity(__nv_bfloat16* out, int n, cudaStream_t st) {
+  const int64_t total = (int64_t)n * n;
+  identity_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(out, n);
+  count_launch();
+  QB_CUDA(cudaGetLastError());
+  return QBLORA_OK;
+}
+
 }  // namespace qb

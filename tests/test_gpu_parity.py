@@ -237,3 +237,26 @@ def test_lowbit_decode_wide_input(qb, T):
     ref = oracle.lowbit_gemm(qw, X)
     dq, Xd = qweight_to_dev(qw), to_bf16_dev(X)
     gate_strict(to_np64(qb.lowbit_gemm(dq, Xd, torch.float32)), ref, f"lowbit wide T={T}")
+
+
+@pytest.mark.parametrize("case", [(300, 320, 448, 64, 8), (150, 128, 512, 8, 8), (77, 136, 192, 4, 4)])
+@pytest.mark.parametrize("visible", [False, True])
+def test_single_matrix_adapter_fwd_bwd(qb, path, case, visible):
+    # Sec. 3.3's single matrix H [P][Q] (B == NULL) trained directly: forward s * repeat(x' H),
+    # backward dH = x'^T dv (returned in dA) and dX with the pooled-input gradient dv H^T.
+    T, d_out, d_in, l1, l2 = case
+    qw, _, X, dY = make_case(61, T, d_out, d_in, l1, l2, 16, qfmt=1)
+    H = synth.round_to_bf16(synth.normal(61, "H", (d_in // l1, d_out // l2), 0.02))
+    ad = oracle.Adapter(l1, l2, 0, 1.0, H, None)
+    Wt = oracle.dequantize(qw)
+    if visible:
+        ad.scaling = visible_scaling(Wt, ad, X)
+    dq, da, Xd, dYd = qweight_to_dev(qw), adapter_to_dev(ad), to_bf16_dev(X), to_bf16_dev(dY)
+    gate_strict(to_np64(qb.linear_fwd(dq, da, Xd, torch.float32)), oracle.linear_fwd(Wt, ad, X), "Y single matrix")
+    gate_bf16(to_np64(qb.linear_fwd(dq, da, Xd, torch.bfloat16)), oracle.linear_fwd(Wt, ad, X), "Y single matrix bf16")
+    rdX, rdH, rdB = oracle.linear_bwd(Wt, ad, X, dY)
+    assert rdB is None
+    dX, dH, dB = qb.linear_bwd(dq, da, Xd, dYd, torch.float32)
+    assert dB is None and tuple(dH.shape) == H.shape
+    gate_strict(to_np64(dX), rdX, "dX single matrix")
+    gate_strict(to_np64(dH), rdH, "dH", per_row=False)
