@@ -25,6 +25,7 @@
 // Two kernels: one token (fragments of x resident in shared memory, row blocks outer) and 2..16
 // tokens (K tiles outer, fragments prepared once in the workspace and streamed per K tile).
 #include <cstdlib>
+#include <atomic>
 #include "tc_ptx.cuh"
 #include "tc_small.cuh"
 
@@ -171,6 +172,43 @@ struct GtParams {
   void* Y;
   int y_dtype;
   int* status;
+  // one-token kernel, split tail (see T1Walk): row blocks done whole, ways the rest is split, hand-over area
+  int tail_first, tail_split;
+  uint32_t epoch;            // value a hand-over flag takes in this launch (never 0, differs from launch to launch)
+  float* tail_partial;       // [tail row block][part][32 rows] fp32
+  uint32_t* tail_flags;      // [tail row block][part]
+};
+
+// Row blocks of one CTA in the one-token kernel.  Whole row blocks b, b + G, ... below tail_first; then,
+// when the remaining row blocks would occupy at most half of the CTAs, each of them is split along K
+// into tail_split parts given to different CTAs (unit u = blockIdx.x: row block tail_first + u /
+// split, part u % split), so the last round takes 1 / split of a round instead of a whole one.  Part
+// 0 owns the row block: it adds the other parts' sums (handed over through global memory) and stores.
+struct T1Walk {
+  int rb, kc0, kc1, part;
+  bool tail;
+  int next_full, done_tail;
+  __device__ T1Walk() : next_full((int)blockIdx.x), done_tail(0) {}
+  __device__ bool next(const GtParams& p) {
+    if (next_full < p.tail_first) {
+      rb = next_full; kc0 = 0; kc1 = p.n_kc; part = 0; tail = false;
+      next_full += gridDim.x;
+      return true;
+    }
+    if (done_tail) return false;
+    done_tail = 1;
+    if (p.tail_split <= 1) {        // the rest as whole row blocks (at most one more per CTA)
+      rb = next_full; kc0 = 0; kc1 = p.n_kc; part = 0; tail = false;
+      return rb < p.n_rb;
+    }
+    const int u = (int)blockIdx.x;
+    rb = p.tail_first + u / p.tail_split;
+    part = u % p.tail_split;
+    if (rb >= p.n_rb) return false;
+    kc0 = p.n_kc * part / p.tail_split; kc1 = p.n_kc * (part + 1) / p.tail_split;
+    tail = true;
+    return true;
+  }
 };
 
 // ---------------------------------------------------------------------------------------------------
@@ -220,8 +258,10 @@ lowbit_gemv_t1_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
       uint32_t it = 0, ph = 0;
       int s = 0;
       bool ok = true;
-      for (int rb = blockIdx.x; rb < p.n_rb && ok; rb += gridDim.x) {
-        for (int kc = 0; kc < p.n_kc; ++kc, ++it) {
+      T1Walk walk;
+      while (ok && walk.next(p)) {
+        const int rb = walk.rb;
+        for (int kc = walk.kc0; kc < walk.kc1; ++kc, ++it) {
           if (!gv_wait(empty(s), ph ^ 1u, p.status)) { ok = false; break; }
           const uint32_t st = base + s * GT_STAGE_BYTES;
           mbar_arrive_expect_tx(full(s), GT_STAGE_BYTES);
@@ -328,9 +368,11 @@ lowbit_gemv_t1_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
                            // barriers still match) but no longer waits or computes
     int s = 0;
     uint32_t ph = 0;
-    for (int rb = blockIdx.x; rb < p.n_rb; rb += gridDim.x) {
+    T1Walk walk;
+    while (walk.next(p)) {
+      const int rb = walk.rb;
       float y[2][2] = {{0.0f, 0.0f}, {0.0f, 0.0f}};    // [row tile][row g, row g + 8], token 0 (lanes tg == 0)
-      for (int kc = 0; kc < p.n_kc; ++kc) {
+      for (int kc = walk.kc0; kc < walk.kc1; ++kc) {
         if (ok && !gv_wait(full(s), ph, p.status)) ok = false;
         const int grp = kc * GT_GROUPS + warp;
         if (ok) {
@@ -386,6 +428,32 @@ lowbit_gemv_t1_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
         for (int ww = 0; ww < GT_WARPS; ++ww) a += red[ww * GT_ROWS + lane];
         __syncwarp();
         if (lane == 0) gv_release(red_free, a, a, a, a);
+        if (walk.tail) {
+          const int slot = (rb - p.tail_first) * p.tail_split;
+          if (walk.part != 0) {
+            // hand this K range's sums to the owner: stores, fence, then the flag (this launch's epoch)
+            p.tail_partial[(slot + walk.part) * GT_ROWS + lane] = a;
+            __threadfence();
+            __syncwarp();
+            if (lane == 0) atomicExch(p.tail_flags + slot + walk.part, p.epoch);
+            ++rcount; rph ^= 1u;
+            continue;
+          }
+          for (int part = 1; part < p.tail_split; ++part) {      // bounded wait, then add in part order
+            uint32_t seen = p.epoch;
+            if (lane == 0 && ok) {
+              const long long w0 = clock64();
+              while ((seen = *reinterpret_cast<volatile uint32_t*>(p.tail_flags + slot + part)) != p.epoch) {
+                __nanosleep(100);
+                if (clock64() - w0 > WAIT_LIMIT_CYCLES) { atomicExch(p.status, (int)QBLORA_ERR_TIMEOUT); break; }
+              }
+            }
+            seen = __shfl_sync(0xFFFFFFFFu, seen, 0);
+            if (seen != p.epoch) ok = false;
+            __threadfence();
+            a += __ldcg(p.tail_partial + (slot + part) * GT_ROWS + lane);
+          }
+        }
         a *= y_scale;
         const int o = rb * GT_ROWS + lane;                // lane = row of the block
         if (o < p.d_out) {
@@ -741,10 +809,15 @@ bool gemv_supported(const QwView& qw, int64_t T) {
   return qw.block_in == 64 && qw.block_out == 1 && qw.qfmt == QBLORA_FMT_AFFINE_MINMAX && T <= 16 && qw.G % 4 == 0 && qw.G <= 1024;
 }
 
+constexpr int T1_TAIL_MAX_BLOCKS = 128, T1_TAIL_MAX_SPLIT = 4;   // row blocks in a split tail, parts each
+constexpr size_t T1_TAIL_BYTES = (size_t)T1_TAIL_MAX_BLOCKS * T1_TAIL_MAX_SPLIT * (GT_ROWS * 4 + 4);
+
 size_t gemv_ws_bytes(const QwView& qw, int64_t T) {
-  // status word, then the token fragments of the K-outer kernel (one K tile after the other)
+  // status word, then either the token fragments of the K-outer kernel (one K tile after the other)
+  // or the hand-over area of the one-token kernel's split tail (sums, then flags)
   const size_t n_kc = (size_t)(qw.G + GT_GROUPS - 1) / GT_GROUPS;
-  return kStatusBytes + n_kc * (T <= 8 ? (size_t)KoCfg<1>::KT_BYTES : (size_t)KoCfg<2>::KT_BYTES);
+  const size_t frag = n_kc * (T <= 8 ? (size_t)KoCfg<1>::KT_BYTES : (size_t)KoCfg<2>::KT_BYTES);
+  return kStatusBytes + (frag > T1_TAIL_BYTES ? frag : T1_TAIL_BYTES);
 }
 
 int launch_lowbit_gemv(const QwView& qw, const __nv_bfloat16* X, int64_t T, void* Y, int y_dtype, int* status,
@@ -768,11 +841,32 @@ int launch_lowbit_gemv(const QwView& qw, const __nv_bfloat16* X, int64_t T, void
   if (rc) return rc;
   int sms = 148;
   { int dev = 0; if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); }
-  const int grid = p.n_rb < sms ? p.n_rb : sms;
+  int grid = p.n_rb < sms ? p.n_rb : sms;
+  const bool one_token = T == 1 && t1_stages(p.G) > 0;
+  p.tail_first = p.n_rb; p.tail_split = 1;
+  if (one_token) {
+    // Split tail (see T1Walk): the row blocks left after the whole rounds, when they would keep at most
+    // half of the CTAs busy, are cut along K so that all CTAs share them.
+    static std::atomic<uint32_t> launches{0};
+    const int whole = p.n_rb >= sms ? (p.n_rb / sms) * sms : 0;
+    const int rem = p.n_rb - whole;
+    int split = rem > 0 ? sms / rem : 1;
+    if (split > T1_TAIL_MAX_SPLIT) split = T1_TAIL_MAX_SPLIT;
+    if (split > p.n_kc) split = p.n_kc;
+    // the hand-over costs about as much as three tiles: split only when it saves clearly more
+    if (split >= 2 && rem <= T1_TAIL_MAX_BLOCKS && p.n_kc - p.n_kc / split >= 8) {
+      p.tail_first = whole; p.tail_split = split;
+      if (whole == 0) grid = rem * split;
+      uint32_t e = launches.fetch_add(1) + 1;
+      p.epoch = e == 0 ? launches.fetch_add(1) + 1 : e;
+      p.tail_partial = reinterpret_cast<float*>(xfrag);
+      p.tail_flags = reinterpret_cast<uint32_t*>(xfrag + (size_t)T1_TAIL_MAX_BLOCKS * T1_TAIL_MAX_SPLIT * GT_ROWS * 4);
+    }
+  }
   {
     DominantKernelTimer timer(st);
     count_launch();
-    if (T == 1 && t1_stages(p.G) > 0) rc = t1_launch(tm_c, tm_a, tm_b, p, grid, st);
+    if (one_token) rc = t1_launch(tm_c, tm_a, tm_b, p, grid, st);
     else if (T <= 8) rc = ko_launch<1>(tm_c, tm_a, tm_b, p, grid, xfrag, st);
     else rc = ko_launch<2>(tm_c, tm_a, tm_b, p, grid, xfrag, st);
     if (rc) return rc;

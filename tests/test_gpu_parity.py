@@ -260,3 +260,17 @@ def test_single_matrix_adapter_fwd_bwd(qb, path, case, visible):
     assert dB is None and tuple(dH.shape) == H.shape
     gate_strict(to_np64(dX), rdX, "dX single matrix")
     gate_strict(to_np64(dH), rdH, "dH", per_row=False)
+
+
+@pytest.mark.parametrize("d_out", [72, 4768])
+def test_lowbit_one_token_split_tail(qb, d_out):
+    # One token, few row blocks against the CTA count: the row blocks left after the whole rounds are cut
+    # along K and summed across CTAs (3 row blocks x 4 parts; 149 row blocks = one whole round + 1 x 4).
+    qw, _, X, _ = make_case(59, 1, d_out, 64 * 256, 64, 8, 16, qfmt=1)      # 16 K tiles
+    ref = oracle.lowbit_gemm(qw, X)
+    dq, Xd = qweight_to_dev(qw), to_bf16_dev(X)
+    for _ in range(3):      # flags carry a per-launch epoch: repeated launches on one workspace
+        ws = qb.alloc_workspace(qb.OP_LOWBIT_GEMM, dq, None, 1)
+        for _ in range(2):
+            gate_strict(to_np64(qb.lowbit_gemm(dq, Xd, torch.float32, ws=ws)), ref, f"lowbit split tail d_out={d_out}")
+            assert qb.device_status(ws) == qb.OK
