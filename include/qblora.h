@@ -152,6 +152,10 @@ int qblora_linear_fwd(const qblora_qweight* qw, const qblora_adapter* adapter, c
  *   dY DEVICE bf16 [tokens][d_out];  dX DEVICE out [tokens][d_in] (dx_dtype BF16 or F32);
  *   dA DEVICE out fp32 [P][r];  dB DEVICE out fp32 [r][Q].  Any of dX, dA, dB may be NULL (skipped).
  *   adapter may be NULL (then dA and dB must be NULL).
+ *   Stream: part of the work (the dA / dB chain) is enqueued on a stream the library creates on first
+ *   use (per host thread and device); it is ordered after `stream` at entry and joined back into
+ *   `stream` before the call returns, so the caller sees ordinary stream semantics (also inside a
+ *   stream capture).  Environment QBLORA_NO_OVERLAP=1 keeps everything on `stream`.
  *   Single-matrix adapter (adapter->B == NULL, Sec. 3.3): the adapter term of the forward is
  *   s * (x' H)[t][o / lambda_out]; dA receives dH = x'^T dv as fp32 [P][Q], dB must be NULL, and the
  *   pooled-input gradient is dv H^T.
