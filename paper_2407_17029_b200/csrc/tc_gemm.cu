@@ -389,36 +389,49 @@ template <bool DIVIDE>
 __global__ void __launch_bounds__(256) segsum_split_kernel(const __nv_bfloat16* __restrict__ src, int64_t rows, int width,
                                                            int lam, float scale, int ld_out,
                                                            __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+  constexpr int UNROLL = 4;       // 16-byte loads in flight per thread (the kernel is a pure stream)
   const int chunks_per_row = width >> 3;
   const int64_t total = rows * chunks_per_row;
-  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  const bool live = idx < total;
-  float v[8];
+  uint4 q4[UNROLL];
+  int64_t tt[UNROLL]; int cc[UNROLL]; bool lv[UNROLL];
 #pragma unroll
-  for (int e = 0; e < 8; ++e) v[e] = 0.0f;
-  int64_t t = 0; int c = 0;
-  if (live) {
-    t = idx / chunks_per_row; c = (int)(idx - t * chunks_per_row);
-    const uint4 q4 = __ldg(reinterpret_cast<const uint4*>(src + t * width) + c);
-    const uint32_t w[4] = {q4.x, q4.y, q4.z, q4.w};
+  for (int k = 0; k < UNROLL; ++k) {
+    const int64_t idx = ((int64_t)blockIdx.x * UNROLL + k) * blockDim.x + threadIdx.x;
+    lv[k] = idx < total;
+    tt[k] = 0; cc[k] = 0;
+    q4[k] = make_uint4(0, 0, 0, 0);
+    if (lv[k]) {
+      if (total < (1ll << 31)) { const uint32_t i32 = (uint32_t)idx; tt[k] = i32 / (uint32_t)chunks_per_row; }
+      else tt[k] = idx / chunks_per_row;
+      cc[k] = (int)(idx - tt[k] * chunks_per_row);
+      q4[k] = __ldg(reinterpret_cast<const uint4*>(src + tt[k] * width) + cc[k]);
+    }
+  }
+#pragma unroll
+  for (int k = 0; k < UNROLL; ++k) {
+    const bool live = lv[k];
+    const int64_t t = tt[k];
+    const int c = cc[k];
+    float v[8];
+    const uint32_t w[4] = {q4[k].x, q4[k].y, q4[k].z, q4[k].w};
 #pragma unroll
     for (int e = 0; e < 4; ++e) { v[2 * e] = __uint_as_float(w[e] << 16); v[2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u); }
-  }
-  if (lam >= 8) {
-    float sacc = ((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7]));
-    const int lanes = lam >> 3;   // power of two, <= 32; windows never straddle a warp (256 % lanes == 0, rows aligned)
-    for (int off = 1; off < lanes; off <<= 1) sacc += __shfl_xor_sync(0xffffffffu, sacc, off);
-    if (live && (c & (lanes - 1)) == 0) {
-      const float r = DIVIDE ? __fdiv_rn(sacc, (float)lam) : scale * sacc;
-      store_split(r, hi, lo, t * ld_out + c / lanes);
-    }
-  } else if (live) {
-    const int per = 8 / lam;      // windows inside this chunk
-    for (int j = 0; j < per; ++j) {
-      float sacc = 0.0f;
-      for (int e = 0; e < lam; ++e) sacc += v[j * lam + e];
-      const float r = DIVIDE ? __fdiv_rn(sacc, (float)lam) : scale * sacc;
-      store_split(r, hi, lo, t * ld_out + c * per + j);
+    if (lam >= 8) {
+      float sacc = ((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7]));
+      const int lanes = lam >> 3;   // power of two, <= 32; windows never straddle a warp (256 % lanes == 0, rows aligned)
+      for (int off = 1; off < lanes; off <<= 1) sacc += __shfl_xor_sync(0xffffffffu, sacc, off);
+      if (live && (c & (lanes - 1)) == 0) {
+        const float r = DIVIDE ? __fdiv_rn(sacc, (float)lam) : scale * sacc;
+        store_split(r, hi, lo, t * ld_out + c / lanes);
+      }
+    } else if (live) {
+      const int per = 8 / lam;      // windows inside this chunk
+      for (int j = 0; j < per; ++j) {
+        float sacc = 0.0f;
+        for (int e = 0; e < lam; ++e) sacc += v[j * lam + e];
+        const float r = DIVIDE ? __fdiv_rn(sacc, (float)lam) : scale * sacc;
+        store_split(r, hi, lo, t * ld_out + c * per + j);
+      }
     }
   }
 }
@@ -570,7 +583,7 @@ int launch_pool(const QwView& qw, const AdView& ad, const __nv_bfloat16* X, int6
   const int64_t n = T * ad.P;
   if (segsum_fast_ok(qw.d_in, ad.l1)) {
     const int64_t chunks = T * (qw.d_in / 8);
-    segsum_split_kernel<true><<<(unsigned)((chunks + 255) / 256), 256, 0, st>>>(X, T, qw.d_in, ad.l1, 0.0f, w.ldp, w.xh, w.xl);
+    segsum_split_kernel<true><<<(unsigned)((chunks + 1023) / 1024), 256, 0, st>>>(X, T, qw.d_in, ad.l1, 0.0f, w.ldp, w.xh, w.xl);
   } else {
     pool_split_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(X, T, qw.d_in, ad.l1, w.ldp, w.xh, w.xl);
   }
@@ -661,7 +674,7 @@ int tc_linear_bwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, co
     const int64_t n = T * ad->Q;
     if (segsum_fast_ok(qw.d_out, ad->l2)) {
       const int64_t chunks = T * (qw.d_out / 8);
-      segsum_split_kernel<false><<<(unsigned)((chunks + 255) / 256), 256, 0, st>>>(dY, T, qw.d_out, ad->l2, ad->s, w.ldq, w.dvh, w.dvl);
+      segsum_split_kernel<false><<<(unsigned)((chunks + 1023) / 1024), 256, 0, st>>>(dY, T, qw.d_out, ad->l2, ad->s, w.ldq, w.dvh, w.dvl);
     } else {
       dv_split_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(dY, T, qw.d_out, ad->l2, ad->s, w.ldq, w.dvh, w.dvl);
     }
