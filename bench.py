@@ -460,7 +460,7 @@ def lowbit_extras(qb, torch, dev, peaks, l2_bytes, shapes=("q", "up"), tokens=(1
                 chain.append(s.elapsed_time(e) / n_chain * 1e3)
             us = statistics.median(chain)
             gbs = nbytes / (us * 1e-6) / 1e9
-            out[f"{spec.name}/T{T}"] = {"kernel_us": us, "timing": f"CUDA-graph chain of {n_chain} launches over {ncopies} weight copies",
+            out[f"{spec.name}/T{T}"] = {"kernel_us": us, "timing": f"CUDA-graph chain of {n_chain} launches over {ncopies} weight copies (launches chained as programmatic dependents)",
                                         "GB/s": gbs, "frac_hbm": gbs / peaks["hbm_gbs"], "bytes": nbytes, "copies": ncopies,
                                         "single_launch_event_pair_us": single_us, "call_us_back_to_back": call_us,
                                         "status": qb.device_status(ws)}

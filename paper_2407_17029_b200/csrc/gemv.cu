@@ -242,6 +242,8 @@ lowbit_gemv_t1_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
   uint4* xs = reinterpret_cast<uint4*>(gbase + xs_off);
   const uint32_t zero_off = xs_off + (uint32_t)p.G * 128;
 
+  // a successor launched as a programmatic dependent may start on every SM this grid has left
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
     if (blockIdx.x == 0) *p.status = 0;   // any give-up below is written at least a wait limit later
@@ -281,6 +283,10 @@ lowbit_gemv_t1_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
   } else {
     // ------------------------------------------------------------------ compute warps
     const int g = lane >> 2, tg = lane & 3;
+    // The weights are constants, x and Y are not: in a chain of launches (one decode step) this kernel may
+    // have been started before its predecessor finished (programmatic dependent launch), so the producer
+    // streams weights at once while everything that reads x or writes results waits here.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     // ---- once per CTA, while the first tiles are in flight: fragments and group sums of x.
     // Item = (group, tg): 16 values of x; the four tg lanes of an item are neighbours.
     const int items = p.G * 4;
@@ -483,7 +489,13 @@ int t1_launch(const CUtensorMap& tm_c, const CUtensorMap& tm_a, const CUtensorMa
   p.stages = t1_stages(p.G);
   const size_t smem = t1_fixed_smem(p.G) + (size_t)p.stages * GT_STAGE_BYTES;
   QB_CUDA(cudaFuncSetAttribute(lowbit_gemv_t1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  lowbit_gemv_t1_kernel<<<grid, GT_THREADS, smem, st>>>(tm_c, tm_a, tm_b, p);
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(GT_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  QB_CUDA(cudaLaunchKernelEx(&cfg, lowbit_gemv_t1_kernel, tm_c, tm_a, tm_b, p));
   return QBLORA_OK;
 }
 
@@ -523,6 +535,9 @@ __global__ void __launch_bounds__(256) x_prepare_kernel(const __nv_bfloat16* __r
   // the main kernel is launched as a programmatic dependent: it may start (set up, stream weights) now and
   // waits for this grid's completion only before it reads the fragments
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // In a chain of launches this grid may itself have started early: the previous launch may still read
+  // the fragment area (same workspace) and may still be producing x.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int idx = blockIdx.x * 256 + threadIdx.x;
   const int total = n_kc * GT_GROUPS * NTOK * 4;
   const bool in_range = idx < total;
@@ -592,6 +607,8 @@ lowbit_gemv_ko_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
   auto xfull = [&](uint32_t b) { return bars + 8u * (2 * STAGES + 2 + b); };
   auto xempty = [&](uint32_t b) { return bars + 8u * (2 * STAGES + 4 + b); };
 
+  // a successor launched as a programmatic dependent may start on every SM this grid has left
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
     if (blockIdx.x == 0) *p.status = 0;   // any give-up below is written at least a wait limit later
@@ -787,15 +804,20 @@ int ko_launch(const CUtensorMap& tm_c, const CUtensorMap& tm_a, const CUtensorMa
               uint8_t* xfrag, cudaStream_t st) {
   p.stages = ko_stages<NT>();
   const int items = p.n_kc * GT_GROUPS * KoCfg<NT>::NTOK * 4;
-  x_prepare_kernel<NT><<<(items + 255) / 256, 256, 0, st>>>(p.X, p.T, p.d_in, p.G, p.n_kc, xfrag);
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  {
+    cudaLaunchConfig_t pc{};
+    pc.gridDim = dim3((unsigned)((items + 255) / 256)); pc.blockDim = dim3(256); pc.dynamicSmemBytes = 0; pc.stream = st;
+    pc.attrs = attr; pc.numAttrs = 1;
+    QB_CUDA(cudaLaunchKernelEx(&pc, x_prepare_kernel<NT>, p.X, p.T, p.d_in, p.G, p.n_kc, xfrag));
+  }
   count_launch();
   const size_t smem = KoCfg<NT>::FIXED + (size_t)p.stages * GT_STAGE_BYTES;
   QB_CUDA(cudaFuncSetAttribute(lowbit_gemv_ko_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(GT_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = 1;
   const uint8_t* xf = xfrag;
   QB_CUDA(cudaLaunchKernelEx(&cfg, lowbit_gemv_ko_kernel<NT>, tm_c, tm_a, tm_b, p, xf));
@@ -810,7 +832,8 @@ bool gemv_supported(const QwView& qw, int64_t T) {
 }
 
 constexpr int T1_TAIL_MAX_BLOCKS = 128, T1_TAIL_MAX_SPLIT = 4;   // row blocks in a split tail, parts each
-constexpr size_t T1_TAIL_BYTES = (size_t)T1_TAIL_MAX_BLOCKS * T1_TAIL_MAX_SPLIT * (GT_ROWS * 4 + 4);
+constexpr size_t T1_TAIL_HALF = (size_t)T1_TAIL_MAX_BLOCKS * T1_TAIL_MAX_SPLIT * (GT_ROWS * 4 + 4);
+constexpr size_t T1_TAIL_BYTES = 2 * T1_TAIL_HALF;   // two areas, used by alternate launches (launches of a chain may overlap)
 
 size_t gemv_ws_bytes(const QwView& qw, int64_t T) {
   // status word, then either the token fragments of the K-outer kernel (one K tile after the other)
@@ -859,8 +882,9 @@ int launch_lowbit_gemv(const QwView& qw, const __nv_bfloat16* X, int64_t T, void
       if (whole == 0) grid = rem * split;
       uint32_t e = launches.fetch_add(1) + 1;
       p.epoch = e == 0 ? launches.fetch_add(1) + 1 : e;
-      p.tail_partial = reinterpret_cast<float*>(xfrag);
-      p.tail_flags = reinterpret_cast<uint32_t*>(xfrag + (size_t)T1_TAIL_MAX_BLOCKS * T1_TAIL_MAX_SPLIT * GT_ROWS * 4);
+      uint8_t* area = xfrag + (p.epoch & 1u) * T1_TAIL_HALF;
+      p.tail_partial = reinterpret_cast<float*>(area);
+      p.tail_flags = reinterpret_cast<uint32_t*>(area + (size_t)T1_TAIL_MAX_BLOCKS * T1_TAIL_MAX_SPLIT * GT_ROWS * 4);
     }
   }
   {
