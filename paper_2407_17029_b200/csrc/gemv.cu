@@ -55,11 +55,11 @@ struct GvConst {
     asm volatile("" : "+r"(m0), "+r"(m1), "+r"(c));
   }
 };
-// ---- fp16 variants (shared-memory token operand only) --------------------------------------------
+// Word of 8 codes -> four fp16 pairs for the A fragments (k.m0 = 0x000F000F, k.m1 = 0x00F000F0,
+// k.c = 0x64006400 = fp16 1024.0 twice).
 // With a 10-bit mantissa two neighbouring nibbles fit below the magic exponent, so a word needs one
 // shift instead of three: v[0], v[2] = 1024 + c for codes (0,4), (2,6); v[1], v[3] = 1024 + 16 c for
 // codes (1,5), (3,7).  The token operand carries 1/16 at the odd positions to match.
-// (k.m0 = 0x000F000F, k.m1 = 0x00F000F0, k.c = 0x64006400)
 __device__ __forceinline__ void gv_unpack_h(uint32_t w, uint32_t (&v)[4], const GvConst& k) {
   const uint32_t t = w >> 8;
   v[0] = gv_and_or(w, k.m0, k.c);
