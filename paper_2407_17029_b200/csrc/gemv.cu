@@ -18,8 +18,8 @@
 // needs one shift only; odd nibbles come out as 1024 + 16 c and the token operand carries 1/16 at
 // those positions.  The order of the k index inside an MMA is free as long as both operands agree,
 // so nibble pairs (e, e + 4) are used as they fall out of the word and the token fragments are laid
-// out to match.  x (bf16) is converted to fp16 after a power-of-two prescale 2^-e (per call for one
-// token, per 64-value slice otherwise).  With P = sum of the fragment values and R = sum of the
+// out to match.  x (bf16) is converted to fp16 after a power-of-two prescale 2^-e of its own for
+// every 64-value slice (group, token).  With P = sum of the fragment values and R = sum of the
 // scaled x over a group, the group contributes  2^e (alpha (acc - 1024 P) + beta R).
 //
 // Two kernels: one token (fragments of x resident in shared memory, row blocks outer) and 2..16
@@ -212,9 +212,9 @@ struct T1Walk {
 };
 
 // ---------------------------------------------------------------------------------------------------
-// One token.  x is converted once per CTA into fp16 fragments in shared memory (with ONE power-of-two
-// prescale 2^-e for the call, undone on the output), the row blocks are the outer loop and only
-// column 0 of the accumulator tile is kept.
+// One token.  x is converted once per CTA into fp16 fragments in shared memory (each group of 64 values
+// with its own power-of-two prescale), the row blocks are the outer loop and only column 0 of the
+// accumulator tile is kept.
 constexpr int T1_RED_BYTES = GT_WARPS * GT_ROWS * 4;        // [16 warps][32 rows]
 constexpr int T1_MAX_STAGES = 10;
 
@@ -234,11 +234,12 @@ lowbit_gemv_t1_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
   auto empty = [&](int s) { return bars + 8u * (STAGES + s); };
   const uint32_t red_done = bars + 8u * (2 * STAGES);       // all 16 warps have written their sums of the row block
   const uint32_t red_free = bars + 8u * (2 * STAGES + 1);   // the summing warp has read them
-  // ss[G] = (1024 * sum of the fp16 fragment values, sum of the scaled x) per group, then
+  // ss[G] = (1024 P 2^e, R 2^e, 2^e, -) per group (P = sum of the fp16 fragment values, R = sum of the
+  // scaled x, 2^-e the group's prescale), then
   // xs[G][4 tg][8 words] = fp16 fragments, then 128 zero bytes
   const uint32_t ss_off = bar_off + 256;
   float* ss = reinterpret_cast<float*>(gbase + ss_off);
-  const uint32_t xs_off = ss_off + (uint32_t)p.G * 8;
+  const uint32_t xs_off = ss_off + (uint32_t)p.G * 16;
   uint4* xs = reinterpret_cast<uint4*>(gbase + xs_off);
   const uint32_t zero_off = xs_off + (uint32_t)p.G * 128;
 
@@ -288,68 +289,49 @@ lowbit_gemv_t1_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
     // streams weights at once while everything that reads x or writes results waits here.
     asm volatile("griddepcontrol.wait;" ::: "memory");
     // ---- once per CTA, while the first tiles are in flight: fragments and group sums of x.
-    // Item = (group, tg): 16 values of x; the four tg lanes of an item are neighbours.
+    // Item = (group, tg): 16 values of x; the four tg lanes of an item are neighbours.  Every group's
+    // 64 values get their own power-of-two prescale 2^-e (max |x| 2^-e in [2^14, 2^15)), so no pass over
+    // all of x and no CTA-wide reduction is needed first.
     const int items = p.G * 4;
-    const bool one_round = items <= GT_WARPS * 32;
-    uint4 c0, c1;     // this thread's item of the first round (x is read from global once when one round covers it)
-    {
-      const int q = tid < items ? tid : 0;
-      const uint4* src = reinterpret_cast<const uint4*>(p.X + q * 16);
-      c0 = __ldg(src); c1 = __ldg(src + 1);
-    }
-    float am = 0.0f;
-    if (one_round) {
-      am = gv_absmax8(c1, gv_absmax8(c0, am));
-    } else {
-      const uint4* xv = reinterpret_cast<const uint4*>(p.X);
-      for (int i = tid; i < (p.d_in >> 3); i += GT_WARPS * 32) am = gv_absmax8(__ldg(xv + i), am);
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) am = fmaxf(am, __shfl_xor_sync(0xFFFFFFFFu, am, o));
-    if (lane == 0) red[warp] = am;
-    asm volatile("bar.sync 1, 512;" ::: "memory");
-    am = red[0];
-#pragma unroll
-    for (int i = 1; i < GT_WARPS; ++i) am = fmaxf(am, red[i]);
-    int e = (int)((__float_as_uint(am) >> 23) & 0xFFu) - 127 - 14;   // max |x| * 2^-e in [2^14, 2^15)
-    e = e < -100 ? -100 : (e > 120 ? 120 : e);
-    const float y_scale = __uint_as_float((uint32_t)(127 + e) << 23);
-    asm volatile("bar.sync 1, 512;" ::: "memory");   // red is free again
     if (tid < 32) reinterpret_cast<uint32_t*>(gbase + zero_off)[tid] = 0u;
-    {
+    for (int i0 = 0; i0 < items; i0 += GT_WARPS * 32) {
+      const int idx = i0 + tid;
+      const bool live = idx < items;
+      const int q = live ? idx : 0;
+      const uint4* src = reinterpret_cast<const uint4*>(p.X + q * 16);
+      const uint4 x0 = __ldg(src), x1 = __ldg(src + 1);
+      float am = gv_absmax8(x1, gv_absmax8(x0, 0.0f));
+      am = fmaxf(am, __shfl_xor_sync(0xFFFFFFFFu, am, 1));
+      am = fmaxf(am, __shfl_xor_sync(0xFFFFFFFFu, am, 2));
+      int e = (int)((__float_as_uint(am) >> 23) & 0xFFu) - 127 - 14;
+      e = e < -100 ? -100 : (e > 120 ? 120 : e);
+      const float up = __uint_as_float((uint32_t)(127 + e) << 23);
       const float in_scale = __uint_as_float((uint32_t)(127 - e) << 23), in_scale16 = in_scale * 0.0625f;
-      for (int i0 = 0; i0 < items; i0 += GT_WARPS * 32) {
-        const int idx = i0 + tid;
-        const bool live = idx < items;
-        const int q = live ? idx : 0;
-        const uint4* src = reinterpret_cast<const uint4*>(p.X + q * 16);
-        const uint4 x0 = i0 == 0 ? c0 : __ldg(src), x1 = i0 == 0 ? c1 : __ldg(src + 1);
-        const uint32_t xw[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
-        uint32_t f[8];
-        float ps = 0.0f, rs = 0.0f;   // sum of fragment values; sum of scaled x as the fragments hold it
+      const uint32_t xw[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+      uint32_t f[8];
+      float ps = 0.0f, rs = 0.0f;   // sum of fragment values; sum of scaled x as the fragments hold it
 #pragma unroll
-        for (int wd = 0; wd < 2; ++wd)
+      for (int wd = 0; wd < 2; ++wd)
 #pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            // word wd holds x at positions 0..7 as pairs (2j, 2j+1) in xw[4 wd + j]; fragment register
-            // 2 (2 wd + h) pairs positions (2h, 2h+4), the next one (2h+1, 2h+5) scaled by 1/16
-            const uint32_t wa = xw[4 * wd + h], wb = xw[4 * wd + h + 2];
-            const uint32_t ev = gv_pack_h2(__uint_as_float(wa << 16) * in_scale, __uint_as_float(wb << 16) * in_scale);
-            const uint32_t od = gv_pack_h2(__uint_as_float(wa & 0xFFFF0000u) * in_scale16,
-                                           __uint_as_float(wb & 0xFFFF0000u) * in_scale16);
-            f[2 * (2 * wd + h)] = ev;
-            f[2 * (2 * wd + h) + 1] = od;
-            const float se = gv_h_lo(ev) + gv_h_hi(ev), so = gv_h_lo(od) + gv_h_hi(od);
-            ps += se + so;
-            rs += se + 16.0f * so;
-          }
-        ps += __shfl_xor_sync(0xFFFFFFFFu, ps, 1); rs += __shfl_xor_sync(0xFFFFFFFFu, rs, 1);
-        ps += __shfl_xor_sync(0xFFFFFFFFu, ps, 2); rs += __shfl_xor_sync(0xFFFFFFFFu, rs, 2);
-        if (live) {
-          if ((q & 3) == 0) *reinterpret_cast<float2*>(ss + (q >> 2) * 2) = make_float2(1024.0f * ps, rs);
-          xs[q * 2] = make_uint4(f[0], f[1], f[2], f[3]);
-          xs[q * 2 + 1] = make_uint4(f[4], f[5], f[6], f[7]);
+        for (int h = 0; h < 2; ++h) {
+          // word wd holds x at positions 0..7 as pairs (2j, 2j+1) in xw[4 wd + j]; fragment register
+          // 2 (2 wd + h) pairs positions (2h, 2h+4), the next one (2h+1, 2h+5) scaled by 1/16
+          const uint32_t wa = xw[4 * wd + h], wb = xw[4 * wd + h + 2];
+          const uint32_t ev = gv_pack_h2(__uint_as_float(wa << 16) * in_scale, __uint_as_float(wb << 16) * in_scale);
+          const uint32_t od = gv_pack_h2(__uint_as_float(wa & 0xFFFF0000u) * in_scale16,
+                                         __uint_as_float(wb & 0xFFFF0000u) * in_scale16);
+          f[2 * (2 * wd + h)] = ev;
+          f[2 * (2 * wd + h) + 1] = od;
+          const float se = gv_h_lo(ev) + gv_h_hi(ev), so = gv_h_lo(od) + gv_h_hi(od);
+          ps += se + so;
+          rs += se + 16.0f * so;
         }
+      ps += __shfl_xor_sync(0xFFFFFFFFu, ps, 1); rs += __shfl_xor_sync(0xFFFFFFFFu, rs, 1);
+      ps += __shfl_xor_sync(0xFFFFFFFFu, ps, 2); rs += __shfl_xor_sync(0xFFFFFFFFu, rs, 2);
+      if (live) {
+        if ((q & 3) == 0) *reinterpret_cast<float4*>(ss + (q >> 2) * 4) = make_float4(1024.0f * ps * up, rs * up, up, 0.0f);
+        xs[q * 2] = make_uint4(f[0], f[1], f[2], f[3]);
+        xs[q * 2 + 1] = make_uint4(f[4], f[5], f[6], f[7]);
       }
     }
     asm volatile("bar.sync 1, 512;" ::: "memory");
@@ -385,7 +367,7 @@ lowbit_gemv_t1_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
           if (grp < p.G) {                                   // warp-uniform
             const uint32_t sb = base + (uint32_t)s * GT_STAGE_BYTES;
             const uint32_t ca = sb + code_off, sa = sb + scale_off;
-            const float2 sg = gv_ldsf2<0>(ss_addr + (uint32_t)grp * 8u);      // (1024 P, R) of the group
+            const float4 sg = gv_ldsf4<0>(ss_addr + (uint32_t)grp * 16u);     // (1024 P 2^e, R 2^e, 2^e, -) of the group
             const uint32_t xa = xs_addr + (uint32_t)grp * xs_stride;
             const uint4 x0 = gv_lds4<0>(xa), x1 = gv_lds4<16>(xa);
             // all shared-memory loads of the group first (they stay in program order), then the math
@@ -405,9 +387,9 @@ lowbit_gemv_t1_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
               gv_mma_h(acc, va[0][2], vb[0][2], va[0][3], vb[0][3], x0.z, x0.w);
               gv_mma_h(acc, va[1][0], vb[1][0], va[1][1], vb[1][1], x1.x, x1.y);
               gv_mma_h(acc, va[1][2], vb[1][2], va[1][3], vb[1][3], x1.z, x1.w);
-              // alpha (acc - 1024 P) + beta R; column 0 of the accumulator tile is held by the tg == 0 lanes
-              y[mt][0] = fmaf(a0[mt], acc[0] - sg.x, fmaf(b0[mt], sg.y, y[mt][0]));
-              y[mt][1] = fmaf(a1[mt], acc[2] - sg.x, fmaf(b1[mt], sg.y, y[mt][1]));
+              // alpha (2^e acc - 1024 P 2^e) + beta R 2^e; column 0 of the accumulator tile is held by the tg == 0 lanes
+              y[mt][0] = fmaf(a0[mt], fmaf(acc[0], sg.z, -sg.x), fmaf(b0[mt], sg.y, y[mt][0]));
+              y[mt][1] = fmaf(a1[mt], fmaf(acc[2], sg.z, -sg.x), fmaf(b1[mt], sg.y, y[mt][1]));
             }
           }
           __syncwarp();
@@ -460,7 +442,6 @@ lowbit_gemv_t1_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
             a += __ldcg(p.tail_partial + (slot + part) * GT_ROWS + lane);
           }
         }
-        a *= y_scale;
         const int o = rb * GT_ROWS + lane;                // lane = row of the block
         if (o < p.d_out) {
           if (p.y_dtype == QBLORA_BF16) reinterpret_cast<__nv_bfloat16*>(p.Y)[o] = __float2bfloat16_rn(a);
@@ -477,7 +458,7 @@ lowbit_gemv_t1_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
 constexpr size_t GT_SMEM_MAX = 227 * 1024;
 // dynamic shared memory besides the stage ring: alignment slack, reduction buffer, barriers, group
 // sums, fragments, zero block
-size_t t1_fixed_smem(int G) { return 1024 + T1_RED_BYTES + 256 + (size_t)G * 8 + (size_t)G * 128 + 128; }
+size_t t1_fixed_smem(int G) { return 1024 + T1_RED_BYTES + 256 + (size_t)G * 16 + (size_t)G * 128 + 128; }
 int t1_stages(int G) {   // ring depth that fits; 0 if fewer than six stages would be left
   const size_t fixed = t1_fixed_smem(G);
   if (fixed + 6 * (size_t)GT_STAGE_BYTES > GT_SMEM_MAX) return 0;
