@@ -438,12 +438,13 @@ def lowbit_extras(qb, torch, dev, peaks, l2_bytes, shapes=("q", "up"), tokens=(1
             e.record(); torch.cuda.synchronize()
             call_us = s.elapsed_time(e) / reps * 1e3
             single_us = statistics.mean(a.elapsed_time(b) for a, b in evs) * 1e3
-            # chain time: 2 * ncopies launches over the rotating copies replayed as one CUDA graph, the way a
+            # chain time: >= 64 launches over the rotating copies replayed as one CUDA graph, the way a
             # decode step issues its products back to back; per-launch time = graph time / launches.  An
             # event pair around ONE launch also counts about 6 us of launch latency that a chain hides.
             side = torch.cuda.Stream()
             side.wait_stream(torch.cuda.current_stream())
-            n_chain = 2 * ncopies
+            n_chain = ncopies * max(2, -(-64 // ncopies))      # >= 64 launches: a decode step issues hundreds;
+                                                                # the graph's own launch cost is spread over them
             with torch.cuda.stream(side):
                 qb.lowbit_gemm(copies[0], Xt, ws=ws, out=Y)
             side.synchronize()
