@@ -338,6 +338,8 @@ def run_gpu(args, wl, geom):
                          "achieved": dom_flops / (dom_ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops_sustained"],
                          "peak_kind": f"bf16 dense, sustained, {peaks['source']}", "unit": "TFLOP/s",
                          "frac": dom_flops / (dom_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+                         "peak_burst": peaks["bf16_tflops"],
+                         "frac_of_burst": dom_flops / (dom_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
                          "traffic": MEASURED_DRAM_TRAFFIC.get((wl.name, geom.name)), "ms_per_launch": dom_ms},
             "step_flops": flops_step,
             "eager": {"ms_per_step": eager_ms / args.steps, "value": flops_step * args.steps / (eager_ms * 1e-3) / 1e12,
