@@ -274,3 +274,13 @@ def test_lowbit_one_token_split_tail(qb, d_out):
         for _ in range(2):
             gate_strict(to_np64(qb.lowbit_gemm(dq, Xd, torch.float32, ws=ws)), ref, f"lowbit split tail d_out={d_out}")
             assert qb.device_status(ws) == qb.OK
+
+
+@pytest.mark.parametrize("T", [1, 2, 16])
+@pytest.mark.parametrize("d_out,d_in", [(8, 256), (40, 512), (33 * 8, 256)])
+def test_lowbit_decode_tiny_shapes(qb, T, d_out, d_in):
+    # fewer output rows than one 32-row tile, a single K tile with unused groups, ragged row blocks
+    qw, _, X, _ = make_case(62, T, d_out, d_in, 64, 8, 8, qfmt=1)
+    ref = oracle.lowbit_gemm(qw, X)
+    dq, Xd = qweight_to_dev(qw), to_bf16_dev(X)
+    gate_strict(to_np64(qb.lowbit_gemm(dq, Xd, torch.float32)), ref, f"lowbit tiny {d_out}x{d_in} T={T}")
