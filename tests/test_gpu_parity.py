@@ -284,3 +284,26 @@ def test_lowbit_decode_tiny_shapes(qb, T, d_out, d_in):
     ref = oracle.lowbit_gemm(qw, X)
     dq, Xd = qweight_to_dev(qw), to_bf16_dev(X)
     gate_strict(to_np64(qb.lowbit_gemm(dq, Xd, torch.float32)), ref, f"lowbit tiny {d_out}x{d_in} T={T}")
+
+
+@pytest.mark.parametrize("bi,bo", [(8, 8), (4, 8), (8, 1), (4, 2)])
+@pytest.mark.parametrize("visible", [False, True])
+def test_two_dimensional_blocks_fwd_bwd(qb, path, bi, bo, visible):
+    # Sec. 3.3's native quantization blocks (lambda_1 x lambda_2 = 8 x 8, 4 x 8) in the min-max format, adapter
+    # windows equal to the block (so the adapter stays mergeable); several tiles, ragged in every dimension.
+    T, d_out, d_in = 300, 328, 448
+    qw, ad, X, dY = make_case(63, T, d_out, d_in, bi, 8, 24, qfmt=1, bi=bi, bo=bo)
+    Wt = oracle.dequantize(qw)
+    if visible:
+        ad.scaling = visible_scaling(Wt, ad, X)
+    dq, da, Xd, dYd = qweight_to_dev(qw), adapter_to_dev(ad), to_bf16_dev(X), to_bf16_dev(dY)
+    gate_strict(to_np64(qb.linear_fwd(dq, da, Xd, torch.float32)), oracle.linear_fwd(Wt, ad, X), f"Y blocks {bi}x{bo}")
+    rdX, rdA, rdB = oracle.linear_bwd(Wt, ad, X, dY)
+    dX, dA, dB = qb.linear_bwd(dq, da, Xd, dYd, torch.float32)
+    gate_strict(to_np64(dX), rdX, f"dX blocks {bi}x{bo}")
+    gate_strict(to_np64(dA), rdA, "dA", per_row=False)
+    gate_strict(to_np64(dB), rdB, "dB", per_row=False)
+    # prefill-shaped low-bit product on the merged weight equals the unmerged forward (merge identity)
+    if 8 % bo == 0:
+        merged = qb.merge(dq, da)
+        gate_strict(to_np64(qb.lowbit_gemm(merged, Xd, torch.float32)), oracle.linear_fwd(Wt, ad, X), f"merged blocks {bi}x{bo}")
