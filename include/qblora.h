@@ -59,7 +59,8 @@ typedef enum {
   QBLORA_OP_LINEAR_FWD = 1,
   QBLORA_OP_LINEAR_BWD = 2,
   QBLORA_OP_MERGE = 3,
-  QBLORA_OP_LOWBIT_GEMM = 4
+  QBLORA_OP_LOWBIT_GEMM = 4,
+  QBLORA_OP_MERGE_DENSE = 5
 } qblora_op;
 
 /* Frozen block-wise 4-bit weight: the triplet (w^, alpha, beta) of Eq. 1 / Sec. 3.3. */
@@ -176,6 +177,19 @@ int qblora_linear_bwd(const qblora_qweight* qw, const qblora_adapter* adapter, c
  */
 int qablora_merge(const qblora_qweight* qw, const qblora_adapter* adapter, float* beta_out,
                   void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Dense 16-bit merge (Sec. 3.1 / 3.2: after fine-tuning the adapter is folded back into a full weight
+ * with no inference overhead; Algorithm 1's dense-update routine read as
+ * dW[o][i] = (A B)[i / lambda_in][o / lambda_out] / lambda_in):
+ *   W_out[o][i] = alpha * level[code] + beta  +  s * dW[o][i]   (A B in fp64, the sum in fp32, then bf16).
+ *   W_out DEVICE out bf16 [d_out][d_in] (16-byte aligned, d_in % 8 == 0).  Either format, any block
+ *   shape, any (lambda_in, lambda_out).  adapter may be NULL (plain dequantization) and may be the
+ *   single matrix H (B == NULL).  The merged weight is then served by any plain bf16 GEMM.
+ *   ws: qblora_workspace_bytes(QBLORA_OP_MERGE_DENSE, ...) bytes.
+ */
+int qblora_merge_dense(const qblora_qweight* qw, const qblora_adapter* adapter, void* W_out, void* ws,
+                       size_t ws_bytes, void* stream);
 
 /*
  * The same merge for callers that cannot give the library a workspace.  (The paper has no

@@ -23,12 +23,12 @@ LIB_PATH = os.path.join(_HERE, "libqblora.so")
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_TOO_LARGE = range(7)
 FMT_CODEBOOK_ABSMAX, FMT_AFFINE_MINMAX = 0, 1
 F32, BF16 = 0, 1
-OP_QUANTIZE, OP_LINEAR_FWD, OP_LINEAR_BWD, OP_MERGE, OP_LOWBIT_GEMM = range(5)
+OP_QUANTIZE, OP_LINEAR_FWD, OP_LINEAR_BWD, OP_MERGE, OP_LOWBIT_GEMM, OP_MERGE_DENSE = range(6)
 
 EXPORTS = ["qblora_default_code_table", "qblora_workspace_bytes", "qblora_status_string",
            "qblora_device_status", "qblora_quantize_blockwise", "qblora_linear_fwd",
            "qblora_linear_bwd", "qablora_merge", "qablora_lowbit_gemm", "qblora_kernel_launches",
-           "qblora_set_timing_events", "qablora_merge_noalloc"]
+           "qblora_set_timing_events", "qablora_merge_noalloc", "qblora_merge_dense"]
 
 
 class _CQWeight(ctypes.Structure):
@@ -70,6 +70,9 @@ _lib.qablora_lowbit_gemm.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_
 
 
 _lib.qablora_merge_noalloc.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+_lib.qblora_merge_dense.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                    ctypes.c_size_t, ctypes.c_void_p]
+_lib.qblora_merge_dense.restype = ctypes.c_int
 _lib.qblora_kernel_launches.restype = ctypes.c_uint64
 _lib.qblora_kernel_launches.argtypes = []
 _lib.qblora_set_timing_events.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
@@ -265,6 +268,20 @@ def merge(qw: QWeight, ad: Adapter, in_place: bool = False, ws: Optional[torch.T
                             ws.numel(), _stream_ptr(stream))
     _check(st, "qablora_merge")
     return QWeight(qw.d_out, qw.d_in, qw.block_in, qw.block_out, qw.qfmt, qw.code, qw.codes, qw.alpha, beta_out)
+
+
+def merge_dense(qw: QWeight, ad: Optional[Adapter], out: Optional[torch.Tensor] = None,
+                ws: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Dense 16-bit merge: bf16 [d_out][d_in] = dequantized weight + s * dense adapter update."""
+    W = out if out is not None else torch.empty((qw.d_out, qw.d_in), dtype=torch.bfloat16, device=qw.codes.device)
+    if ws is None:
+        ws = alloc_workspace(OP_MERGE_DENSE, qw, ad, 0)
+    cq = qw.c_struct()
+    ca = ad.c_struct() if ad is not None else None
+    st = _lib.qblora_merge_dense(ctypes.byref(cq), _ref(ca), W.data_ptr(), ws.data_ptr(), ws.numel(),
+                                 _stream_ptr(stream))
+    _check(st, "qblora_merge_dense")
+    return W
 
 
 def merge_noalloc(qw: QWeight, ad: Adapter, beta_out: torch.Tensor, stream=None) -> QWeight:

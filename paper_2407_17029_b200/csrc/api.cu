@@ -104,6 +104,7 @@ size_t ws_bytes_impl(int op, const QwView& q, const AdView* ad, int64_t T) {
       if (!force_general() && tc_supported(q, ad, T)) return tc_ws_bytes(op, q, ad, T);
       return simt_ws_bytes(op, q, ad, T);
     case QBLORA_OP_MERGE: return ad ? merge_ws_bytes(q, *ad) : 0;
+    case QBLORA_OP_MERGE_DENSE: return merge_dense_ws_bytes(q, ad);
     case QBLORA_OP_LOWBIT_GEMM:
       if (gemv_supported(q, T)) return gemv_ws_bytes(q, T);
       if (!force_general() && tc_supported(q, nullptr, T)) return tc_ws_bytes(QBLORA_OP_LINEAR_FWD, q, nullptr, T);
@@ -149,7 +150,7 @@ size_t qblora_workspace_bytes(int op, const qblora_qweight* qw, const qblora_ada
     if (make_ad(adapter, q, false, &ad) != QBLORA_OK) return 0;
     adp = &ad;
   }
-  if (op != QBLORA_OP_MERGE && op != QBLORA_OP_QUANTIZE && tokens < 1) return 0;
+  if (op != QBLORA_OP_MERGE && op != QBLORA_OP_MERGE_DENSE && op != QBLORA_OP_QUANTIZE && tokens < 1) return 0;
   if (adp && !adapter->B && (op == QBLORA_OP_LINEAR_FWD || op == QBLORA_OP_LINEAR_BWD))
     return ws_bytes_single(op, q, ad, tokens);
   return ws_bytes_impl(op, q, adp, tokens);
@@ -269,6 +270,26 @@ int qablora_merge(const qblora_qweight* qw, const qblora_adapter* adapter, float
   rc = reset_status(ws, st);
   if (rc) return rc;
   return launch_merge(q, ad, adapter->B == nullptr, beta_out, static_cast<char*>(ws), st);
+}
+
+int qblora_merge_dense(const qblora_qweight* qw, const qblora_adapter* adapter, void* W_out, void* ws,
+                       size_t ws_bytes, void* stream) {
+  QwView q; int rc = make_qw(qw, &q);
+  if (rc) return rc;
+  if (!W_out || !aligned16(W_out) || q.d_in % 8) return QBLORA_ERR_INVALID_ARG;
+  AdView ad; const AdView* adp = nullptr;
+  if (adapter) {
+    rc = make_ad(adapter, q, true, &ad);
+    if (rc) return rc;
+    adp = &ad;
+  }
+  const size_t need = merge_dense_ws_bytes(q, adp);
+  if (!ws || !aligned16(ws) || ws_bytes < need) return QBLORA_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  rc = reset_status(ws, st);
+  if (rc) return rc;
+  return launch_merge_dense(q, adp, adapter && adapter->B == nullptr, static_cast<__nv_bfloat16*>(W_out),
+                            static_cast<char*>(ws), st);
 }
 
 int qablora_merge_noalloc(const qblora_qweight* qw, const qblora_adapter* adapter, float* beta_out,

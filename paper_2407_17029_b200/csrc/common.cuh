@@ -65,6 +65,8 @@ int launch_merge_noalloc(const QwView& qw, const AdView& ad, bool single_matrix,
                          cudaStream_t st);
 
 // Bandwidth-bound low-bit product for small token counts (block_out == 1, block_in == 64).
+size_t merge_dense_ws_bytes(const QwView& qw, const AdView* ad);
+int launch_merge_dense(const QwView& qw, const AdView* ad, bool single_matrix, __nv_bfloat16* W, char* ws, cudaStream_t st);
 int launch_identity(__nv_bfloat16* out, int n, cudaStream_t st);   // bf16 identity [n][n]
 bool gemv_supported(const QwView& qw, int64_t T);
 size_t gemv_ws_bytes(const QwView& qw, int64_t T);   // status word + (T > 1) token fragments

@@ -307,3 +307,23 @@ def test_two_dimensional_blocks_fwd_bwd(qb, path, bi, bo, visible):
     if 8 % bo == 0:
         merged = qb.merge(dq, da)
         gate_strict(to_np64(qb.lowbit_gemm(merged, Xd, torch.float32)), oracle.linear_fwd(Wt, ad, X), f"merged blocks {bi}x{bo}")
+
+
+@pytest.mark.parametrize("case", [(320, 448, 64, 8, 48, 0, 64, 1), (136, 192, 4, 4, 16, 1, 64, 1), (128, 512, 8, 8, 0, 1, 8, 8)])
+def test_dense_16bit_merge(qb, case):
+    # W' = dequantized weight + s * dense adapter update (Sec. 3.1 / 3.2), rounded once to bf16; rank 0 = single
+    # matrix H.  Then "zero inference overhead": X W'^T equals the adapted forward.
+    d_out, d_in, l1, l2, r, qfmt, bi, bo = case
+    qw, ad, X, _ = make_case(64, 96, d_out, d_in, l1, l2, max(r, 8), qfmt=qfmt, bi=bi, bo=bo)
+    if r == 0:
+        ad = oracle.Adapter(l1, l2, 0, 1.0, synth.round_to_bf16(synth.normal(64, "H", (d_in // l1, d_out // l2), 0.02)), None)
+    Wt = oracle.dequantize(qw)
+    ad.scaling = visible_scaling(Wt, ad, X)
+    ref = Wt + ad.scaling * oracle.dense_delta_w(d_out, d_in, ad)
+    dq, da = qweight_to_dev(qw), adapter_to_dev(ad)
+    got = to_np64(qb.merge_dense(dq, da))
+    assert np.all(np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref) + 1e-30)          # one bf16 rounding
+    base = to_np64(qb.merge_dense(dq, None))
+    assert np.all(np.abs(base - Wt) <= 2.0 ** -8 * np.abs(Wt) + 1e-30)
+    Y = torch.matmul(to_bf16_dev(X).float(), qb.merge_dense(dq, da).float().t())
+    gate_strict(to_np64(Y), oracle.linear_fwd(Wt, ad, X), "X W'^T vs adapted forward")
