@@ -26,6 +26,11 @@ _LIB = os.path.join(_HERE, "liboracle.so")
 FMT_CODEBOOK_ABSMAX = 0
 FMT_AFFINE_MINMAX = 1
 
+# parameter-free operator pair around the adapter (Sec. 3.2; alternatives from the Sec. 4 ablation)
+OP_AVGPOOL_REPEAT = 0       # AvgPool & repeat_interleave (the method's own)
+OP_TRUNCATE_ZEROPAD = 1     # truncation & supplement_0
+OP_SAMPLE_ZEROFILL = 2      # interval_sampling & interpolation (zeros between the samples)
+
 
 def build(force: bool = False) -> str:
     """Compile the C oracle with gcc (OpenMP, no fast-math, no FMA contraction)."""
@@ -90,6 +95,7 @@ class Adapter:
     scaling: float
     A: np.ndarray                   # [d_in/lambda_in][rank]  (or H [P][Q] when B is None)
     B: Optional[np.ndarray]         # [rank][d_out/lambda_out]
+    scale_op: int = 0               # OP_AVGPOOL_REPEAT / OP_TRUNCATE_ZEROPAD / OP_SAMPLE_ZEROFILL
 
 
 def quantize_blockwise(W, block_in=64, block_out=1, qfmt=FMT_CODEBOOK_ABSMAX, code=None) -> QWeight:
@@ -122,10 +128,10 @@ def dequantize(qw: QWeight) -> np.ndarray:
 
 def _ad_args(ad: Optional[Adapter]):
     if ad is None:
-        return 0, 1, 1, 0, ctypes.c_double(0.0), None, None, None, None
+        return 0, 0, 1, 1, 0, ctypes.c_double(0.0), None, None, None, None
     A = _f32(ad.A)
     B = _f32(ad.B)
-    return (1, ad.lambda_in, ad.lambda_out, ad.rank, ctypes.c_double(float(ad.scaling)),
+    return (1, int(ad.scale_op), ad.lambda_in, ad.lambda_out, ad.rank, ctypes.c_double(float(ad.scaling)),
             _p(A, ctypes.c_float), _p(B, ctypes.c_float), A, B)
 
 
@@ -136,9 +142,9 @@ def linear_fwd(Wt: np.ndarray, ad: Optional[Adapter], X) -> np.ndarray:
     T, d_in = X.shape
     d_out = Wt.shape[0]
     Y = np.zeros((T, d_out), dtype=np.float64)
-    has, l1, l2, r, s, pA, pB, _A, _B = _ad_args(ad)
+    has, op, l1, l2, r, s, pA, pB, _A, _B = _ad_args(ad)
     rc = _L().orc_linear_fwd(_p(Wt, ctypes.c_double), d_out, d_in, _p(X, ctypes.c_float),
-                             ctypes.c_int64(T), has, l1, l2, r, s, pA, pB, _p(Y, ctypes.c_double))
+                             ctypes.c_int64(T), has, op, l1, l2, r, s, pA, pB, _p(Y, ctypes.c_double))
     _check(rc, "linear_fwd")
     return Y
 
@@ -152,7 +158,7 @@ def linear_bwd(Wt: Optional[np.ndarray], ad: Optional[Adapter], X, dY, d_out=Non
     d_out = dY.shape[1]
     if Wt is not None:
         Wt = np.ascontiguousarray(Wt, dtype=np.float64)
-    has, l1, l2, r, s, pA, pB, A, B = _ad_args(ad)
+    has, op, l1, l2, r, s, pA, pB, A, B = _ad_args(ad)
     dX = np.zeros((T, d_in), dtype=np.float64) if want_dx else None
     dA = dB = None
     if ad is not None:
@@ -161,7 +167,7 @@ def linear_bwd(Wt: Optional[np.ndarray], ad: Optional[Adapter], X, dY, d_out=Non
         if want_db and B is not None:
             dB = np.zeros(B.shape, dtype=np.float64)
     rc = _L().orc_linear_bwd(_p(Wt, ctypes.c_double), d_out, d_in, _p(X, ctypes.c_float),
-                             _p(dY, ctypes.c_float), ctypes.c_int64(T), has, l1, l2, r, s, pA, pB,
+                             _p(dY, ctypes.c_float), ctypes.c_int64(T), has, op, l1, l2, r, s, pA, pB,
                              _p(dX, ctypes.c_double), _p(dA, ctypes.c_double), _p(dB, ctypes.c_double))
     _check(rc, "linear_bwd")
     return dX, dA, dB
@@ -171,7 +177,7 @@ def dense_delta_w(d_out: int, d_in: int, ad: Adapter) -> np.ndarray:
     A = _f32(ad.A)
     B = _f32(ad.B)
     dW = np.zeros((d_out, d_in), dtype=np.float64)
-    rc = _L().orc_dense_delta_w(d_out, d_in, ad.lambda_in, ad.lambda_out, ad.rank,
+    rc = _L().orc_dense_delta_w(int(ad.scale_op), d_out, d_in, ad.lambda_in, ad.lambda_out, ad.rank,
                                 _p(A, ctypes.c_float), _p(B, ctypes.c_float), _p(dW, ctypes.c_double))
     _check(rc, "dense_delta_w")
     return dW
@@ -181,6 +187,8 @@ def merge(qw: QWeight, ad: Adapter) -> QWeight:
     """QA-BLoRA merge: returns a new QWeight with beta' (codes and alpha are the same arrays)."""
     if qw.qfmt != FMT_AFFINE_MINMAX:
         raise ValueError("oracle merge: needs the min-max format")
+    if ad.scale_op != OP_AVGPOOL_REPEAT:
+        raise ValueError("oracle merge: the update is constant per block only for AvgPool & repeat_interleave")
     A = _f32(ad.A)
     B = _f32(ad.B)
     beta_out = np.zeros_like(qw.beta)

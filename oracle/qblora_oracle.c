@@ -18,7 +18,9 @@
  * Pins (see tests/test_oracle_*.py): quantizer closed forms, round trip and
  * brute force; B = 0; lambda = 1 textbook LoRA; dense equivalent-weight
  * identity (Eq. 2 and the paragraph after it); finite differences and adjoint
- * identity for the backward pass; merge identity (Sec. 3.3).
+ * identity for the backward pass; merge identity (Sec. 3.3); for the alternative
+ * scale operators of the Sec. 4 ablation: slicing / zero-padding restatements,
+ * the dense equivalent update, untouched outputs and finite differences.
  * Parity unpinned: only two *conventions* -- the choice of the built-in 16-level
  * table (the paper cites NF4 without printing it) and which (lambda1, lambda2)
  * a benchmark config means.  Everything computed downstream of them is pinned.
@@ -173,15 +175,43 @@ int orc_dequantize(const uint8_t* codes, const float* alpha, const float* beta,
   return ORC_OK;
 }
 
-/* AvgPool(lambda1) over the feature axis (Sec. 3.2; written out before Eq. 2). */
-static void pool_rows(const float* X, int64_t T, int d_in, int l1, double* xp) {
+/*
+ * The parameter-free pair of operators around the adapter (Sec. 3.2; the
+ * alternatives are the ones listed in the Sec. 4 ablation on scale operators).
+ *   op 0  AvgPool & repeat_interleave:   x'[p] = mean of x[l1 p .. l1 p + l1 - 1];  y[o] += v[o / l2]
+ *   op 1  truncation & supplement_0:     x'[p] = x[p]      (front part kept);      y[o] += v[o] if o < Q, else 0
+ *   op 2  interval_sampling & interpolation: x'[p] = x[l1 p] (every l1-th value);  y[l2 q] += v[q], zeros between
+ * in_src / out_src give, for a full-size index, the compressed index it is tied
+ * to (or -1 for none); the tie's coefficient is 1 / in_divisor.
+ */
+static int in_src(int op, int i, int l1, int P) {
+  if (op == 0) return i / l1;
+  if (op == 1) return i < P ? i : -1;
+  return (i % l1 == 0) ? i / l1 : -1;
+}
+static double in_divisor(int op, int l1) { return op == 0 ? (double)l1 : 1.0; }
+static int out_src(int op, int o, int l2, int Q) {
+  if (op == 0) return o / l2;
+  if (op == 1) return o < Q ? o : -1;
+  return (o % l2 == 0) ? o / l2 : -1;
+}
+
+/* Input compression over the feature axis: x'[t][p] = sum_i c(p, i) X[t][i]. */
+static void compress_rows(int op, const float* X, int64_t T, int d_in, int l1, double* xp) {
   int P = d_in / l1;
 #pragma omp parallel for schedule(static)
   for (int64_t t = 0; t < T; ++t)
     for (int p = 0; p < P; ++p) {
       double s = 0.0;
-      for (int j = 0; j < l1; ++j) s += (double)X[t * d_in + (int64_t)p * l1 + j];
-      xp[t * P + p] = s / (double)l1;
+      if (op == 0) {
+        for (int j = 0; j < l1; ++j) s += (double)X[t * d_in + (int64_t)p * l1 + j];
+        s /= (double)l1;
+      } else if (op == 1) {
+        s = (double)X[t * d_in + p];
+      } else {
+        s = (double)X[t * d_in + (int64_t)p * l1];
+      }
+      xp[t * P + p] = s;
     }
 }
 
@@ -192,18 +222,19 @@ static void pool_rows(const float* X, int64_t T, int d_in, int l1, double* xp) {
  * The scaling s multiplies the adapter term only; repeat_interleave(lambda2)
  * is the index o / lambda2.  With B == NULL, A is the single matrix H of
  * Sec. 3.3 (shape [P][Q]) and v = x' H.  has_adapter == 0: base term only.
+ * op selects the compress / expand pair (0 = the method's own; see above).
  */
 int orc_linear_fwd(const double* Wt, int d_out, int d_in, const float* X,
-                   int64_t T, int has_adapter, int l1, int l2, int r, double s,
+                   int64_t T, int has_adapter, int op, int l1, int l2, int r, double s,
                    const float* A, const float* B, double* Y) {
   int P = 0, Q = 0;
   double *xp = NULL, *u = NULL, *v = NULL;
   if (has_adapter) {
-    if (d_in % l1 || d_out % l2) return ORC_BAD;
+    if (d_in % l1 || d_out % l2 || op < 0 || op > 2) return ORC_BAD;
     P = d_in / l1; Q = d_out / l2;
     xp = (double*)malloc(sizeof(double) * (size_t)T * P);
     v = (double*)calloc((size_t)T * Q, sizeof(double));
-    pool_rows(X, T, d_in, l1, xp);
+    compress_rows(op, X, T, d_in, l1, xp);
     if (B) {
       u = (double*)calloc((size_t)T * r, sizeof(double));
 #pragma omp parallel for schedule(static)
@@ -235,7 +266,10 @@ int orc_linear_fwd(const double* Wt, int d_out, int d_in, const float* X,
       double acc = 0.0;
       for (int i = 0; i < d_in; ++i)
         acc += (double)X[t * d_in + i] * Wt[(size_t)o * d_in + i];
-      if (has_adapter) acc += s * v[t * Q + o / l2];
+      if (has_adapter) {
+        int q = out_src(op, o, l2, Q);
+        if (q >= 0) acc += s * v[t * Q + q];
+      }
       Y[t * d_out + o] = acc;
     }
   free(xp); free(u); free(v);
@@ -248,29 +282,33 @@ int orc_linear_fwd(const double* Wt, int d_out, int d_in, const float* X,
  *   dv[t][q] = s * sum_{j<lambda2} dY[t][lambda2 q + j]
  *   du = dv B^T,  dB = u^T dv,  dx' = du A^T,  dA = x'^T du
  *   dX[t][i] = sum_o dY[t][o] w~[o][i] + dx'[t][i / lambda1] / lambda1
+ * (written for op 0; in general dv[t][q] = s * sum of dY[t][o] over the outputs
+ * o that the expansion ties to q, and dX[t][i] gets dx'[t][p] / in_divisor for
+ * the p that the compression ties i to).
  * Single-matrix mode (B == NULL): dA receives dH = x'^T dv and dx' = dv H^T.
  * Any of dX, dA, dB may be NULL (skipped).  Wt may be NULL when dX is NULL.
  */
 int orc_linear_bwd(const double* Wt, int d_out, int d_in, const float* X,
-                   const float* dY, int64_t T, int has_adapter, int l1, int l2,
+                   const float* dY, int64_t T, int has_adapter, int op, int l1, int l2,
                    int r, double s, const float* A, const float* B, double* dX,
                    double* dA, double* dB) {
   int P = 0, Q = 0;
   double *xp = NULL, *u = NULL, *dv = NULL, *du = NULL, *dxp = NULL;
   if (has_adapter) {
-    if (d_in % l1 || d_out % l2) return ORC_BAD;
+    if (d_in % l1 || d_out % l2 || op < 0 || op > 2) return ORC_BAD;
     P = d_in / l1; Q = d_out / l2;
     xp = (double*)malloc(sizeof(double) * (size_t)T * P);
-    dv = (double*)malloc(sizeof(double) * (size_t)T * Q);
+    dv = (double*)calloc((size_t)T * Q, sizeof(double));
     dxp = (double*)calloc((size_t)T * P, sizeof(double));
-    pool_rows(X, T, d_in, l1, xp);
+    compress_rows(op, X, T, d_in, l1, xp);
 #pragma omp parallel for schedule(static)
-    for (int64_t t = 0; t < T; ++t)
-      for (int q = 0; q < Q; ++q) {
-        double acc = 0.0;
-        for (int j = 0; j < l2; ++j) acc += (double)dY[t * d_out + (int64_t)q * l2 + j];
-        dv[t * Q + q] = s * acc;
+    for (int64_t t = 0; t < T; ++t) {
+      for (int o = 0; o < d_out; ++o) {
+        int q = out_src(op, o, l2, Q);
+        if (q >= 0) dv[t * Q + q] += (double)dY[t * d_out + o];
       }
+      for (int q = 0; q < Q; ++q) dv[t * Q + q] *= s;
+    }
     if (B) {
       u = (double*)malloc(sizeof(double) * (size_t)T * r);
       du = (double*)malloc(sizeof(double) * (size_t)T * r);
@@ -334,7 +372,10 @@ int orc_linear_bwd(const double* Wt, int d_out, int d_in, const float* X,
         double acc = 0.0;
         for (int o = 0; o < d_out; ++o)
           acc += (double)dY[t * d_out + o] * Wt[(size_t)o * d_in + i];
-        if (has_adapter) acc += dxp[t * P + i / l1] / (double)l1;
+        if (has_adapter) {
+          int p = in_src(op, i, l1, P);
+          if (p >= 0) acc += dxp[t * P + p] / in_divisor(op, l1);
+        }
         dX[t * d_in + i] = acc;
       }
   }
@@ -347,10 +388,13 @@ int orc_linear_bwd(const double* Wt, int d_out, int d_in, const float* X,
  *   dW[o][i] = (A B)[i / lambda1][o / lambda2] / lambda1
  * i.e. constant on every aligned (lambda1 x lambda2) tile; the 1/lambda1 comes
  * from the averaging (Eq. 2's condition w_in = lambda1 * w).  B == NULL: A is H.
+ * For the alternative operator pairs the update is H itself placed on the kept
+ * (op 1: leading P x Q corner) or sampled (op 2: every l1-th input, l2-th output)
+ * positions and zero elsewhere.
  */
-int orc_dense_delta_w(int d_out, int d_in, int l1, int l2, int r,
+int orc_dense_delta_w(int op, int d_out, int d_in, int l1, int l2, int r,
                       const float* A, const float* B, double* dW) {
-  if (d_in % l1 || d_out % l2) return ORC_BAD;
+  if (d_in % l1 || d_out % l2 || op < 0 || op > 2) return ORC_BAD;
   int P = d_in / l1, Q = d_out / l2;
   double* H = (double*)malloc(sizeof(double) * (size_t)P * Q);
   for (int p = 0; p < P; ++p)
@@ -362,7 +406,10 @@ int orc_dense_delta_w(int d_out, int d_in, int l1, int l2, int r,
     }
   for (int o = 0; o < d_out; ++o)
     for (int i = 0; i < d_in; ++i)
-      dW[(size_t)o * d_in + i] = H[(size_t)(i / l1) * Q + (o / l2)] / (double)l1;
+    {
+      int p = in_src(op, i, l1, P), q = out_src(op, o, l2, Q);
+      dW[(size_t)o * d_in + i] = (p >= 0 && q >= 0) ? H[(size_t)p * Q + q] / in_divisor(op, l1) : 0.0;
+    }
   free(H);
   return ORC_OK;
 }
@@ -403,7 +450,7 @@ int orc_lowbit_gemm(const uint8_t* codes, const float* alpha, const float* beta,
   double* Wt = (double*)malloc(sizeof(double) * (size_t)d_out * d_in);
   if (!Wt) return ORC_BAD;
   int rc = orc_dequantize(codes, alpha, beta, d_out, d_in, block_in, block_out, 1, NULL, Wt);
-  if (rc == ORC_OK) rc = orc_linear_fwd(Wt, d_out, d_in, X, T, 0, 1, 1, 0, 0.0, NULL, NULL, Y);
+  if (rc == ORC_OK) rc = orc_linear_fwd(Wt, d_out, d_in, X, T, 0, 0, 1, 1, 0, 0.0, NULL, NULL, Y);
   free(Wt);
   return rc;
 }
