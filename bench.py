@@ -35,6 +35,9 @@ METRIC = "fused 4-bit+BLoRA linear fwd+bwd TFLOP/s & low-bit GEMM GB/s, % of roo
 
 
 # ----------------------------------------------------------------------------------- accounting
+SCALE_OP = 0   # adapter operator pair of the run (--scale-op)
+
+
 def linear_flops(T, d_out, d_in, r, geom):
     """Algorithmic flops of one adapted linear, forward + backward: two base contractions
     (2*T*D_in*D_out each) and the adapter's (2*T*r*(P+Q) forward, twice that backward)."""
@@ -114,7 +117,7 @@ def oracle_step(wl, geom, sample_rows, cache):
     t0 = time.perf_counter()
     for spec in wl.linears:
         qw, Wt, li = cache[spec.name]
-        ad = oracle.Adapter(geom.lambda_in, geom.lambda_out, wl.rank, wl.scaling, li.A, li.B)
+        ad = oracle.Adapter(geom.lambda_in, geom.lambda_out, wl.rank, wl.scaling, li.A, li.B, SCALE_OP)
         oracle.linear_fwd(Wt, ad, li.X)
         oracle.linear_bwd(Wt, ad, li.X, li.dY)
         b, a = linear_flops(sample_rows, spec.d_out, spec.d_in, wl.rank, geom)
@@ -153,7 +156,7 @@ def run_reference(args, wl, geom):
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
             "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": tot_t / steps * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-            "data": "synthetic", "config": {"workload": wl.name, "geometry": geom.name, "sample": sample},
+            "data": "synthetic", "config": {"workload": wl.name, "geometry": geom.name, "scale_op": SCALE_OP, "sample": sample},
             "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
@@ -198,7 +201,7 @@ def run_gpu(args, wl, geom):
             # distinct device copies (same values): what matters is that the addresses differ
             q2 = qb.QWeight(dq.d_out, dq.d_in, dq.block_in, dq.block_out, dq.qfmt, dq.code,
                             dq.codes.clone(), dq.alpha.clone(), dq.beta.clone() if dq.beta is not None else None)
-            ad = qb.Adapter(geom.lambda_in, geom.lambda_out, r, wl.scaling, bf(li.A), bf(li.B))
+            ad = qb.Adapter(geom.lambda_in, geom.lambda_out, r, wl.scaling, bf(li.A), bf(li.B), SCALE_OP)
             X, dY = bf(li.X), bf(li.dY)
             Y = torch.empty((T, spec.d_out), dtype=torch.bfloat16, device=dev)
             dX = torch.empty((T, spec.d_in), dtype=torch.bfloat16, device=dev)
@@ -327,7 +330,7 @@ def run_gpu(args, wl, geom):
     line = {"metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": wl.name, "geometry": f"{geom.name} (lambda_in={geom.lambda_in}, lambda_out={geom.lambda_out})",
+            "config": {"workload": wl.name, "scale_op": SCALE_OP, "geometry": f"{geom.name} (lambda_in={geom.lambda_in}, lambda_out={geom.lambda_out})",
                        "tokens": T, "linears": [f"{s.name}[{s.d_out},{s.d_in}]" for s in wl.linears], "rank": r,
                        "quant": "4-bit, block 64 along input, " + ("min-max" if wl.qfmt else "level table + absmax"),
                        "parallelism": "replicas only" if world > 1 else "single GPU",
@@ -482,6 +485,9 @@ def main():
     ap.add_argument("--impl", default="gpu", choices=["gpu", "reference"])
     ap.add_argument("--workload", default="C2", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--geometry", default="GA", choices=["GA", "GB"])
+    ap.add_argument("--scale-op", type=int, default=0, choices=[0, 1, 2],
+                    help="adapter operator pair: 0 AvgPool & repeat_interleave (the method), 1 truncation & zero padding, "
+                         "2 interval sampling & zero fill (Sec. 4 ablation)")
     ap.add_argument("--ref-rows", type=int, default=512, help="token rows per oracle step (bounded sample)")
     ap.add_argument("--ref-max-steps", type=int, default=3)
     ap.add_argument("--no-extras", action="store_true")
@@ -490,6 +496,8 @@ def main():
     ap.add_argument("--lowbit-shapes", default="q,up", help="linears of C5 timed in the lowbit extras")
     ap.add_argument("--lowbit-tokens", default="1,16,2048", help="token counts timed in the lowbit extras")
     args = ap.parse_args()
+    global SCALE_OP
+    SCALE_OP = args.scale_op
     args.warmup = max(args.warmup, 3) if args.impl == "gpu" else args.warmup
     wl = synth.WORKLOADS[args.workload]
     geom = synth.GEOM_A if args.geometry == "GA" else synth.GEOM_B

@@ -75,6 +75,21 @@ typedef struct {
   const float* beta;           /* DEVICE same shape; NULL for the code-table format */
 } qblora_qweight;
 
+/* The parameter-free operator pair that compresses the adapter's input and restores its output
+ * size.  The method's own pair is AvgPool & repeat_interleave (Sec. 3.2); the other two are the
+ * alternatives of the Sec. 4 ablation on scale operators (the paper finds them clearly worse; they
+ * exist here to reproduce that comparison).  With P = d_in / lambda_in, Q = d_out / lambda_out:
+ *   AVGPOOL_REPEAT    x'[p] = mean(x[lambda_in p .. lambda_in p + lambda_in - 1]);  y[o] += s y'[o / lambda_out]
+ *   TRUNCATE_ZEROPAD  x'[p] = x[p]            (front part kept);   y[o] += s y'[o] for o < Q, nothing beyond
+ *   SAMPLE_ZEROFILL   x'[p] = x[lambda_in p]  (regular interval);  y[lambda_out q] += s y'[q], nothing between
+ * Only AVGPOOL_REPEAT gives an update that is constant over a quantization block, so qablora_merge
+ * and qablora_merge_noalloc return QBLORA_ERR_INVALID_ARG for the other two; qblora_merge_dense takes all. */
+typedef enum {
+  QBLORA_SCALE_AVGPOOL_REPEAT = 0,
+  QBLORA_SCALE_TRUNCATE_ZEROPAD = 1,
+  QBLORA_SCALE_SAMPLE_ZEROFILL = 2
+} qblora_scale_op;
+
 /* Balanced low-rank adapter (Sec. 3.2): x' = AvgPool_{lambda_in}(x), y' = (A B)^T x',
  * y_adapter = scaling * repeat_interleave_{lambda_out}(y'). */
 typedef struct {
@@ -84,6 +99,7 @@ typedef struct {
   const void* A;                 /* DEVICE bf16 [P][r] */
   const void* B;                 /* DEVICE bf16 [r][Q]; NULL => A is the single matrix H, bf16 [P][Q],
                                     of Sec. 3.3 / Algorithm 2 (rank is then ignored) */
+  int32_t scale_op;              /* qblora_scale_op; 0 = the method's AvgPool & repeat_interleave */
 } qblora_adapter;
 
 /* Writes the built-in 16-level table (HOST out): nine non-negative levels

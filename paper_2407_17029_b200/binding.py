@@ -24,6 +24,8 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_
 FMT_CODEBOOK_ABSMAX, FMT_AFFINE_MINMAX = 0, 1
 F32, BF16 = 0, 1
 OP_QUANTIZE, OP_LINEAR_FWD, OP_LINEAR_BWD, OP_MERGE, OP_LOWBIT_GEMM, OP_MERGE_DENSE = range(6)
+# qblora_scale_op: the parameter-free operator pair around the adapter (Sec. 3.2; Sec. 4 scale-operator ablation)
+SCALE_AVGPOOL_REPEAT, SCALE_TRUNCATE_ZEROPAD, SCALE_SAMPLE_ZEROFILL = range(3)
 
 EXPORTS = ["qblora_default_code_table", "qblora_workspace_bytes", "qblora_status_string",
            "qblora_device_status", "qblora_quantize_blockwise", "qblora_linear_fwd",
@@ -41,7 +43,7 @@ class _CQWeight(ctypes.Structure):
 class _CAdapter(ctypes.Structure):
     _fields_ = [("lambda_in", ctypes.c_int32), ("lambda_out", ctypes.c_int32),
                 ("rank", ctypes.c_int32), ("scaling", ctypes.c_float),
-                ("A", ctypes.c_void_p), ("B", ctypes.c_void_p)]
+                ("A", ctypes.c_void_p), ("B", ctypes.c_void_p), ("scale_op", ctypes.c_int32)]
 
 
 if not os.path.exists(LIB_PATH):
@@ -137,17 +139,20 @@ class QWeight:
 
 @dataclass
 class Adapter:
-    """Balanced adapter: A bf16 [P][r], B bf16 [r][Q] (device); B None => A is H [P][Q] (merge only)."""
+    """Balanced adapter: A bf16 [P][r], B bf16 [r][Q] (device); B None => A is the single matrix H [P][Q].
+    scale_op picks the compress / restore operator pair (default: AvgPool & repeat_interleave)."""
     lambda_in: int
     lambda_out: int
     rank: int
     scaling: float
     A: torch.Tensor
     B: Optional[torch.Tensor]
+    scale_op: int = SCALE_AVGPOOL_REPEAT
 
     def c_struct(self) -> _CAdapter:
         c = _CAdapter()
         c.lambda_in, c.lambda_out, c.rank, c.scaling = self.lambda_in, self.lambda_out, self.rank, self.scaling
+        c.scale_op = int(self.scale_op)
         c.A = self.A.data_ptr()
         c.B = self.B.data_ptr() if self.B is not None else None
         return c

@@ -59,11 +59,12 @@ int make_ad(const qblora_adapter* a, const QwView& q, bool need_ptrs, AdView* v)
   if (a->lambda_in < 1 || a->lambda_out < 1) return QBLORA_ERR_INVALID_ARG;
   if (q.d_in % a->lambda_in || q.d_out % a->lambda_out) return QBLORA_ERR_INVALID_ARG;
   if (a->B && a->rank < 1) return QBLORA_ERR_INVALID_ARG;
+  if (a->scale_op < QBLORA_SCALE_AVGPOOL_REPEAT || a->scale_op > QBLORA_SCALE_SAMPLE_ZEROFILL) return QBLORA_ERR_INVALID_ARG;
   if (need_ptrs) {
     if (!a->A || !aligned16(a->A)) return QBLORA_ERR_INVALID_ARG;
     if (a->B && !aligned16(a->B)) return QBLORA_ERR_INVALID_ARG;
   }
-  v->l1 = a->lambda_in; v->l2 = a->lambda_out; v->r = a->rank; v->s = a->scaling;
+  v->l1 = a->lambda_in; v->l2 = a->lambda_out; v->r = a->rank; v->s = a->scaling; v->op = a->scale_op;
   v->P = q.d_in / a->lambda_in; v->Q = q.d_out / a->lambda_out;
   v->A = static_cast<const __nv_bfloat16*>(a->A);
   v->B = static_cast<const __nv_bfloat16*>(a->B);
@@ -262,8 +263,9 @@ int qablora_merge(const qblora_qweight* qw, const qblora_adapter* adapter, float
   if (q.qfmt != QBLORA_FMT_AFFINE_MINMAX || !adapter || !beta_out || !aligned16(beta_out)) return QBLORA_ERR_INVALID_ARG;
   AdView ad; rc = make_ad(adapter, q, true, &ad);
   if (rc) return rc;
-  // every quantization block must lie inside one (lambda_in x lambda_out) tile of the dense update
-  if (ad.l1 % q.block_in || ad.l2 % q.block_out) return QBLORA_ERR_INVALID_ARG;
+  // every quantization block must lie inside one (lambda_in x lambda_out) tile of the dense update, and
+  // the update must be constant on that tile (only AvgPool & repeat_interleave gives that)
+  if (ad.l1 % q.block_in || ad.l2 % q.block_out || ad.op != QBLORA_SCALE_AVGPOOL_REPEAT) return QBLORA_ERR_INVALID_ARG;
   const size_t need = merge_ws_bytes(q, ad);
   if (!ws || !aligned16(ws) || ws_bytes < need) return QBLORA_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -299,7 +301,7 @@ int qablora_merge_noalloc(const qblora_qweight* qw, const qblora_adapter* adapte
   if (q.qfmt != QBLORA_FMT_AFFINE_MINMAX || !adapter || !beta_out || !aligned16(beta_out)) return QBLORA_ERR_INVALID_ARG;
   AdView ad; rc = make_ad(adapter, q, true, &ad);
   if (rc) return rc;
-  if (ad.l1 % q.block_in || ad.l2 % q.block_out) return QBLORA_ERR_INVALID_ARG;
+  if (ad.l1 % q.block_in || ad.l2 % q.block_out || ad.op != QBLORA_SCALE_AVGPOOL_REPEAT) return QBLORA_ERR_INVALID_ARG;
   if ((int64_t)ad.P * ad.Q > merge_noalloc_capacity()) return QBLORA_ERR_TOO_LARGE;
   return launch_merge_noalloc(q, ad, adapter->B == nullptr, beta_out, static_cast<cudaStream_t>(stream));
 }

@@ -24,10 +24,21 @@ struct QwView {
 
 struct AdView {
   int l1, l2, r, P, Q;
+  int op;  // qblora_scale_op
   float s;
   const __nv_bfloat16* A;
   const __nv_bfloat16* B;
 };
+
+// Index map of the adapter's parameter-free operator pair (Sec. 3.2 and the scale-operator ablation of
+// Sec. 4): the compressed index that full-size index `idx` is tied to, or -1 for none.  `lam` is the
+// factor of that side, `n_small` the compressed size.  The tie's coefficient is 1 / lam on the input side
+// of AvgPool & repeat_interleave and 1 everywhere else.
+__host__ __device__ __forceinline__ int scale_src(int op, int idx, int lam, int n_small) {
+  if (op == QBLORA_SCALE_AVGPOOL_REPEAT) return idx / lam;
+  if (op == QBLORA_SCALE_TRUNCATE_ZEROPAD) return idx < n_small ? idx : -1;
+  return (idx % lam == 0) ? idx / lam : -1;
+}
 
 constexpr size_t kStatusBytes = 256;  // first bytes of every workspace: device status word
 

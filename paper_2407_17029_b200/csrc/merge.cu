@@ -41,8 +41,8 @@ struct Level16 { float v[16]; };
 __global__ void __launch_bounds__(256) merge_dense_kernel(const uint8_t* __restrict__ codes, const float* __restrict__ alpha,
                                                           const float* __restrict__ beta, int d_out, int d_in,
                                                           int block_in, int block_out, const Level16 level16,
-                                                          const double* __restrict__ H, int Q, int l1, int l2,
-                                                          double s_over_l1, __nv_bfloat16* __restrict__ W) {
+                                                          const double* __restrict__ H, int P, int Q, int l1, int l2,
+                                                          int op, double s_over_l1, __nv_bfloat16* __restrict__ W) {
   __shared__ float lev[16];
   if (threadIdx.x < 16) lev[threadIdx.x] = level16.v[threadIdx.x];
   __syncthreads();
@@ -61,16 +61,26 @@ __global__ void __launch_bounds__(256) merge_dense_kernel(const uint8_t* __restr
     // running block / window indices instead of a division per element
     int b = i0 / block_in, brem = i0 - b * block_in;
     int win = i0 / l1, wrem = i0 - win * l1;
-    const double* hcol = H ? H + o / l2 : nullptr;
-    float delta = hcol ? (float)(hcol[(int64_t)win * Q] * s_over_l1) : 0.0f;
+    // AvgPool & repeat_interleave: constant per pooling window.  The alternative operator pairs place
+    // s * H on single kept / sampled positions (s_over_l1 is then s itself) and are looked up per element.
+    const int hq = H ? scale_src(op, o, l2, Q) : -1;
+    const double* hcol = hq >= 0 ? H + hq : nullptr;
+    float delta = (hcol && op == QBLORA_SCALE_AVGPOOL_REPEAT) ? (float)(hcol[(int64_t)win * Q] * s_over_l1) : 0.0f;
     float al = arow[b], be = brow ? brow[b] : 0.0f;
     float v[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
       const int c = (w >> (4 * e)) & 15;
+      if (op != QBLORA_SCALE_AVGPOOL_REPEAT) {
+        const int hp = hcol ? scale_src(op, i0 + e, l1, P) : -1;
+        delta = hp >= 0 ? (float)(hcol[(int64_t)hp * Q] * s_over_l1) : 0.0f;
+      }
       v[e] = fmaf(al, lev[c], be) + delta;
       if (++brem == block_in && e < 7) { brem = 0; ++b; al = arow[b]; be = brow ? brow[b] : 0.0f; }
-      if (++wrem == l1 && e < 7) { wrem = 0; ++win; if (hcol) delta = (float)(hcol[(int64_t)win * Q] * s_over_l1); }
+      if (++wrem == l1 && e < 7) {
+        wrem = 0; ++win;
+        if (hcol && op == QBLORA_SCALE_AVGPOOL_REPEAT) delta = (float)(hcol[(int64_t)win * Q] * s_over_l1);
+      }
     }
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
@@ -105,8 +115,9 @@ int launch_merge_dense(const QwView& qw, const AdView* ad, bool single, __nv_bfl
   }
   const dim3 grid((unsigned)((qw.d_in / 8 + 255) / 256), (unsigned)(qw.d_out < 65535 ? qw.d_out : 65535));
   merge_dense_kernel<<<grid, 256, 0, st>>>(qw.codes, qw.alpha, qw.beta, qw.d_out, qw.d_in, qw.block_in,
-                                                                qw.block_out, lev, H, ad ? ad->Q : 1, ad ? ad->l1 : 1,
-                                                                ad ? ad->l2 : 1, ad ? (double)ad->s / (double)ad->l1 : 0.0, W);
+                                                                qw.block_out, lev, H, ad ? ad->P : 1, ad ? ad->Q : 1, ad ? ad->l1 : 1,
+                                                                ad ? ad->l2 : 1, ad ? ad->op : 0,
+                                                                !ad ? 0.0 : ad->op == QBLORA_SCALE_AVGPOOL_REPEAT ? (double)ad->s / (double)ad->l1 : (double)ad->s, W);
   count_launch();
   QB_CUDA(cudaGetLastError());
   return QBLORA_OK;

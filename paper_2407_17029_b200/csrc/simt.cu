@@ -45,7 +45,7 @@ int simt_linear_fwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, 
   int rc;
   if (ad) {
     int64_t n = T * ad->P;
-    pool_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(X, T, qw.d_in, ad->l1, w.xp);
+    pool_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(X, T, qw.d_in, ad->l1, ad->op, w.xp);
     count_launch();
     QB_CUDA(cudaGetLastError());
     // u = x' A : A is [P][r] -> lb(n = k_rank, k = p) = A[p][k_rank]
@@ -58,7 +58,7 @@ int simt_linear_fwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, 
     if (rc) return rc;
   }
   EpOut ep{Y, y_dtype, qw.d_out, ad ? w.v : nullptr, ad ? ad->Q : 0, ad ? ad->l2 : 1,
-           ad ? ad->s : 0.0f, false};
+           ad ? ad->s : 0.0f, false, ad ? ad->op : 0};
   DominantKernelTimer timer(st);
   return gemm<true, true>(T, qw.d_out, qw.d_in, LdBF16{X, qw.d_in, 1}, LdWq{qw, true}, ep, st);
 }
@@ -70,11 +70,11 @@ int simt_linear_bwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X,
   int rc;
   if (ad) {
     int64_t n = T * ad->P;
-    pool_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(X, T, qw.d_in, ad->l1, w.xp);
+    pool_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(X, T, qw.d_in, ad->l1, ad->op, w.xp);
     count_launch();
     QB_CUDA(cudaGetLastError());
     n = T * ad->Q;
-    dv_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(dY, T, qw.d_out, ad->l2, ad->s, w.dv);
+    dv_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(dY, T, qw.d_out, ad->l2, ad->op, ad->s, w.dv);
     count_launch();
     QB_CUDA(cudaGetLastError());
     // du = dv B^T : lb(n = k_rank, k = q) = B[k_rank][q]
@@ -104,7 +104,7 @@ int simt_linear_bwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X,
     }
   }
   if (dX) {
-    EpOut ep{dX, dx_dtype, qw.d_in, ad ? w.dxp : nullptr, ad ? ad->P : 0, ad ? ad->l1 : 1, 0.0f, true};
+    EpOut ep{dX, dx_dtype, qw.d_in, ad ? w.dxp : nullptr, ad ? ad->P : 0, ad ? ad->l1 : 1, 0.0f, true, ad ? ad->op : 0};
     // dX[t][i] = sum_o dY[t][o] w~[o][i] : lb(n = i, k = o)
     DominantKernelTimer timer(st);
     return gemm<true, false>(T, qw.d_in, qw.d_out, LdBF16{dY, qw.d_out, 1}, LdWq{qw, false}, ep, st);

@@ -39,13 +39,17 @@ struct EpStoreF32 {
   float* C; int64_t ld;
   __device__ void operator()(int m, int n, float acc) const { C[m * ld + n] = acc; }
 };
-struct EpOut {  // out[m][n] = acc + scale * side[m][n / div]   (side may be NULL)
+struct EpOut {  // out[m][n] = acc + scale * side[m][src(n)]   (side may be NULL; src = the operator pair's index map)
   void* out; int dtype; int64_t ld; const float* side; int side_ld; int div; float scale;
-  bool divide;  // true: side / div (backward unpooling), false: side * scale (forward repeat)
+  bool divide;  // true: side / div (backward un-pooling; no division for the sampling operators), false: side * scale (forward)
+  int op;       // qblora_scale_op
   __device__ void operator()(int m, int n, float acc) const {
     if (side) {
-      float sv = side[(int64_t)m * side_ld + n / div];
-      acc += divide ? __fdiv_rn(sv, (float)div) : scale * sv;
+      const int j = scale_src(op, n, div, side_ld);
+      if (j >= 0) {
+        const float sv = side[(int64_t)m * side_ld + j];
+        acc += divide ? (op == QBLORA_SCALE_AVGPOOL_REPEAT ? __fdiv_rn(sv, (float)div) : sv) : scale * sv;
+      }
     }
     if (dtype == QBLORA_BF16) reinterpret_cast<__nv_bfloat16*>(out)[m * ld + n] = __float2bfloat16_rn(acc);
     else reinterpret_cast<float*>(out)[m * ld + n] = acc;
@@ -110,25 +114,35 @@ inline int gemm(int64_t M, int64_t N, int64_t K, LA la, LB lb, EP ep, cudaStream
   return QBLORA_OK;
 }
 
-// x'[t][p] = mean of lambda_in consecutive inputs (AvgPool of Sec. 3.2), fp32.
-static __global__ void pool_kernel(const __nv_bfloat16* __restrict__ X, int64_t T, int d_in, int l1,
+// x'[t][p] = mean of lambda_in consecutive inputs (AvgPool of Sec. 3.2), fp32; for the alternative operators
+// of the Sec. 4 ablation the kept value x[p] (truncation) or the sample x[lambda_in p] (interval sampling).
+static __global__ void pool_kernel(const __nv_bfloat16* __restrict__ X, int64_t T, int d_in, int l1, int op,
                             float* __restrict__ xp) {
   const int P = d_in / l1;
   int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= T * P) return;
   const int64_t t = idx / P; const int p = (int)(idx % P);
+  if (op != QBLORA_SCALE_AVGPOOL_REPEAT) {
+    xp[idx] = __bfloat162float(X[t * d_in + (op == QBLORA_SCALE_TRUNCATE_ZEROPAD ? p : (int64_t)p * l1)]);
+    return;
+  }
   float s = 0.0f;
   for (int j = 0; j < l1; ++j) s += __bfloat162float(X[t * d_in + (int64_t)p * l1 + j]);
   xp[idx] = __fdiv_rn(s, (float)l1);
 }
 
-// dv[t][q] = s * sum of lambda_out consecutive output gradients (adjoint of repeat_interleave).
-static __global__ void dv_kernel(const __nv_bfloat16* __restrict__ dY, int64_t T, int d_out, int l2, float s,
+// dv[t][q] = s * sum of lambda_out consecutive output gradients (adjoint of repeat_interleave); the adjoint
+// of zero padding / zero filling reads the single output the value was written to.
+static __global__ void dv_kernel(const __nv_bfloat16* __restrict__ dY, int64_t T, int d_out, int l2, int op, float s,
                           float* __restrict__ dv) {
   const int Q = d_out / l2;
   int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= T * Q) return;
   const int64_t t = idx / Q; const int q = (int)(idx % Q);
+  if (op != QBLORA_SCALE_AVGPOOL_REPEAT) {
+    dv[idx] = s * __bfloat162float(dY[t * d_out + (op == QBLORA_SCALE_TRUNCATE_ZEROPAD ? q : (int64_t)q * l2)]);
+    return;
+  }
   float a = 0.0f;
   for (int j = 0; j < l2; ++j) a += __bfloat162float(dY[t * d_out + (int64_t)q * l2 + j]);
   dv[idx] = s * a;

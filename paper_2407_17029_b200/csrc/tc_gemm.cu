@@ -57,6 +57,7 @@ struct TcParams {
   float level[16];
   const __nv_bfloat16* ex;  // adapter matrix feeding the extra K-blocks: forward B [r][Q], backward A [P][r]
   int ex_ld, ex_rows, lam;  // its leading dimension; the rank r; forward lambda_out, backward lambda_in
+  int op, n_small;          // operator pair (qblora_scale_op) and the compressed size on that side (forward Q, backward P)
   void* out;                // forward Y [T][d_out]; backward dX [T][d_in]
   int out_dtype;
   int* status;
@@ -332,13 +333,30 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
             const int o0 = m0 + (d >> 6) * 64;
             const unsigned short* src = reinterpret_cast<const unsigned short*>(p.ex) + (int64_t)krow * p.ex_ld;
             const bool live = krow < p.ex_rows;
-            if ((p.lam & 7) == 0) {       // a 16-byte chunk (8 outputs) repeats a single element of B
+            if ((p.lam & 7) == 0 && p.op == QBLORA_SCALE_AVGPOOL_REPEAT) {   // a 16-byte chunk (8 outputs) repeats a single element of B
 #pragma unroll
               for (int j = 0; j < 8; ++j) {
                 const int o = o0 + j * 8;
                 uint32_t v = (live && o < p.d_out) ? (uint32_t)__ldg(src + o / p.lam) : 0u;
                 v |= v << 16;
                 st_shared_v4(dst + (((uint32_t)j ^ xr) << 4), v, v, v, v);
+              }
+            } else if (p.op == QBLORA_SCALE_TRUNCATE_ZEROPAD) {
+              // the first Q outputs take B's row as it is (Q is a multiple of 8: whole aligned 16-byte chunks), the rest nothing
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                const int o = o0 + j * 8;
+                uint4 v = make_uint4(0, 0, 0, 0);
+                if (live && o < p.n_small) v = __ldg(reinterpret_cast<const uint4*>(src + o));
+                st_shared_v4(dst + (((uint32_t)j ^ xr) << 4), v.x, v.y, v.z, v.w);
+              }
+            } else if ((p.lam & 7) == 0) {
+              // zero fill with a factor that is a multiple of 8: only the first output of a chunk can be a sampled one
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                const int o = o0 + j * 8;
+                const uint32_t v = (live && o < p.d_out && o % p.lam == 0) ? (uint32_t)__ldg(src + o / p.lam) : 0u;
+                st_shared_v4(dst + (((uint32_t)j ^ xr) << 4), v, 0u, 0u, 0u);
               }
             } else {
 #pragma unroll
@@ -347,8 +365,10 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                   const int oa = o0 + j * 8 + 2 * e, ob = oa + 1;
-                  const uint32_t lo = (live && oa < p.d_out) ? (uint32_t)__ldg(src + oa / p.lam) : 0u;
-                  const uint32_t hi = (live && ob < p.d_out) ? (uint32_t)__ldg(src + ob / p.lam) : 0u;
+                  // column of B that the operator pair ties this output to (none: the output gets no adapter term)
+                  const int qa = scale_src(p.op, oa, p.lam, p.n_small), qb_ = scale_src(p.op, ob, p.lam, p.n_small);
+                  const uint32_t lo = (live && oa < p.d_out && qa >= 0) ? (uint32_t)__ldg(src + qa) : 0u;
+                  const uint32_t hi = (live && ob < p.d_out && qb_ >= 0) ? (uint32_t)__ldg(src + qb_) : 0u;
                   o4[e] = lo | (hi << 16);
                 }
                 st_shared_v4(dst + (((uint32_t)j ^ xr) << 4), o4[0], o4[1], o4[2], o4[3]);
@@ -358,11 +378,12 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
             // K-major tile: A[m = i][k] = A_adapter[i / lambda_in][kk + k]; thread = input column i,
             // reading 128 contiguous bytes of a row of A_adapter (rank is a multiple of 8)
             const int i = m0 + d;
-            const uint4* src = reinterpret_cast<const uint4*>(p.ex + (int64_t)(i / p.lam) * p.ex_ld + kk);
+            const int prow = i < p.d_in ? scale_src(p.op, i, p.lam, p.n_small) : -1;   // -1: input not seen by the adapter
+            const uint4* src = reinterpret_cast<const uint4*>(p.ex + (int64_t)(prow < 0 ? 0 : prow) * p.ex_ld + kk);
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
               uint4 v = make_uint4(0, 0, 0, 0);
-              if (i < p.d_in && kk + j * 8 < p.ex_rows) v = __ldg(src + j);
+              if (prow >= 0 && kk + j * 8 < p.ex_rows) v = __ldg(src + j);
               st_shared_v4(dst + (((uint32_t)j ^ xr) << 4), v.x, v.y, v.z, v.w);
             }
           }
@@ -538,6 +559,16 @@ __global__ void dv_split_kernel(const __nv_bfloat16* __restrict__ dY, int64_t T,
   store_split(scaling * a, hi, lo, t * ldq + q);
 }
 
+// The alternative operator pairs of the Sec. 4 ablation read single values: out[t][j] = scale * src[t][j * stride]
+// (stride 1 = truncation, lambda = interval sampling; scale = 1 for x', s for dv), stored as a hi + lo pair.
+__global__ void sample_split_kernel(const __nv_bfloat16* __restrict__ src, int64_t T, int width, int n_small, int stride,
+                                    float scale, int ld_out, __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= T * n_small) return;
+  const int64_t t = idx / n_small; const int j = (int)(idx - t * n_small);
+  store_split(scale * __bfloat162float(src[t * width + (int64_t)j * stride]), hi, lo, t * ld_out + j);
+}
+
 int num_sms() {
   static int n = []() {
     int dev = 0, v = 0;
@@ -608,6 +639,8 @@ int launch_main(int mode, const QwView& qw, const AdView* ad, const __nv_bfloat1
   p.ex_ld = ad ? (mode == 0 ? ad->Q : ad->r) : 0;
   p.ex_rows = ad ? ad->r : 0;
   p.lam = ad ? (mode == 0 ? ad->l2 : ad->l1) : 1;
+  p.op = ad ? ad->op : 0;
+  p.n_small = ad ? (mode == 0 ? ad->Q : ad->P) : 0;
   p.out = out; p.out_dtype = out_dtype; p.status = status;
 
   CUtensorMap tm_b, tm_bx, tm_p;
@@ -635,7 +668,10 @@ int launch_main(int mode, const QwView& qw, const AdView* ad, const __nv_bfloat1
 
 int launch_pool(const QwView& qw, const AdView& ad, const __nv_bfloat16* X, int64_t T, const TcWs& w, cudaStream_t st) {
   const int64_t n = T * ad.P;
-  if (segsum_fast_ok(qw.d_in, ad.l1)) {
+  if (ad.op != QBLORA_SCALE_AVGPOOL_REPEAT) {
+    sample_split_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(
+        X, T, qw.d_in, ad.P, ad.op == QBLORA_SCALE_TRUNCATE_ZEROPAD ? 1 : ad.l1, 1.0f, w.ldp, w.xh, w.xl);
+  } else if (segsum_fast_ok(qw.d_in, ad.l1)) {
     const int64_t chunks = T * (qw.d_in / 8);
     segsum_split_kernel<true><<<(unsigned)((chunks + 1023) / 1024), 256, 0, st>>>(X, T, qw.d_in, ad.l1, 0.0f, w.ldp, w.xh, w.xl);
   } else {
@@ -729,7 +765,10 @@ int tc_linear_bwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, co
       QB_CUDA(cudaStreamWaitEvent(lane->stream, lane->fork, 0));
     }
     const int64_t n = T * ad->Q;
-    if (segsum_fast_ok(qw.d_out, ad->l2)) {
+    if (ad->op != QBLORA_SCALE_AVGPOOL_REPEAT) {
+      sample_split_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(
+          dY, T, qw.d_out, ad->Q, ad->op == QBLORA_SCALE_TRUNCATE_ZEROPAD ? 1 : ad->l2, ad->s, w.ldq, w.dvh, w.dvl);
+    } else if (segsum_fast_ok(qw.d_out, ad->l2)) {
       const int64_t chunks = T * (qw.d_out / 8);
       segsum_split_kernel<false><<<(unsigned)((chunks + 1023) / 1024), 256, 0, st>>>(dY, T, qw.d_out, ad->l2, ad->s, w.ldq, w.dvh, w.dvl);
     } else {
@@ -741,7 +780,8 @@ int tc_linear_bwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, co
       const SgOperand b_mat{ad->B, ad->Q, true};   // (n = rank index, k = q) at B[n * Q + k]
       SgSegment segs[2] = {{{w.dvh, w.ldq, true}, b_mat, ad->Q}, {{w.dvl, w.ldq, true}, b_mat, ad->Q}};
       SgOut out{};
-      out.hi = w.duh; out.lo = w.dul; out.scaled = w.du16; out.ld16 = w.ldr; out.scale = (float)ad->l1; out.divide = true;
+      out.hi = w.duh; out.lo = w.dul; out.scaled = w.du16; out.ld16 = w.ldr; out.divide = true;
+      out.scale = ad->op == QBLORA_SCALE_AVGPOOL_REPEAT ? (float)ad->l1 : 1.0f;   // only the average carries 1 / lambda_in
       rc = small_gemm((int)T, ad->r, segs, 2, out, status, st);
       if (rc) return rc;
     }

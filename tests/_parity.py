@@ -72,13 +72,13 @@ def qweight_to_dev(qw: oracle.QWeight) -> qb.QWeight:
 
 def adapter_to_dev(ad: oracle.Adapter) -> qb.Adapter:
     return qb.Adapter(ad.lambda_in, ad.lambda_out, ad.rank, float(ad.scaling), to_bf16_dev(ad.A),
-                      to_bf16_dev(ad.B) if ad.B is not None else None)
+                      to_bf16_dev(ad.B) if ad.B is not None else None, int(ad.scale_op))
 
 
 def visible_scaling(Wt, ad: oracle.Adapter, X) -> float:
     """Scaling s* (fp32-representable) at which the adapter term's RMS equals the base term's."""
     base = oracle.linear_fwd(Wt, None, X)
-    one = oracle.Adapter(ad.lambda_in, ad.lambda_out, ad.rank, 1.0, ad.A, ad.B)
+    one = oracle.Adapter(ad.lambda_in, ad.lambda_out, ad.rank, 1.0, ad.A, ad.B, ad.scale_op)
     term = oracle.linear_fwd(Wt, one, X) - base
     return float(np.float32(rms(base) / max(rms(term), 1e-30)))
 
