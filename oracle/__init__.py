@@ -98,7 +98,9 @@ class Adapter:
     scale_op: int = 0               # OP_AVGPOOL_REPEAT / OP_TRUNCATE_ZEROPAD / OP_SAMPLE_ZEROFILL
 
 
-def quantize_blockwise(W, block_in=64, block_out=1, qfmt=FMT_CODEBOOK_ABSMAX, code=None) -> QWeight:
+def quantize_blockwise(W, block_in=64, block_out=1, qfmt=FMT_CODEBOOK_ABSMAX, code=None, nbits=4) -> QWeight:
+    """Eq. 1 per block.  nbits < 4 (min-max format only) restricts the grid to 2^nbits levels; the codes are
+    still stored one per nibble, so everything downstream treats the result as a 4-bit weight."""
     W = _f32(W)
     d_out, d_in = W.shape
     if qfmt == FMT_CODEBOOK_ABSMAX and code is None:
@@ -109,7 +111,7 @@ def quantize_blockwise(W, block_in=64, block_out=1, qfmt=FMT_CODEBOOK_ABSMAX, co
     codes = np.zeros((d_out, d_in // 2), dtype=np.uint8)
     alpha = np.zeros((d_out // block_out, d_in // block_in), dtype=np.float32)
     beta = np.zeros_like(alpha) if qfmt == FMT_AFFINE_MINMAX else None
-    rc = _L().orc_quantize_blockwise(_p(W, ctypes.c_float), d_out, d_in, block_in, block_out, qfmt,
+    rc = _L().orc_quantize_blockwise(_p(W, ctypes.c_float), d_out, d_in, block_in, block_out, qfmt, int(nbits),
                                      _p(code, ctypes.c_float), _p(codes, ctypes.c_uint8),
                                      _p(alpha, ctypes.c_float), _p(beta, ctypes.c_float))
     _check(rc, "quantize_blockwise")

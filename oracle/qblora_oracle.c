@@ -88,14 +88,20 @@ static int get_code(const uint8_t* codes, int d_in, int o, int i) {
  *   read with the level table in place of the integer grid.
  * qfmt 1 (min-max, Eq. 1 with N = 4): beta = min, alpha = fl32(fl32(max-min)/15),
  *   code = clamp(round-half-even(fl32(fl32(w-beta)/alpha)), 0, 15).
+ *   With nbits = N < 4 (Eq. 1 is stated for N bits) the grid has 2^N levels:
+ *   alpha = fl32(fl32(max-min)/(2^N-1)), codes clamp to [0, 2^N-1]; they are
+ *   still stored one per nibble (packing denser than 4 bits is not modelled).
+ *   nbits applies to the min-max format only; the level table has 16 entries.
  * A block is block_out consecutive rows by block_in consecutive columns.
  * Degenerate block (alpha = 0): qfmt 0 -> every code is the level-0.0 index
  * (or nearest-to-zero level); qfmt 1 -> every code 0, so w~ = beta exactly.
  */
 int orc_quantize_blockwise(const float* W, int d_out, int d_in, int block_in,
-                           int block_out, int qfmt, const float* code,
+                           int block_out, int qfmt, int nbits, const float* code,
                            uint8_t* codes, float* alpha, float* beta) {
   if (d_in % 2 || d_in % block_in || d_out % block_out) return ORC_BAD;
+  if (nbits < 1 || nbits > 4 || (qfmt == 0 && nbits != 4)) return ORC_BAD;
+  const float qmax = (float)((1 << nbits) - 1);
   int G = d_in / block_in, R = d_out / block_out;
   float mid[15];
   int zero_idx = 0;
@@ -134,7 +140,7 @@ int orc_quantize_blockwise(const float* W, int d_out, int d_in, int block_in,
           }
       } else {
         float d = f32_sub(wmax, wmin);
-        float a = f32_div(d, 15.0f);
+        float a = f32_div(d, qmax);
         int degenerate = (d == 0.0f) || (a == 0.0f);
         beta[bi] = wmin;
         alpha[bi] = degenerate ? 0.0f : a;
@@ -145,7 +151,7 @@ int orc_quantize_blockwise(const float* W, int d_out, int d_in, int block_in,
               float q = f32_div(f32_sub(W[(size_t)o * d_in + i], wmin), a);
               double rq = nearbyint((double)q); /* default mode: half to even */
               if (rq < 0.0) rq = 0.0;
-              if (rq > 15.0) rq = 15.0;
+              if (rq > (double)qmax) rq = (double)qmax;
               c = (int)rq;
             }
             set_code(codes, d_in, o, i, c);

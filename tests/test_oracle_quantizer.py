@@ -185,3 +185,57 @@ def test_affine_tie_rounds_half_to_even():
     W[0, 2:6] = [0.5, 1.5, 2.5, 13.5]
     c = unpack(oracle.quantize_blockwise(W, 64, 1, 1).codes)[0]
     assert list(c[2:6]) == [0, 2, 2, 14]
+
+
+# ----------------------------------------------------------------- N-bit grids (Eq. 1 with N < 4)
+@pytest.mark.parametrize("nbits", [1, 2, 3])
+def test_nbit_closed_form_grid_maps_to_integers(nbits):
+    # block = beta + alpha*k, k = 0 .. 2^N-1: Eq. 1 min-max returns alpha, beta and codes = k exactly
+    levels = 1 << nbits
+    alpha, beta = np.float32(0.25), np.float32(-0.75)
+    k = np.tile(np.arange(levels), 64 // levels)
+    W = (beta + alpha * k).astype(np.float32)[None, :]
+    qw = oracle.quantize_blockwise(W, 64, 1, oracle.FMT_AFFINE_MINMAX, nbits=nbits)
+    assert qw.alpha[0, 0] == alpha and qw.beta[0, 0] == beta
+    assert np.array_equal(unpack(qw.codes)[0], k)
+    assert np.array_equal(oracle.dequantize(qw), W.astype(np.float64))
+
+
+@pytest.mark.parametrize("nbits", [2, 3])
+@pytest.mark.parametrize("bi,bo", [(64, 1), (8, 8)])
+def test_nbit_brute_force_rounding_and_error_bound(nbits, bi, bo):
+    qmax = (1 << nbits) - 1
+    W = synth.normal(5, f"nbit/{nbits}/{bi}x{bo}", (64, 256), 0.02)
+    qw = oracle.quantize_blockwise(W, bi, bo, oracle.FMT_AFFINE_MINMAX, nbits=nbits)
+    Wb = _blocks(W.astype(np.float64), bi, bo)
+    mn, mx = Wb.min(axis=2), Wb.max(axis=2)
+    assert np.array_equal(qw.beta, mn.astype(np.float32))
+    a = (mx - mn) / qmax                                              # alpha = (max-min)/(2^N-1)
+    assert np.allclose(qw.alpha, a, rtol=3e-7, atol=0)
+    q = (Wb - mn[..., None]) / a[..., None]
+    clear = np.abs(q - np.floor(q) - 0.5) > 1e-4
+    got = _blocks(unpack(qw.codes), bi, bo)
+    assert got.max() == qmax and got.min() == 0                      # the whole N-bit range and nothing beyond it
+    assert np.array_equal(got[clear], np.clip(np.rint(q), 0, qmax).astype(np.uint8)[clear])
+    # rounding to the nearest grid point: |w - w~| <= alpha / 2 (small slack for the fp32 steps)
+    err = np.abs(_blocks(oracle.dequantize(qw), bi, bo) - Wb)
+    assert np.all(err <= 0.5 * qw.alpha.astype(np.float64)[..., None] * (1 + 1e-5))
+    # one bit less doubles the step: the worst error grows accordingly
+    qw4 = oracle.quantize_blockwise(W, bi, bo, oracle.FMT_AFFINE_MINMAX)
+    assert np.abs(oracle.dequantize(qw4) - W).max() < err.max()
+
+
+def test_nbit_four_is_the_default_and_round_trip_is_stable():
+    W = synth.normal(6, "nbit/rt", (32, 128), 0.02)
+    q4 = oracle.quantize_blockwise(W, 64, 1, oracle.FMT_AFFINE_MINMAX)
+    q4b = oracle.quantize_blockwise(W, 64, 1, oracle.FMT_AFFINE_MINMAX, nbits=4)
+    assert np.array_equal(q4.codes, q4b.codes) and np.array_equal(q4.alpha, q4b.alpha)
+    for nbits in (2, 3):
+        q = oracle.quantize_blockwise(W, 64, 1, oracle.FMT_AFFINE_MINMAX, nbits=nbits)
+        again = oracle.quantize_blockwise(oracle.dequantize(q).astype(np.float32), 64, 1,
+                                          oracle.FMT_AFFINE_MINMAX, nbits=nbits)
+        assert np.mean(unpack(again.codes) == unpack(q.codes)) > 0.995       # codes stable under a second pass
+    with pytest.raises(ValueError):
+        oracle.quantize_blockwise(W, 64, 1, oracle.FMT_AFFINE_MINMAX, nbits=5)
+    with pytest.raises(ValueError):
+        oracle.quantize_blockwise(W, 64, 1, oracle.FMT_CODEBOOK_ABSMAX, nbits=3)
