@@ -29,7 +29,7 @@ from paper_2407_17029_b200 import synth  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, per launch, from the ncu
 # capture summarised in profiles/ncu_full_tc_dq_gemm_C2.md (set to None when that kernel changes)
-MEASURED_DRAM_TRAFFIC = {("C2", "GA"): 27.6e6 + 0.06e6}
+MEASURED_DRAM_TRAFFIC = {("C2", "GA"): 27.61e6 + 0.36e6}
 
 METRIC = "fused 4-bit+BLoRA linear fwd+bwd TFLOP/s & low-bit GEMM GB/s, % of roofline"
 

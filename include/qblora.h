@@ -148,6 +148,20 @@ int qblora_quantize_blockwise(const void* W, int w_dtype, int32_t d_out, int32_t
                               void* stream);
 
 /*
+ * Min-max quantization on an N-bit grid, N = bits in 1..4 (Eq. 1 is stated for N bits; Sec. 3.1):
+ *   beta = min; alpha = (max - min) / (2^N - 1); code = clamp(rint((w - beta) / alpha), 0, 2^N - 1), ties to even;
+ *   constant block: alpha = 0, code = 0.  Same single-rounding fp32 arithmetic as above; bits = 4 gives exactly
+ *   qblora_quantize_blockwise's min-max result.
+ * Storage is unchanged: one code per nibble, codes uint8 [d_out][d_in/2] (no packing denser than 4 bits), so
+ * the result is an ordinary QBLORA_FMT_AFFINE_MINMAX weight for every other call of this library (forward,
+ * backward, both merges, low-bit product); what changes is the number of levels a weight can take.
+ * Arguments and requirements as for qblora_quantize_blockwise; beta must not be NULL.
+ */
+int qblora_quantize_minmax_nbit(const void* W, int w_dtype, int32_t d_out, int32_t d_in,
+                                int32_t block_in, int32_t block_out, int32_t bits,
+                                uint8_t* codes, float* alpha, float* beta, void* stream);
+
+/*
  * Forward of the adapted quantized linear (Sec. 3.1 combined formula with the Sec. 3.2 adapter;
  * Algorithm 1's forward read as its prose):
  *   Y[t][o] = sum_i X[t][i] * w~[o][i]  +  s * ((x' A) B)[t][o / lambda_out],

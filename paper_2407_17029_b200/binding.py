@@ -30,7 +30,8 @@ SCALE_AVGPOOL_REPEAT, SCALE_TRUNCATE_ZEROPAD, SCALE_SAMPLE_ZEROFILL = range(3)
 EXPORTS = ["qblora_default_code_table", "qblora_workspace_bytes", "qblora_status_string",
            "qblora_device_status", "qblora_quantize_blockwise", "qblora_linear_fwd",
            "qblora_linear_bwd", "qablora_merge", "qablora_lowbit_gemm", "qblora_kernel_launches",
-           "qblora_set_timing_events", "qablora_merge_noalloc", "qblora_merge_dense"]
+           "qblora_set_timing_events", "qablora_merge_noalloc", "qblora_merge_dense",
+           "qblora_quantize_minmax_nbit"]
 
 
 class _CQWeight(ctypes.Structure):
@@ -59,6 +60,9 @@ _lib.qblora_device_status.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
 _lib.qblora_quantize_blockwise.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int32, ctypes.c_int32,
                                            ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p,
                                            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+_lib.qblora_quantize_minmax_nbit.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int32, ctypes.c_int32,
+                                             ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p,
+                                             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
 _lib.qblora_linear_fwd.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
                                    ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t,
                                    ctypes.c_void_p]
@@ -213,6 +217,20 @@ def quantize_blockwise(W: torch.Tensor, block_in: int = 64, block_out: int = 1,
     _check(st, "qblora_quantize_blockwise")
     return QWeight(d_out, d_in, block_in, block_out, qfmt, list(code) if code is not None else [0.0] * 16,
                    codes, alpha, beta)
+
+
+def quantize_minmax_nbit(W: torch.Tensor, bits: int, block_in: int = 64, block_out: int = 1, stream=None) -> QWeight:
+    """Min-max quantization of W [d_out][d_in] (fp32 or bf16) on a 2^bits-level grid (Eq. 1 with N = bits).
+    The codes stay one per nibble, so the result is an ordinary min-max QWeight for every other call."""
+    assert W.is_cuda and W.is_contiguous() and W.dim() == 2
+    d_out, d_in = W.shape
+    codes = torch.empty((d_out, d_in // 2), dtype=torch.uint8, device=W.device)
+    alpha = torch.empty((max(d_out // block_out, 1), max(d_in // block_in, 1)), dtype=torch.float32, device=W.device)
+    beta = torch.empty_like(alpha)
+    st = _lib.qblora_quantize_minmax_nbit(W.data_ptr(), _dt(W.dtype), d_out, d_in, block_in, block_out, int(bits),
+                                          codes.data_ptr(), alpha.data_ptr(), beta.data_ptr(), _stream_ptr(stream))
+    _check(st, "qblora_quantize_minmax_nbit")
+    return QWeight(d_out, d_in, block_in, block_out, FMT_AFFINE_MINMAX, [0.0] * 16, codes, alpha, beta)
 
 
 def linear_fwd(qw: QWeight, ad: Optional[Adapter], X: torch.Tensor, out_dtype=torch.bfloat16,

@@ -181,8 +181,20 @@ int qblora_quantize_blockwise(const void* W, int w_dtype, int32_t d_out, int32_t
   } else {
     return QBLORA_ERR_INVALID_ARG;
   }
-  return launch_quantize(W, w_dtype, d_out, d_in, block_in, block_out, qfmt, code, codes, alpha, beta,
+  return launch_quantize(W, w_dtype, d_out, d_in, block_in, block_out, qfmt, 4, code, codes, alpha, beta,
                          static_cast<cudaStream_t>(stream));
+}
+
+int qblora_quantize_minmax_nbit(const void* W, int w_dtype, int32_t d_out, int32_t d_in, int32_t block_in,
+                                int32_t block_out, int32_t bits, uint8_t* codes, float* alpha, float* beta,
+                                void* stream) {
+  if (bits < 1 || bits > 4) return QBLORA_ERR_INVALID_ARG;
+  if (!W || !codes || !alpha || !beta || !dtype_ok(w_dtype)) return QBLORA_ERR_INVALID_ARG;
+  if (d_in <= 0 || d_out <= 0 || block_in <= 0 || block_out <= 0) return QBLORA_ERR_INVALID_ARG;
+  if (d_in % 2 || d_in % block_in || d_out % block_out) return QBLORA_ERR_INVALID_ARG;
+  if (!aligned16(W) || !aligned16(codes) || !aligned16(alpha) || !aligned16(beta)) return QBLORA_ERR_INVALID_ARG;
+  return launch_quantize(W, w_dtype, d_out, d_in, block_in, block_out, QBLORA_FMT_AFFINE_MINMAX, bits, nullptr, codes,
+                         alpha, beta, static_cast<cudaStream_t>(stream));
 }
 
 int qblora_linear_fwd(const qblora_qweight* qw, const qblora_adapter* adapter, const void* X, int64_t tokens,

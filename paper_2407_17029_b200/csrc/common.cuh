@@ -56,7 +56,7 @@ struct DominantKernelTimer {
 
 // ---- entry points of the individual translation units (host side) ----------------------------
 int launch_quantize(const void* W, int w_dtype, int d_out, int d_in, int block_in, int block_out,
-                    int qfmt, const float* level, uint8_t* codes, float* alpha, float* beta,
+                    int qfmt, int bits, const float* level, uint8_t* codes, float* alpha, float* beta,
                     cudaStream_t st);
 
 // General path (any block shape, any size): CUDA-core kernels.

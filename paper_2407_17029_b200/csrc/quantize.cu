@@ -9,6 +9,7 @@ namespace {
 struct QuantTable {
   float mid[15];  // fl32 midpoints between adjacent levels
   int zero_idx;   // index of the level closest to 0 (used for all-zero blocks)
+  float qmax;     // largest code of the min-max grid: 2^N - 1 (15 for the 4-bit weight)
 };
 
 __device__ __forceinline__ float load_w(const float* W, int64_t i) { return W[i]; }
@@ -23,10 +24,10 @@ __device__ __forceinline__ int code_of_level(float v, const QuantTable& t) {
   return c;
 }
 
-__device__ __forceinline__ int code_of_affine(float w, float beta, float alpha) {
+__device__ __forceinline__ int code_of_affine(float w, float beta, float alpha, float qmax) {
   float q = __fdiv_rn(__fsub_rn(w, beta), alpha);
   float rq = rintf(q);  // ties to even
-  rq = fminf(fmaxf(rq, 0.0f), 15.0f);
+  rq = fminf(fmaxf(rq, 0.0f), qmax);
   return (int)rq;
 }
 
@@ -81,11 +82,11 @@ __global__ void __launch_bounds__(256) quantize_b64_kernel(const TIn* __restrict
       if (live && part == 0) alpha[b] = am;
     } else {
       const float d = __fsub_rn(mx, mn);
-      const float a = __fdiv_rn(d, 15.0f);
+      const float a = __fdiv_rn(d, tab.qmax);
       const bool degenerate = (d == 0.0f) || (a == 0.0f);
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
-        const int c = degenerate ? 0 : code_of_affine(v[e], mn, a);
+        const int c = degenerate ? 0 : code_of_affine(v[e], mn, a, tab.qmax);
         packed |= (uint32_t)c << (4 * e);
       }
       if (live && part == 0) {
@@ -121,7 +122,7 @@ __global__ void quantize_generic_kernel(const TIn* __restrict__ W, int d_out, in
     alpha[b] = am;
   } else {
     float d = __fsub_rn(mx, mn);
-    a = __fdiv_rn(d, 15.0f);
+    a = __fdiv_rn(d, tab.qmax);
     degenerate = (d == 0.0f) || (a == 0.0f);
     alpha[b] = degenerate ? 0.0f : a;
     beta[b] = mn;
@@ -135,7 +136,7 @@ __global__ void quantize_generic_kernel(const TIn* __restrict__ W, int d_out, in
         if (qfmt == QBLORA_FMT_CODEBOOK_ABSMAX)
           c[e] = degenerate ? tab.zero_idx : code_of_level(__fdiv_rn(w, am), tab);
         else
-          c[e] = degenerate ? 0 : code_of_affine(w, mn, a);
+          c[e] = degenerate ? 0 : code_of_affine(w, mn, a, tab.qmax);
       }
       codes[(int64_t)o * (d_in / 2) + i / 2] = (uint8_t)(c[0] | (c[1] << 4));
     }
@@ -144,10 +145,11 @@ __global__ void quantize_generic_kernel(const TIn* __restrict__ W, int d_out, in
 }  // namespace
 
 int launch_quantize(const void* W, int w_dtype, int d_out, int d_in, int block_in, int block_out,
-                    int qfmt, const float* level, uint8_t* codes, float* alpha, float* beta,
+                    int qfmt, int bits, const float* level, uint8_t* codes, float* alpha, float* beta,
                     cudaStream_t st) {
   QuantTable tab;
   tab.zero_idx = 0;
+  tab.qmax = (float)((1 << bits) - 1);
   for (int j = 0; j < 15; ++j) tab.mid[j] = 0.0f;
   if (qfmt == QBLORA_FMT_CODEBOOK_ABSMAX) {
     for (int j = 0; j < 15; ++j)

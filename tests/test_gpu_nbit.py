@@ -1,0 +1,79 @@
+"""GPU parity for the N-bit min-max quantizer (Eq. 1 with N < 4): codes, alpha and beta bit for bit
+against the CPU oracle, and the quantized weight used through the rest of the library (forward,
+backward, offset merge, low-bit product) like any other min-max weight."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2407_17029_b200 import synth
+from tests._parity import (adapter_to_dev, gate_strict, to_bf16_dev, to_dev, to_np64, visible_scaling)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def qb():
+    from paper_2407_17029_b200 import binding
+    return binding
+
+
+@pytest.mark.parametrize("bits", [1, 2, 3, 4])
+@pytest.mark.parametrize("shape,bi,bo", [((256, 1024), 64, 1), ((200, 192), 64, 1), ((64, 256), 8, 8), ((1, 64), 64, 1)])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_quantize_nbit_bit_exact(qb, bits, shape, bi, bo, dtype):
+    W = synth.normal(81, f"nbit/{shape}/{bi}x{bo}", shape, 0.02)
+    W[0, :bi] = 0.25                      # a constant block
+    if dtype == "bf16":
+        W = synth.round_to_bf16(W)
+        Wd = to_bf16_dev(W)
+    else:
+        Wd = to_dev(W)
+    ref = oracle.quantize_blockwise(W, bi, bo, oracle.FMT_AFFINE_MINMAX, nbits=bits)
+    got = qb.quantize_minmax_nbit(Wd, bits, bi, bo)
+    codes = got.codes.cpu().numpy()
+    assert np.array_equal(codes, ref.codes)
+    top = max(int((codes & 15).max()), int((codes >> 4).max()))
+    assert top == ((1 << bits) - 1 if W.size > bi * bo else 0)           # (the single-block case is all constant)
+    assert np.array_equal(got.alpha.cpu().numpy().view(np.uint32), ref.alpha.view(np.uint32))
+    assert np.array_equal(got.beta.cpu().numpy().view(np.uint32), ref.beta.view(np.uint32))
+    if bits == 4:
+        same = qb.quantize_blockwise(Wd, bi, bo, qb.FMT_AFFINE_MINMAX)
+        assert torch.equal(same.codes, got.codes) and torch.equal(same.alpha, got.alpha) and torch.equal(same.beta, got.beta)
+
+
+@pytest.mark.parametrize("bits", [2, 3])
+def test_nbit_weight_through_the_layer(qb, bits):
+    T, d_out, d_in, l1, l2, r = 300, 320, 448, 64, 8, 48
+    W = synth.normal(82, "nbit/layer/W", (d_out, d_in), 0.02)
+    X, _ = synth.make_activations(82, "nbit/layer/X", T, d_in, 0.0)
+    dY = synth.round_to_bf16(synth.normal(82, "nbit/layer/dY", (T, d_out)))
+    A = synth.round_to_bf16(synth.normal(82, "nbit/layer/A", (d_in // l1, r), 0.01))
+    B = synth.round_to_bf16(synth.normal(82, "nbit/layer/B", (r, d_out // l2), 0.01))
+    qw = oracle.quantize_blockwise(W, 64, 1, oracle.FMT_AFFINE_MINMAX, nbits=bits)
+    Wt = oracle.dequantize(qw)
+    ad = oracle.Adapter(l1, l2, r, 1.0, A, B)
+    ad.scaling = visible_scaling(Wt, ad, X)
+    dq = qb.quantize_minmax_nbit(to_dev(W), bits)
+    da, Xd, dYd = adapter_to_dev(ad), to_bf16_dev(X), to_bf16_dev(dY)
+    gate_strict(to_np64(qb.linear_fwd(dq, da, Xd, torch.float32)), oracle.linear_fwd(Wt, ad, X), "Y f32")
+    rdX, rdA, rdB = oracle.linear_bwd(Wt, ad, X, dY)
+    dX, dA, dB = qb.linear_bwd(dq, da, Xd, dYd, torch.float32)
+    gate_strict(to_np64(dX), rdX, "dX f32")
+    gate_strict(to_np64(dA), rdA, "dA", per_row=False)
+    gate_strict(to_np64(dB), rdB, "dB", per_row=False)
+    merged = qb.merge(dq, da)
+    assert np.array_equal(merged.beta.cpu().numpy(), oracle.merge(qw, ad).beta)
+    # (token counts as in the 4-bit merge-identity test: the merged operand carries the adapter inside the
+    # bf16-rounded weight, so with only 7 pooled inputs rows with a small adapter term see a larger relative error)
+    for Tl in (1, 16, 40):
+        gate_strict(to_np64(qb.lowbit_gemm(merged, Xd[:Tl].contiguous(), torch.float32)),
+                    oracle.linear_fwd(Wt, ad, X[:Tl]), f"merged low-bit product T={Tl}")
+
+
+def test_nbit_rejects_bad_width(qb):
+    W = to_dev(synth.normal(83, "nbit/bad", (8, 64), 0.02))
+    for bits in (0, 5):
+        with pytest.raises(qb.QbloraError) as e:
+            qb.quantize_minmax_nbit(W, bits)
+        assert e.value.status == qb.ERR_INVALID_ARG
