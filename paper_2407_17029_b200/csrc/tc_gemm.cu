@@ -173,6 +173,7 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
+      bool adapter_input_ready = false;
       for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
         const int m0 = (tile % p.m_tiles) * (2 * BM) + (int)rank * BM;
         const int t0 = (tile / p.m_tiles) * BN + (int)rank * BN_HALF;
@@ -190,6 +191,13 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
               tma_load_2d(sP + s * P_BYTES + P_BYTES / 2, &tm_p, full(s), m0 / 2 + 32, kb * BK);
             }
           } else {
+            // The compressed adapter activation is written by the kernel launched just before this one.  With the
+            // programmatic-dependent launch this grid started while that kernel was still running (everything up
+            // to here reads only the caller's inputs); its result is complete and visible after this wait.
+            if (!adapter_input_ready) {
+              asm volatile("griddepcontrol.wait;" ::: "memory");
+              adapter_input_ready = true;
+            }
             mbar_arrive_expect_tx(full(s), B_BYTES);
             tma_load_2d(sB + s * B_BYTES, &tm_bx, full(s), (kb - p.kb_base) * BK, t0);
           }
@@ -462,6 +470,7 @@ template <bool DIVIDE>
 __global__ void __launch_bounds__(256) segsum_split_kernel(const __nv_bfloat16* __restrict__ src, int64_t rows, int width,
                                                            int lam, float scale, int ld_out,
                                                            __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the small product that follows may set up now
   constexpr int UNROLL = 4;       // 16-byte loads in flight per thread (the kernel is a pure stream)
   const int chunks_per_row = width >> 3;
   const int64_t total = rows * chunks_per_row;
@@ -519,6 +528,7 @@ inline bool segsum_fast_ok(int width, int lam) {
 // x'[t][p] = AvgPool_{lambda_in}(X) (Sec. 3.2) as a bf16 hi + lo pair (hi + lo carries ~16 mantissa bits)
 __global__ void pool_split_kernel(const __nv_bfloat16* __restrict__ X, int64_t T, int d_in, int l1, int ldp,
                                   __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the small product that follows may set up now
   const int P = d_in / l1;
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= T * P) return;
@@ -540,6 +550,7 @@ __global__ void pool_split_kernel(const __nv_bfloat16* __restrict__ X, int64_t T
 // dv[t][q] = s * sum of lambda_out consecutive output gradients (adjoint of repeat_interleave), hi + lo
 __global__ void dv_split_kernel(const __nv_bfloat16* __restrict__ dY, int64_t T, int d_out, int l2, float scaling,
                                 int ldq, __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the small product that follows may set up now
   const int Q = d_out / l2;
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= T * Q) return;
@@ -563,6 +574,7 @@ __global__ void dv_split_kernel(const __nv_bfloat16* __restrict__ dY, int64_t T,
 // (stride 1 = truncation, lambda = interval sampling; scale = 1 for x', s for dv), stored as a hi + lo pair.
 __global__ void sample_split_kernel(const __nv_bfloat16* __restrict__ src, int64_t T, int width, int n_small, int stride,
                                     float scale, int ld_out, __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the small product that follows may set up now
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= T * n_small) return;
   const int64_t t = idx / n_small; const int j = (int)(idx - t * n_small);
@@ -608,6 +620,12 @@ TcWs carve(int op, const AdView* ad, int64_t T, char* ws) {
   }
   w.bytes = off;
   return w;
+}
+
+// QBLORA_NO_PDL=1 launches the fused contraction as an ordinary kernel (for A/B timing).
+bool overlap_adapter_prologue() {
+  static const bool on = []() { const char* v = getenv("QBLORA_NO_PDL"); return !(v && v[0] == '1'); }();
+  return on;
 }
 
 // Launches the fused-dequant GEMM.  Bop: X (forward) / dY (backward); Bx: the compressed adapter
@@ -656,12 +674,24 @@ int launch_main(int mode, const QwView& qw, const AdView* ad, const __nv_bfloat1
   const int tiles = p.m_tiles * p.n_tiles;                      // one tile per CTA pair
   const int pairs = num_sms() / 2;
   const int grid = 2 * (tiles < pairs ? tiles : pairs);
+  // With an adapter the kernel in front of this one on the stream is the small product that writes Bx, and only
+  // the last K-blocks of a tile read it: launch as its programmatic dependent, so that the weight K-blocks run
+  // while that product finishes (the producer warp waits for it before the first adapter K-block).  Without an
+  // adapter the predecessor is the caller's own work and the launch is an ordinary one.
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(NUM_THREADS); cfg.dynamicSmemBytes = SMEM_BYTES; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = (ad && overlap_adapter_prologue()) ? 1 : 0;
+  cudaError_t le;
   {
     DominantKernelTimer timer(st);
-    if (mode == 0) tc_dq_gemm_kernel<0><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(tm_b, tm_bx, tm_p, p);
-    else tc_dq_gemm_kernel<1><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(tm_b, tm_bx, tm_p, p);
+    le = mode == 0 ? cudaLaunchKernelEx(&cfg, tc_dq_gemm_kernel<0>, tm_b, tm_bx, tm_p, p)
+                   : cudaLaunchKernelEx(&cfg, tc_dq_gemm_kernel<1>, tm_b, tm_bx, tm_p, p);
     count_launch();
   }
+  QB_CUDA(le);
   QB_CUDA(cudaGetLastError());
   return QBLORA_OK;
 }
@@ -686,7 +716,8 @@ int launch_pool(const QwView& qw, const AdView& ad, const __nv_bfloat16* X, int6
 int launch_u_gemm(const AdView& ad, int64_t T, const TcWs& w, const SgOut& out, int* status, cudaStream_t st) {
   const SgOperand a_mat{ad.A, ad.r, false};   // (n = rank index, k = p) at A[k * r + n]
   SgSegment segs[2] = {{{w.xh, w.ldp, true}, a_mat, ad.P}, {{w.xl, w.ldp, true}, a_mat, ad.P}};
-  return small_gemm((int)T, ad.r, segs, 2, out, status, st);
+  // directly behind the compression kernel on the same stream: its programmatic dependent
+  return small_gemm((int)T, ad.r, segs, 2, out, status, st, nullptr, overlap_adapter_prologue());
 }
 
 }  // namespace
@@ -782,7 +813,7 @@ int tc_linear_bwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, co
       SgOut out{};
       out.hi = w.duh; out.lo = w.dul; out.scaled = w.du16; out.ld16 = w.ldr; out.divide = true;
       out.scale = ad->op == QBLORA_SCALE_AVGPOOL_REPEAT ? (float)ad->l1 : 1.0f;   // only the average carries 1 / lambda_in
-      rc = small_gemm((int)T, ad->r, segs, 2, out, status, st);
+      rc = small_gemm((int)T, ad->r, segs, 2, out, status, st, nullptr, overlap_adapter_prologue());   // behind dv's kernel
       if (rc) return rc;
     }
     if (lane) QB_CUDA(cudaEventRecord(lane->du_done, st));

@@ -29,8 +29,11 @@ struct SgOut {
 // All segments must use the same operand majors.  `status` = device status word (bounded waits).
 // `partial` (optional, fp32 output only): scratch of small_gemm_splits(M, N, K) * M * N floats; the
 // contraction is then split over that many CTAs per output tile and summed in a fixed order.
+// `dependent`: the kernel in front of this one on `st` is one of this library's that signals
+// griddepcontrol.launch_dependents and writes an operand; this product is then launched as its programmatic
+// dependent (set-up overlaps that kernel's tail; the operand loads wait for its completion).
 int small_gemm(int M, int N, const SgSegment* segs, int nseg, const SgOut& out, int* status, cudaStream_t st,
-               float* partial = nullptr);
+               float* partial = nullptr, bool dependent = false);
 int small_gemm_splits(int M, int N, int K);
 
 // Encodes a 2-D tensor map (shared with the main kernel's host code).

@@ -43,6 +43,10 @@ small_gemm_kernel(const __grid_constant__ SgMaps maps, const __grid_constant__ S
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int m0 = blockIdx.y * SG_BM, n0 = blockIdx.x * p.bn;
+  // A successor launched as a programmatic dependent (the fused contraction, which needs this product only for
+  // its last K-blocks) may start now; it waits for this grid's completion before it reads the result.
+  // No effect on ordinary successors.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (tid == 0) {
     for (int s = 0; s < SG_STAGES; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
     mbar_init(accfull, 1);
@@ -62,6 +66,8 @@ small_gemm_kernel(const __grid_constant__ SgMaps maps, const __grid_constant__ S
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
+      // launched as a programmatic dependent of the kernel that writes an operand: that kernel is complete after this
+      asm volatile("griddepcontrol.wait;" ::: "memory");
       for (int g = 0; g < p.nseg && ok; ++g) {
         const int per = (p.kblocks[g] + p.splits - 1) / p.splits;
         const int kb0 = (int)blockIdx.z * per, kb1 = min(kb0 + per, p.kblocks[g]);
@@ -97,6 +103,8 @@ small_gemm_kernel(const __grid_constant__ SgMaps maps, const __grid_constant__ S
                              ((uint32_t)(SG_BM >> 4) << 24);
       uint32_t it = 0;
       bool ok = true;
+      // launched as a programmatic dependent of the kernel that writes an operand: that kernel is complete after this
+      asm volatile("griddepcontrol.wait;" ::: "memory");
       for (int g = 0; g < p.nseg && ok; ++g) {
         const int per = (p.kblocks[g] + p.splits - 1) / p.splits;
         const int kb0 = (int)blockIdx.z * per, kb1 = min(kb0 + per, p.kblocks[g]);
@@ -269,7 +277,7 @@ int small_gemm_splits(int M, int N, int K) {
 }
 
 int small_gemm(int M, int N, const SgSegment* segs, int nseg, const SgOut& out, int* status, cudaStream_t st,
-               float* partial) {
+               float* partial, bool dependent) {
   if (nseg < 1 || nseg > SG_MAX_SEG || M < 1 || N < 1) return QBLORA_ERR_INVALID_ARG;
   static bool attr_set = false;
   if (!attr_set) {
@@ -310,7 +318,13 @@ int small_gemm(int M, int N, const SgSegment* segs, int nseg, const SgOut& out, 
     }
   }
   dim3 grid((unsigned)((N + p.bn - 1) / p.bn), (unsigned)((M + SG_BM - 1) / SG_BM), (unsigned)p.splits);
-  small_gemm_kernel<<<grid, SG_THREADS, SG_SMEM, st>>>(maps, p);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = dim3(SG_THREADS); cfg.dynamicSmemBytes = SG_SMEM; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = dependent ? 1 : 0;
+  QB_CUDA(cudaLaunchKernelEx(&cfg, small_gemm_kernel, maps, p));
   count_launch();
   QB_CUDA(cudaGetLastError());
   if (p.splits > 1) {
