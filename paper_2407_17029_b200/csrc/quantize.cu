@@ -24,9 +24,16 @@ __device__ __forceinline__ int code_of_level(float v, const QuantTable& t) {
   return c;
 }
 
-__device__ __forceinline__ int code_of_affine(float w, float beta, float alpha, float qmax) {
-  float q = __fdiv_rn(__fsub_rn(w, beta), alpha);
-  float rq = rintf(q);  // ties to even
+// code = clamp(rint(fl32(fl32(w - beta) / alpha)), 0, qmax), ties to even (Eq. 1), without a division per element.
+// inv = fl32(1 / alpha).  qa = fl32(x * inv) is within 2^-23 relative of the exact quotient x / alpha, and so is
+// fl32(x / alpha) (within 2^-24); the quotient is at most 15, so both lie within 2e-6 of it.  When qa is farther
+// than 1e-5 from every half-integer, rint(qa) and rint(fl32(x / alpha)) are therefore the same integer.  Otherwise
+// (about one element in 10^5, and whenever inv overflowed or qa is not finite) the exact quotient decides.
+__device__ __forceinline__ int code_of_affine(float w, float beta, float alpha, float inv, float qmax) {
+  const float x = __fsub_rn(w, beta);
+  const float qa = __fmul_rn(x, inv);
+  float rq = rintf(qa);
+  if (!(fabsf(__fsub_rn(qa, rq)) < 0.49999f)) rq = rintf(__fdiv_rn(x, alpha));   // ties to even on the exact quotient
   rq = fminf(fmaxf(rq, 0.0f), qmax);
   return (int)rq;
 }
@@ -84,9 +91,10 @@ __global__ void __launch_bounds__(256) quantize_b64_kernel(const TIn* __restrict
       const float d = __fsub_rn(mx, mn);
       const float a = __fdiv_rn(d, tab.qmax);
       const bool degenerate = (d == 0.0f) || (a == 0.0f);
+      const float inv = __frcp_rn(a);
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
-        const int c = degenerate ? 0 : code_of_affine(v[e], mn, a, tab.qmax);
+        const int c = degenerate ? 0 : code_of_affine(v[e], mn, a, inv, tab.qmax);
         packed |= (uint32_t)c << (4 * e);
       }
       if (live && part == 0) {
@@ -127,6 +135,7 @@ __global__ void quantize_generic_kernel(const TIn* __restrict__ W, int d_out, in
     alpha[b] = degenerate ? 0.0f : a;
     beta[b] = mn;
   }
+  const float inv = __frcp_rn(a);
   for (int o = o0; o < o0 + block_out; ++o)
     for (int i = i0; i < i0 + block_in; i += 2) {
       int c[2];
@@ -136,7 +145,7 @@ __global__ void quantize_generic_kernel(const TIn* __restrict__ W, int d_out, in
         if (qfmt == QBLORA_FMT_CODEBOOK_ABSMAX)
           c[e] = degenerate ? tab.zero_idx : code_of_level(__fdiv_rn(w, am), tab);
         else
-          c[e] = degenerate ? 0 : code_of_affine(w, mn, a, tab.qmax);
+          c[e] = degenerate ? 0 : code_of_affine(w, mn, a, inv, tab.qmax);
       }
       codes[(int64_t)o * (d_in / 2) + i / 2] = (uint8_t)(c[0] | (c[1] << 4));
     }

@@ -77,3 +77,30 @@ def test_nbit_rejects_bad_width(qb):
         with pytest.raises(qb.QbloraError) as e:
             qb.quantize_minmax_nbit(W, bits)
         assert e.value.status == qb.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("bits", [2, 4])
+def test_quantize_ties_and_near_ties_bit_exact(qb, bits):
+    # values on and within a few ulps of the rounding boundaries k + 1/2 of Eq. 1's grid: the library decides
+    # these with the exact quotient, everything else without a division; both must agree with the oracle
+    qmax = (1 << bits) - 1
+    rng = np.random.Generator(np.random.Philox(key=84))
+    rows = []
+    for trial in range(256):
+        alpha = np.float32(0.125) if trial % 4 == 0 else np.float32(rng.uniform(1e-3, 0.3))
+        beta = np.float32(0.0) if trial % 4 == 0 else np.float32(rng.normal(0, 0.05))
+        k = rng.integers(0, qmax, size=62)
+        w = (beta + alpha * (k.astype(np.float32) + np.float32(0.5))).astype(np.float32)
+        for step in range(int(rng.integers(0, 4))):                       # 0..3 ulps off the boundary, either way
+            w = np.nextafter(w, np.float32(np.inf if trial % 2 else -np.inf))
+        row = np.concatenate([[beta, np.float32(beta + alpha * qmax)], w]).astype(np.float32)   # pins min and max
+        rows.append(row)
+    W = np.stack(rows)
+    ref = oracle.quantize_blockwise(W, 64, 1, oracle.FMT_AFFINE_MINMAX, nbits=bits)
+    got = qb.quantize_minmax_nbit(to_dev(W), bits)
+    assert np.array_equal(got.alpha.cpu().numpy().view(np.uint32), ref.alpha.view(np.uint32))
+    assert np.array_equal(got.beta.cpu().numpy().view(np.uint32), ref.beta.view(np.uint32))
+    assert np.array_equal(got.codes.cpu().numpy(), ref.codes)
+    # the case is what it claims to be: a good share of the elements sits within 1e-5 of a boundary
+    q = (W.astype(np.float64) - ref.beta.astype(np.float64)) / ref.alpha.astype(np.float64)
+    assert np.mean(np.abs(q - np.floor(q) - 0.5) < 1e-5) > 0.5
