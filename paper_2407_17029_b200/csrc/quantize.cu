@@ -32,10 +32,13 @@ __device__ __forceinline__ int code_of_level(float v, const QuantTable& t) {
 __device__ __forceinline__ int code_of_affine(float w, float beta, float alpha, float inv, float qmax) {
   const float x = __fsub_rn(w, beta);
   const float qa = __fmul_rn(x, inv);
-  float rq = rintf(qa);
-  if (!(fabsf(__fsub_rn(qa, rq)) < 0.49999f)) rq = rintf(__fdiv_rn(x, alpha));   // ties to even on the exact quotient
-  rq = fminf(fmaxf(rq, 0.0f), qmax);
-  return (int)rq;
+  // adding 2^23 rounds qa (0 <= qa < 16) to the nearest integer, ties to even, and leaves that integer in the low
+  // mantissa bits; x lies in [0, max - min], so the integer is already inside [0, qmax] and needs no clamp
+  const float m = __fadd_rn(qa, 8388608.0f);
+  const float rq = __fsub_rn(m, 8388608.0f);
+  if (fabsf(__fsub_rn(qa, rq)) < 0.49999f) return (int)(__float_as_uint(m) & 15u);
+  // near a rounding boundary, or qa not finite: the exact quotient decides (ties to even), with the clamp of Eq. 1
+  return (int)fminf(fmaxf(rintf(__fdiv_rn(x, alpha)), 0.0f), qmax);
 }
 
 // block_in == 64, block_out == 1.  Because d_in is a multiple of 64, block b is the flat element range
