@@ -466,12 +466,17 @@ __device__ __forceinline__ void store_split(float x, __nv_bfloat16* hi, __nv_bfl
 // (AvgPool) or *scale (adjoint of repeat_interleave), written as a bf16 hi + lo pair.  One 16-byte load
 // (8 elements) per thread; windows wider than a chunk are finished with warp shuffles.  Needs width % 8
 // == 0 and lam in {1, 2, 4} or 8 * 2^k <= 256 with chunks-per-row % (lam / 8) == 0 (true when lam | width).
+// 16-byte loads in flight per thread.  Two, at 32 registers per thread, measured best inside a step (C2 forward
+// call 110 -> 107 us against four loads at 48 registers, 113 us with eight, 109 us with one): a 256-thread CTA of
+// this kernel then fits on an SM beside a CTA of the fused contraction (448 x 128 registers), so the contraction,
+// launched as a programmatic dependent further down the chain, can move in while the last CTAs here drain.
+constexpr int SEGSUM_UNROLL = 2;
 template <bool DIVIDE>
-__global__ void __launch_bounds__(256) segsum_split_kernel(const __nv_bfloat16* __restrict__ src, int64_t rows, int width,
+__global__ void __launch_bounds__(256, 8) segsum_split_kernel(const __nv_bfloat16* __restrict__ src, int64_t rows, int width,
                                                            int lam, float scale, int ld_out,
                                                            __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the small product that follows may set up now
-  constexpr int UNROLL = 4;       // 16-byte loads in flight per thread (the kernel is a pure stream)
+  constexpr int UNROLL = SEGSUM_UNROLL;   // 16-byte loads in flight per thread (the kernel is a pure stream)
   const int chunks_per_row = width >> 3;
   const int64_t total = rows * chunks_per_row;
   uint4 q4[UNROLL];
@@ -703,7 +708,7 @@ int launch_pool(const QwView& qw, const AdView& ad, const __nv_bfloat16* X, int6
         X, T, qw.d_in, ad.P, ad.op == QBLORA_SCALE_TRUNCATE_ZEROPAD ? 1 : ad.l1, 1.0f, w.ldp, w.xh, w.xl);
   } else if (segsum_fast_ok(qw.d_in, ad.l1)) {
     const int64_t chunks = T * (qw.d_in / 8);
-    segsum_split_kernel<true><<<(unsigned)((chunks + 1023) / 1024), 256, 0, st>>>(X, T, qw.d_in, ad.l1, 0.0f, w.ldp, w.xh, w.xl);
+    segsum_split_kernel<true><<<(unsigned)((chunks + 256 * SEGSUM_UNROLL - 1) / (256 * SEGSUM_UNROLL)), 256, 0, st>>>(X, T, qw.d_in, ad.l1, 0.0f, w.ldp, w.xh, w.xl);
   } else {
     pool_split_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(X, T, qw.d_in, ad.l1, w.ldp, w.xh, w.xl);
   }
@@ -801,7 +806,7 @@ int tc_linear_bwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, co
           dY, T, qw.d_out, ad->Q, ad->op == QBLORA_SCALE_TRUNCATE_ZEROPAD ? 1 : ad->l2, ad->s, w.ldq, w.dvh, w.dvl);
     } else if (segsum_fast_ok(qw.d_out, ad->l2)) {
       const int64_t chunks = T * (qw.d_out / 8);
-      segsum_split_kernel<false><<<(unsigned)((chunks + 1023) / 1024), 256, 0, st>>>(dY, T, qw.d_out, ad->l2, ad->s, w.ldq, w.dvh, w.dvl);
+      segsum_split_kernel<false><<<(unsigned)((chunks + 256 * SEGSUM_UNROLL - 1) / (256 * SEGSUM_UNROLL)), 256, 0, st>>>(dY, T, qw.d_out, ad->l2, ad->s, w.ldq, w.dvh, w.dvl);
     } else {
       dv_split_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(dY, T, qw.d_out, ad->l2, ad->s, w.ldq, w.dvh, w.dvl);
     }
