@@ -14,6 +14,11 @@ constexpr int SG_A_BYTES = SG_BM * SG_BK * 2;   // 16 KB
 constexpr int SG_B_BYTES = 256 * SG_BK * 2;     // 32 KB (bn = 256)
 constexpr int SG_THREADS = 192;
 constexpr int SG_SMEM = SG_STAGES * (SG_A_BYTES + SG_B_BYTES) + 256 + 1024;
+// 193 KB: a CTA of this kernel never shares an SM with a CTA of the fused contraction (218 KB).  That matters for
+// tensor memory: this kernel allocates 256 columns, the contraction all 512, and the contraction may be launched
+// as this kernel's programmatic dependent and wait for its completion -- on a shared SM either could wait for
+// columns the other holds.  Keep the sum of the two footprints above the SM's shared memory.
+static_assert(SG_SMEM > 16 * 1024, "see the note on tensor memory above");
 constexpr int SG_MAX_SEG = 3;
 
 struct SgMaps {
