@@ -24,6 +24,24 @@ __device__ __forceinline__ int code_of_level(float v, const QuantTable& t) {
   return c;
 }
 
+// Level-table code without a division per element: code = #{ j : fl32(w / absmax) > mid_j }.
+// va = fl32(w * fl32(1 / absmax)) is within 1.2e-7 of the exact quotient (|quotient| <= 1), the rounded quotient
+// within 6e-8, and a comparison with mid_j can only differ between the two when the exact quotient lies within one
+// ulp of mid_j.  So the position of va among the midpoints (binary search in a shared-memory copy, s_mid[0] = -inf,
+// s_mid[1 + j] = mid_j, s_mid[16] = +inf) is the code whenever va is farther than 1e-6 from both neighbouring
+// midpoints; otherwise (and for a non-finite va) the exact quotient is compared with all fifteen as before.
+__device__ __forceinline__ int code_of_level_fast(float w, float absmax, float inv, const float* s_mid, const QuantTable& t) {
+  const float va = __fmul_rn(w, inv);
+  int k = 0;
+  k += (va > s_mid[k + 8]) ? 8 : 0;
+  k += (va > s_mid[k + 4]) ? 4 : 0;
+  k += (va > s_mid[k + 2]) ? 2 : 0;
+  k += (va > s_mid[k + 1]) ? 1 : 0;
+  const float lo = s_mid[k], hi = s_mid[k + 1];
+  if ((__fsub_rn(va, lo) > 1e-6f) && (__fsub_rn(hi, va) > 1e-6f)) return k;
+  return code_of_level(__fdiv_rn(w, absmax), t);
+}
+
 // code = clamp(rint(fl32(fl32(w - beta) / alpha)), 0, qmax), ties to even (Eq. 1), without a division per element.
 // inv = fl32(1 / alpha).  qa = fl32(x * inv) is within 2^-23 relative of the exact quotient x / alpha, and so is
 // fl32(x / alpha) (within 2^-24); the quotient is at most 15, so both lie within 2e-6 of it.  When qa is farther
@@ -52,6 +70,10 @@ __global__ void __launch_bounds__(256) quantize_b64_kernel(const TIn* __restrict
                                                            uint8_t* __restrict__ codes,
                                                            float* __restrict__ alpha,
                                                            float* __restrict__ beta) {
+  __shared__ float s_mid[17];
+  if (threadIdx.x < 17)
+    s_mid[threadIdx.x] = threadIdx.x == 0 ? -INFINITY : threadIdx.x == 16 ? INFINITY : tab.mid[min(max((int)threadIdx.x, 1), 15) - 1];
+  __syncthreads();
   const int lane = threadIdx.x & 31, sub = lane >> 3, part = lane & 7;
   const int64_t warps_per_grid = (int64_t)gridDim.x * (blockDim.x >> 5);
   const int64_t steps = (nblocks + 3) >> 2;
@@ -84,9 +106,10 @@ __global__ void __launch_bounds__(256) quantize_b64_kernel(const TIn* __restrict
     }
     uint32_t packed = 0;
     if (qfmt == QBLORA_FMT_CODEBOOK_ABSMAX) {
+      const float inv = __frcp_rn(am);
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
-        const int c = am != 0.0f ? code_of_level(__fdiv_rn(v[e], am), tab) : tab.zero_idx;
+        const int c = am != 0.0f ? code_of_level_fast(v[e], am, inv, s_mid, tab) : tab.zero_idx;
         packed |= (uint32_t)c << (4 * e);
       }
       if (live && part == 0) alpha[b] = am;

@@ -104,3 +104,29 @@ def test_quantize_ties_and_near_ties_bit_exact(qb, bits):
     # the case is what it claims to be: a good share of the elements sits within 1e-5 of a boundary
     q = (W.astype(np.float64) - ref.beta.astype(np.float64)) / ref.alpha.astype(np.float64)
     assert np.mean(np.abs(q - np.floor(q) - 0.5) < 1e-5) > 0.5
+
+
+def test_quantize_level_table_near_midpoints_bit_exact(qb):
+    # level-table format: elements whose quotient w / absmax sits on or within a few ulps of a midpoint between
+    # two levels (decided by the exact quotient in the library), mixed with ordinary ones
+    rng = np.random.Generator(np.random.Philox(key=85))
+    t = oracle.default_code_table().astype(np.float64)
+    mids = ((t[:-1] + t[1:]) / 2).astype(np.float32)
+    rows = []
+    for trial in range(256):
+        a = np.float32(0.5) if trial % 4 == 0 else np.float32(rng.uniform(1e-3, 0.3))
+        j = rng.integers(0, 15, size=63)
+        w = (a * mids[j]).astype(np.float32)
+        for step in range(int(rng.integers(0, 4))):
+            w = np.nextafter(w, np.float32(np.inf if trial % 2 else -np.inf))
+        sign = np.float32(1.0 if trial % 3 else -1.0)
+        rows.append(np.concatenate([[sign * a], w]).astype(np.float32))           # pins absmax
+    W = np.stack(rows)
+    W[::7, 1:] = synth.normal(85, "lvl/plain", (len(W[::7]), 63), 0.02).clip(-1e-3, 1e-3)
+    ref = oracle.quantize_blockwise(W, 64, 1, oracle.FMT_CODEBOOK_ABSMAX)
+    got = qb.quantize_blockwise(to_dev(W), 64, 1, qb.FMT_CODEBOOK_ABSMAX)
+    assert np.array_equal(got.alpha.cpu().numpy().view(np.uint32), ref.alpha.view(np.uint32))
+    assert np.array_equal(got.codes.cpu().numpy(), ref.codes)
+    v = W.astype(np.float64) / ref.alpha.astype(np.float64)
+    near = np.abs(v[..., None] - mids.astype(np.float64)).min(axis=-1) < 1e-6
+    assert near.mean() > 0.5
