@@ -327,3 +327,37 @@ def test_dense_16bit_merge(qb, case):
     assert np.all(np.abs(base - Wt) <= 2.0 ** -8 * np.abs(Wt) + 1e-30)
     Y = torch.matmul(to_bf16_dev(X).float(), qb.merge_dense(dq, da).float().t())
     gate_strict(to_np64(Y), oracle.linear_fwd(Wt, ad, X), "X W'^T vs adapted forward")
+
+
+@pytest.mark.parametrize("shape", [(300, 320, 448, 64, 8, 48), (2048, 1024, 1024, 64, 8, 64), (515, 256, 640, 4, 4, 64)])
+def test_back_to_back_calls_through_one_workspace_do_not_see_stale_adapter_inputs(qb, shape):
+    # The fused contraction starts before the small adapter products in front of it have finished and waits for
+    # them only where it needs their result.  Alternate two different inputs through ONE workspace, back to back
+    # with no host synchronisation in between: a contraction that read the compressed adapter activation too
+    # early would pick up the other input's values.  Every result must equal, bit for bit, the one computed alone.
+    T, d_out, d_in, l1, l2, r = shape
+    qw, ad, X0, dY0 = make_case(91, T, d_out, d_in, l1, l2, r)
+    _, _, X1, dY1 = make_case(92, T, d_out, d_in, l1, l2, r)
+    ad.scaling = 30.0                                     # the adapter term is a large part of every output
+    dq, da = qweight_to_dev(qw), adapter_to_dev(ad)
+    Xs, dYs = [to_bf16_dev(X0), to_bf16_dev(X1)], [to_bf16_dev(dY0), to_bf16_dev(dY1)]
+    wf = qb.alloc_workspace(qb.OP_LINEAR_FWD, dq, da, T)
+    wb = qb.alloc_workspace(qb.OP_LINEAR_BWD, dq, da, T)
+    alone = []
+    for k in range(2):
+        Y = qb.linear_fwd(dq, da, Xs[k], torch.float32, ws=wf)
+        dX, dA, dB = qb.linear_bwd(dq, da, Xs[k], dYs[k], torch.float32, ws=wb)
+        torch.cuda.synchronize()
+        alone.append((Y.clone(), dX.clone(), dA.clone(), dB.clone()))
+    assert not torch.equal(alone[0][0], alone[1][0])
+    results = []
+    for it in range(60):
+        k = it & 1
+        Y = qb.linear_fwd(dq, da, Xs[k], torch.float32, ws=wf)
+        dX, dA, dB = qb.linear_bwd(dq, da, Xs[k], dYs[k], torch.float32, ws=wb)
+        results.append((k, Y, dX, dA, dB))
+    torch.cuda.synchronize()
+    for k, Y, dX, dA, dB in results:
+        assert torch.equal(Y, alone[k][0]) and torch.equal(dX, alone[k][1])
+        assert torch.equal(dA, alone[k][2]) and torch.equal(dB, alone[k][3])
+    assert qb.device_status(wf) == 0 and qb.device_status(wb) == 0
