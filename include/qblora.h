@@ -36,7 +36,7 @@ extern "C" {
 typedef enum {
   QBLORA_OK = 0,
   QBLORA_ERR_INVALID_ARG = 1, /* null / misaligned pointer, sizes that do not divide, tokens < 1 */
-  QBLORA_ERR_UNSUPPORTED = 2, /* valid request this build has no kernel for */
+  QBLORA_ERR_UNSUPPORTED = 2, /* valid request the library has no kernel for */
   QBLORA_ERR_WORKSPACE = 3,   /* ws == NULL or ws_bytes too small */
   QBLORA_ERR_CUDA = 4,        /* a CUDA runtime call or launch failed */
   QBLORA_ERR_TIMEOUT = 5,     /* a bounded device-side wait gave up (see qblora_device_status) */
