@@ -96,3 +96,31 @@ def test_workspace_bytes_and_merge_alignment_rule(lib):
     rc = lib.qablora_merge(ctypes.byref(q), ctypes.byref(a), ctypes.c_void_p(0x1000), ctypes.c_void_p(0x1000),
                            ctypes.c_size_t(1 << 30), None)
     assert rc == qb.ERR_INVALID_ARG
+
+
+def test_binding_struct_layouts_match_the_header(tmp_path):
+    # the header is plain C: compile a probe against it and compare sizes and member offsets with the ctypes mirrors
+    import subprocess
+    from paper_2407_17029_b200 import binding
+    members = {"qblora_qweight": ["d_in", "d_out", "block_in", "block_out", "qfmt", "code", "codes", "alpha", "beta"],
+               "qblora_adapter": ["lambda_in", "lambda_out", "rank", "scaling", "A", "B", "scale_op"]}
+    lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "qblora.h"', 'int main(void) {']
+    for s, ms in members.items():
+        lines.append(f'  printf("{s} %zu\\n", sizeof({s}));')
+        for m in ms:
+            lines.append(f'  printf("{s}.{m} %zu\\n", offsetof({s}, {m}));')
+    lines += ['  printf("enum %d %d %d\\n", QBLORA_SCALE_AVGPOOL_REPEAT, QBLORA_SCALE_TRUNCATE_ZEROPAD, QBLORA_SCALE_SAMPLE_ZEROFILL);',
+              '  return 0;', '}']
+    src = tmp_path / "probe.c"
+    src.write_text("\n".join(lines))
+    exe = tmp_path / "probe"
+    subprocess.run(["gcc", "-std=c99", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)], check=True)
+    out = dict(l.split(" ", 1) for l in subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.splitlines())
+    mirrors = {"qblora_qweight": binding._CQWeight, "qblora_adapter": binding._CAdapter}
+    for s, ms in members.items():
+        assert int(out[s]) == ctypes.sizeof(mirrors[s])
+        assert [f[0] for f in mirrors[s]._fields_] == ms
+        for m in ms:
+            assert int(out[f"{s}.{m}"]) == getattr(mirrors[s], m).offset, (s, m)
+    assert out["enum"].split() == [str(binding.SCALE_AVGPOOL_REPEAT), str(binding.SCALE_TRUNCATE_ZEROPAD),
+                                   str(binding.SCALE_SAMPLE_ZEROFILL)]
