@@ -361,3 +361,44 @@ def test_back_to_back_calls_through_one_workspace_do_not_see_stale_adapter_input
         assert torch.equal(Y, alone[k][0]) and torch.equal(dX, alone[k][1])
         assert torch.equal(dA, alone[k][2]) and torch.equal(dB, alone[k][3])
     assert qb.device_status(wf) == 0 and qb.device_status(wb) == 0
+
+
+def test_cuda_graph_replay_equals_eager_calls(qb):
+    # forward + backward captured once through the C ABI (side stream, programmatic-dependent launches and all) and
+    # replayed on changing inputs in static buffers: every replay equals the eager result for the same input
+    T, d_out, d_in, l1, l2, r = 515, 256, 640, 64, 8, 64
+    qw, ad, X0, dY0 = make_case(93, T, d_out, d_in, l1, l2, r)
+    _, _, X1, dY1 = make_case(94, T, d_out, d_in, l1, l2, r)
+    ad.scaling = 30.0
+    dq, da = qweight_to_dev(qw), adapter_to_dev(ad)
+    ins = [(to_bf16_dev(X0), to_bf16_dev(dY0)), (to_bf16_dev(X1), to_bf16_dev(dY1))]
+    wf = qb.alloc_workspace(qb.OP_LINEAR_FWD, dq, da, T)
+    wb = qb.alloc_workspace(qb.OP_LINEAR_BWD, dq, da, T)
+    eager = []
+    for X, dY in ins:
+        Y = qb.linear_fwd(dq, da, X, torch.bfloat16, ws=wf)
+        dX, dA, dB = qb.linear_bwd(dq, da, X, dY, torch.bfloat16, ws=wb)
+        torch.cuda.synchronize()
+        eager.append((Y.clone(), dX.clone(), dA.clone(), dB.clone()))
+    Xs, dYs = torch.empty_like(ins[0][0]), torch.empty_like(ins[0][1])
+    Y = torch.empty((T, d_out), dtype=torch.bfloat16, device=Xs.device)
+    dX = torch.empty((T, d_in), dtype=torch.bfloat16, device=Xs.device)
+    dA, dB = torch.empty_like(eager[0][2]), torch.empty_like(eager[0][3])
+    st = torch.cuda.Stream()
+    with torch.cuda.stream(st):
+        Xs.copy_(ins[0][0]); dYs.copy_(ins[0][1])
+        qb.linear_fwd(dq, da, Xs, ws=wf, out=Y)                       # warm-up outside the capture (lazy set-up)
+        qb.linear_bwd(dq, da, Xs, dYs, ws=wb, outs=(dX, dA, dB))
+        st.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=st):
+            qb.linear_fwd(dq, da, Xs, ws=wf, out=Y)
+            qb.linear_bwd(dq, da, Xs, dYs, ws=wb, outs=(dX, dA, dB))
+        for it in range(12):
+            k = it & 1
+            Xs.copy_(ins[k][0]); dYs.copy_(ins[k][1])
+            g.replay()
+            st.synchronize()
+            assert torch.equal(Y, eager[k][0]) and torch.equal(dX, eager[k][1]), f"replay {it}"
+            assert torch.equal(dA, eager[k][2]) and torch.equal(dB, eager[k][3]), f"replay {it}"
+    assert qb.device_status(wf) == 0 and qb.device_status(wb) == 0
