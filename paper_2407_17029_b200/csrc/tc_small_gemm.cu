@@ -274,7 +274,9 @@ int small_gemm_splits(int M, int N, int K) {
   const int tiles = ((N + bn - 1) / bn) * ((M + SG_BM - 1) / SG_BM);
   const int kb = (K + SG_BK - 1) / SG_BK;
   int want = 148 / tiles;
-  if (want > 32) want = 32;
+  // at most 16 shares: the gradient products run beside the dX contraction on the few SMs its last wave leaves
+  // free, where 32 shares of one K-block each took several rounds (C2 backward call 128 -> 115 us; 8 shares: 113)
+  if (want > 16) want = 16;
   if (want > kb) want = kb;
   if (want < 1) want = 1;
   const int per = (kb + want - 1) / want;
