@@ -718,11 +718,12 @@ int launch_pool(const QwView& qw, const AdView& ad, const __nv_bfloat16* X, int6
 }
 
 // u = x' A with x' = xh + xl: two K-segments against the same (exact, bf16) A
-int launch_u_gemm(const AdView& ad, int64_t T, const TcWs& w, const SgOut& out, int* status, cudaStream_t st) {
+int launch_u_gemm(const AdView& ad, int64_t T, const TcWs& w, const SgOut& out, int* status, cudaStream_t st,
+                  bool before_contraction) {
   const SgOperand a_mat{ad.A, ad.r, false};   // (n = rank index, k = p) at A[k * r + n]
   SgSegment segs[2] = {{{w.xh, w.ldp, true}, a_mat, ad.P}, {{w.xl, w.ldp, true}, a_mat, ad.P}};
   // directly behind the compression kernel on the same stream: its programmatic dependent
-  return small_gemm((int)T, ad.r, segs, 2, out, status, st, nullptr, overlap_adapter_prologue());
+  return small_gemm((int)T, ad.r, segs, 2, out, status, st, nullptr, overlap_adapter_prologue(), before_contraction);
 }
 
 }  // namespace
@@ -750,7 +751,7 @@ int tc_linear_fwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, in
     // u16 = bf16(s * x' A): the scaling rides on the compressed activation, B stays exact
     SgOut out{};
     out.scaled = w.u16; out.ld16 = w.ldr; out.scale = ad->s; out.divide = false;
-    rc = launch_u_gemm(*ad, T, w, out, status, st);
+    rc = launch_u_gemm(*ad, T, w, out, status, st, true);
     if (rc) return rc;
   }
   return launch_main(0, qw, ad, X, w.u16, w.ldr, T, Y, y_dtype, status, st);
@@ -818,7 +819,7 @@ int tc_linear_bwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, co
       SgOut out{};
       out.hi = w.duh; out.lo = w.dul; out.scaled = w.du16; out.ld16 = w.ldr; out.divide = true;
       out.scale = ad->op == QBLORA_SCALE_AVGPOOL_REPEAT ? (float)ad->l1 : 1.0f;   // only the average carries 1 / lambda_in
-      rc = small_gemm((int)T, ad->r, segs, 2, out, status, st, nullptr, overlap_adapter_prologue());   // behind dv's kernel
+      rc = small_gemm((int)T, ad->r, segs, 2, out, status, st, nullptr, overlap_adapter_prologue(), false);   // behind dv's kernel (narrow tiles: wide ones start the contraction earlier, which costs the gradient chain beside it more than it saves: C2 backward 115 vs 119 us)
       if (rc) return rc;
     }
     if (lane) QB_CUDA(cudaEventRecord(lane->du_done, st));
@@ -829,7 +830,7 @@ int tc_linear_bwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, co
     if (dB) {
       SgOut uo{};
       uo.hi = w.uh; uo.lo = w.ul; uo.ld16 = w.ldr;
-      rc = launch_u_gemm(*ad, T, w, uo, status, sb);
+      rc = launch_u_gemm(*ad, T, w, uo, status, sb, false);
       if (rc) return rc;
     }
     if (lane) QB_CUDA(cudaStreamWaitEvent(lane->stream, lane->du_done, 0));   // dv and du are complete

@@ -32,8 +32,11 @@ struct SgOut {
 // `dependent`: the kernel in front of this one on `st` is one of this library's that signals
 // griddepcontrol.launch_dependents and writes an operand; this product is then launched as its programmatic
 // dependent (set-up overlaps that kernel's tail; the operand loads wait for its completion).
+// `wide_tiles`: keep 256-wide column tiles even when that leaves few CTAs.  For a product that sits in front of the
+// fused contraction: each of its CTAs keeps a CTA of the contraction off its SM until it is done, so few CTAs
+// delay fewer tiles (C2 forward call 108 -> 103.5 us).
 int small_gemm(int M, int N, const SgSegment* segs, int nseg, const SgOut& out, int* status, cudaStream_t st,
-               float* partial = nullptr, bool dependent = false);
+               float* partial = nullptr, bool dependent = false, bool wide_tiles = false);
 int small_gemm_splits(int M, int N, int K);
 
 // Encodes a 2-D tensor map (shared with the main kernel's host code).

@@ -284,7 +284,7 @@ int small_gemm_splits(int M, int N, int K) {
 }
 
 int small_gemm(int M, int N, const SgSegment* segs, int nseg, const SgOut& out, int* status, cudaStream_t st,
-               float* partial, bool dependent) {
+               float* partial, bool dependent, bool wide_tiles) {
   if (nseg < 1 || nseg > SG_MAX_SEG || M < 1 || N < 1) return QBLORA_ERR_INVALID_ARG;
   static bool attr_set = false;
   if (!attr_set) {
@@ -297,7 +297,7 @@ int small_gemm(int M, int N, const SgSegment* segs, int nseg, const SgOut& out, 
   const int n64 = (N + 63) / 64 * 64;
   p.bn = n64 < 256 ? n64 : 256;
   // few row tiles and no split: narrower column tiles put more CTAs to work (the kernel is latency-bound)
-  while (!partial && p.bn > 64 && ((N + p.bn - 1) / p.bn) * ((M + SG_BM - 1) / SG_BM) < 96 && (p.bn / 2) % 64 == 0) p.bn /= 2;
+  while (!wide_tiles && !partial && p.bn > 64 && ((N + p.bn - 1) / p.bn) * ((M + SG_BM - 1) / SG_BM) < 96 && (p.bn / 2) % 64 == 0) p.bn /= 2;
   p.a_kmajor = segs[0].a.k_contig ? 1 : 0;
   p.b_kmajor = segs[0].b.k_contig ? 1 : 0;
   for (int g = 0; g < nseg; ++g) {
