@@ -86,7 +86,7 @@ static int get_code(const uint8_t* codes, int d_in, int o, int i) {
  *   code = number of midpoints between adjacent levels that fl32(w/alpha)
  *   exceeds (nearest level, ties to the lower index).  Eq. 1's absmax variant
  *   read with the level table in place of the integer grid.
- * qfmt 1 (min-max, Eq. 1 with N = 4): beta = min, alpha = fl32(fl32(max-min)/15),
+ * qfmt 1 (min-max, Eq. 1 with N = 4): beta = min (a zero minimum as +0), alpha = fl32(fl32(max-min)/15),
  *   code = clamp(round-half-even(fl32(fl32(w-beta)/alpha)), 0, 15).
  *   With nbits = N < 4 (Eq. 1 is stated for N bits) the grid has 2^N levels:
  *   alpha = fl32(fl32(max-min)/(2^N-1)), codes clamp to [0, 2^N-1]; they are
@@ -142,7 +142,8 @@ int orc_quantize_blockwise(const float* W, int d_out, int d_in, int block_in,
         float d = f32_sub(wmax, wmin);
         float a = f32_div(d, qmax);
         int degenerate = (d == 0.0f) || (a == 0.0f);
-        beta[bi] = wmin;
+        /* min() does not say which zero a zero minimum is (+0 == -0): it is stored as +0 */
+        beta[bi] = (wmin == 0.0f) ? 0.0f : wmin;
         alpha[bi] = degenerate ? 0.0f : a;
         for (int o = o0; o < o0 + block_out; ++o)
           for (int i = i0; i < i0 + block_in; ++i) {

@@ -187,6 +187,32 @@ def test_affine_tie_rounds_half_to_even():
     assert list(c[2:6]) == [0, 2, 2, 14]
 
 
+def test_zero_minimum_is_stored_as_positive_zero():
+    # Eq. 1: beta = min(w).  +0 and -0 compare equal, so "min" does not say which one a zero minimum is;
+    # the stored beta is +0 whatever the order and signs of the zeros in the block, and codes / alpha do
+    # not depend on it (w - (+0) and w - (-0) round to the same code).
+    base = np.zeros((1, 64), dtype=np.float32)
+    base[0, 2:] = np.linspace(0.0, 1.5, 62, dtype=np.float32)
+    ref = None
+    for z0, z1 in [(0.0, 0.0), (-0.0, 0.0), (0.0, -0.0), (-0.0, -0.0)]:
+        W = base.copy()
+        W[0, 0], W[0, 1] = np.float32(z0), np.float32(z1)
+        qw = oracle.quantize_blockwise(W, 64, 1, oracle.FMT_AFFINE_MINMAX)
+        assert qw.beta.view(np.uint32)[0, 0] == 0            # +0.0 bit pattern
+        assert qw.alpha[0, 0] == np.float32(np.float32(1.5) / np.float32(15.0))
+        if ref is None:
+            ref = qw
+        assert np.array_equal(qw.codes, ref.codes) and np.array_equal(qw.alpha, ref.alpha)
+    # a block of zeros of mixed sign is degenerate: alpha = 0, beta = +0, codes 0
+    W = np.zeros((1, 64), dtype=np.float32)
+    W[0, ::2] = np.float32(-0.0)
+    qw = oracle.quantize_blockwise(W, 64, 1, oracle.FMT_AFFINE_MINMAX)
+    assert qw.beta.view(np.uint32)[0, 0] == 0 and qw.alpha[0, 0] == 0 and not qw.codes.any()
+    # a negative minimum is untouched
+    W[0, 5] = np.float32(-0.25)
+    assert oracle.quantize_blockwise(W, 64, 1, oracle.FMT_AFFINE_MINMAX).beta[0, 0] == np.float32(-0.25)
+
+
 # ----------------------------------------------------------------- N-bit grids (Eq. 1 with N < 4)
 @pytest.mark.parametrize("nbits", [1, 2, 3])
 def test_nbit_closed_form_grid_maps_to_integers(nbits):
