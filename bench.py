@@ -2,8 +2,12 @@
 """Benchmark of the adapted quantized linear layer (Q-BLoRA / QA-BLoRA hot path) on B200.
 
 One step = forward + backward (dX, dA, dB) of every adapted linear of the workload through the
-C-ABI library, inputs resident in HBM.  Prints ONE JSON line.  ``--impl reference`` times the fp64
-CPU oracle on the host cores instead (a bounded sample of the same workload per step).
+C-ABI library, inputs resident in HBM.  The headline workload is the largest single-GPU configuration
+(the 13B-shaped decoder layer of seven linears); the other fine-tuning configurations are timed after it and
+reported under ``configs``.  A timed region is exactly ``--steps`` steps; it is repeated until about 1.5 s of
+timed work have run, so the clocks sampled beside it are those of a sustained run.  Prints ONE JSON line.
+``--impl reference`` times the fp64 CPU oracle on the host cores instead (a bounded sample of the same
+workload per step).
 
 Multi-GPU: the path has no exchange step; ``--gpus N`` (launched with torch.distributed.run) runs
 N independent replicas and reports the aggregate ("replicas only", weak scaling).
@@ -27,9 +31,29 @@ if ROOT not in sys.path:
 
 from paper_2407_17029_b200 import synth  # noqa: E402
 
-# dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, per launch, from the ncu
-# capture summarised in profiles/ncu_full_tc_dq_gemm_C2.md (set to None when that kernel changes)
-MEASURED_DRAM_TRAFFIC = {("C2", "GA"): 27.61e6 + 0.36e6}
+# dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel come from profiles/dram_traffic.json, which
+# records, next to each figure, the SHA-256 of the kernel source it was captured on: a figure whose kernel has
+# changed since is reported as null.
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "dram_traffic.json")
+DOMINANT_KERNEL_SOURCE = os.path.join(ROOT, "paper_2407_17029_b200", "csrc", "tc_gemm.cu")
+BURST_REGION_S = 0.1    # a timed region shorter than this runs at boost clocks: compare with the burst peak
+
+
+def measured_traffic(workload, geometry):
+    """(bytes per launch, note) of the dominant kernel from the ncu capture on record, or (None, why)."""
+    try:
+        import hashlib
+        rec = json.load(open(TRAFFIC_FILE))
+        sha = hashlib.sha256(open(DOMINANT_KERNEL_SOURCE, "rb").read()).hexdigest()
+        for e in rec["entries"]:
+            if e["workload"] == workload and e["geometry"] == geometry:
+                if e["kernel_source_sha256"] != sha:
+                    return None, "kernel source changed since the ncu capture on record"
+                return float(e["dram_bytes_per_launch"]), e.get("note", "ncu capture, profiles/")
+        return None, "no ncu capture on record for this workload"
+    except Exception as ex:   # missing file: no figure
+        return None, f"no traffic record ({type(ex).__name__})"
+
 
 METRIC = "fused 4-bit+BLoRA linear fwd+bwd TFLOP/s & low-bit GEMM GB/s, % of roofline"
 
@@ -141,7 +165,7 @@ def run_reference(args, wl, geom):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    rows = args.ref_rows
+    rows = ref_rows_for(wl, geom, args.ref_rows)
     cache = oracle_cache(wl, geom, rows)
     for _ in range(min(args.warmup, 1)):
         oracle_step(wl, geom, rows, cache)
@@ -163,37 +187,58 @@ def run_reference(args, wl, geom):
 
 
 # --------------------------------------------------------------------------------------- GPU arm
-def run_gpu(args, wl, geom):
-    import torch
-    from paper_2407_17029_b200 import binding as qb
+class GpuCtx:
+    """Device, rank and process-group plumbing shared by the measurements of one run."""
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
+    def __init__(self):
+        import torch
+        from paper_2407_17029_b200 import binding as qb
+        self.torch, self.qb = torch, qb
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.local = int(os.environ.get("LOCAL_RANK", "0"))
+        torch.cuda.set_device(self.local)
+        self.dev = torch.device("cuda", self.local)
+        self.dist = None
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.init_process_group("nccl", device_id=self.dev)
+            self.dist = dist
+        self.peaks = measured_peaks()
+        self.l2_bytes = torch.cuda.get_device_properties(self.dev).L2_cache_size
 
-    def bf(a):
-        return torch.from_numpy(synth.bf16_bits(a).view(np.int16).copy()).to(dev).view(torch.bfloat16)
+    def bf(self, a):
+        return self.torch.from_numpy(synth.bf16_bits(a).view(np.int16).copy()).to(self.dev).view(self.torch.bfloat16)
 
+    def barrier(self):
+        if self.dist is not None:
+            self.dist.barrier()
+        self.torch.cuda.synchronize()
+
+    def max_over_ranks(self, x):
+        if self.dist is None:
+            return float(x)
+        t = self.torch.tensor([x], dtype=self.torch.float64, device=self.dev)
+        self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
+        return float(t.item())
+
+
+def measure_workload(ctx, wl, geom, steps, warmup, min_region_s, no_graph=False, want_e2e=True):
+    """Times forward + backward steps of one workload.  A timed region is EXACTLY `steps` steps between a barrier +
+    synchronize on both sides; the region is repeated until at least `min_region_s` seconds of timed work have
+    run (so that clocks and power settle where a long job would hold them), and the mean region is reported."""
+    torch, qb, dev = ctx.torch, ctx.qb, ctx.dev
     T, r = wl.tokens, wl.rank
-    peaks = measured_peaks()
-    l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
-    # ---- build the sets of resident buffers; rotate over enough distinct sets to exceed 2x L2
+    # ---- resident buffers; rotate over enough distinct sets to exceed 2x L2
     lin = []
     step_bytes = 0
     for spec in wl.linears:
-        li = synth.make_linear_inputs(wl, spec, geom, seed=rank)
+        li = synth.make_linear_inputs(wl, spec, geom, seed=ctx.rank)
         dq = qb.quantize_blockwise(torch.from_numpy(li.W).to(dev), wl.block_in, 1, wl.qfmt)
         li.W = None
-        per_set = (li.X.size + li.dY.size) * 2 * 2 + packed_bytes(spec.d_out, spec.d_in, wl.block_in, wl.qfmt == 1)
-        step_bytes += per_set
+        step_bytes += (li.X.size + li.dY.size) * 2 * 2 + packed_bytes(spec.d_out, spec.d_in, wl.block_in, wl.qfmt == 1)
         lin.append((spec, li, dq))
-    nsets = max(2, int(np.ceil(2.0 * l2_bytes / step_bytes)) + 1)
+    nsets = max(2, int(np.ceil(2.0 * ctx.l2_bytes / step_bytes)) + 1)
     sets = []
     for s in range(nsets):
         items = []
@@ -201,8 +246,8 @@ def run_gpu(args, wl, geom):
             # distinct device copies (same values): what matters is that the addresses differ
             q2 = qb.QWeight(dq.d_out, dq.d_in, dq.block_in, dq.block_out, dq.qfmt, dq.code,
                             dq.codes.clone(), dq.alpha.clone(), dq.beta.clone() if dq.beta is not None else None)
-            ad = qb.Adapter(geom.lambda_in, geom.lambda_out, r, wl.scaling, bf(li.A), bf(li.B), SCALE_OP)
-            X, dY = bf(li.X), bf(li.dY)
+            ad = qb.Adapter(geom.lambda_in, geom.lambda_out, r, wl.scaling, ctx.bf(li.A), ctx.bf(li.B), SCALE_OP)
+            X, dY = ctx.bf(li.X), ctx.bf(li.dY)
             Y = torch.empty((T, spec.d_out), dtype=torch.bfloat16, device=dev)
             dX = torch.empty((T, spec.d_in), dtype=torch.bfloat16, device=dev)
             dA = torch.empty(tuple(ad.A.shape), dtype=torch.float32, device=dev)
@@ -211,6 +256,7 @@ def run_gpu(args, wl, geom):
             wsb = qb.alloc_workspace(qb.OP_LINEAR_BWD, q2, ad, T)
             items.append((spec, q2, ad, X, dY, Y, dX, dA, dB, wsf, wsb))
         sets.append(items)
+    del lin
 
     def step(i, ev=None):
         for j, (spec, q2, ad, X, dY, Y, dX, dA, dB, wsf, wsb) in enumerate(sets[i % nsets]):
@@ -219,43 +265,19 @@ def run_gpu(args, wl, geom):
             qb.linear_fwd(q2, ad, X, ws=wsf, out=Y)
             qb.linear_bwd(q2, ad, X, dY, ws=wsb, outs=(dX, dA, dB))
 
-    def barrier():
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
-
     flops_step = sum(sum(linear_flops(T, s.d_out, s.d_in, r, geom)) for s in wl.linears)
     # dominant kernel: the forward base contraction of the largest linear
     dom = max(range(len(wl.linears)), key=lambda j: wl.linears[j].d_out * wl.linears[j].d_in)
     dspec = wl.linears[dom]
     dom_flops = 2.0 * T * dspec.d_in * dspec.d_out
 
-    for i in range(args.warmup):
+    for i in range(warmup):
         step(i)
-    barrier()
-    sampler = ClockSampler(local)
-    sampler.start()
-    time.sleep(0.3)
-    kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True), dom) for _ in range(args.steps)]
-    for a, b, _ in kev:          # torch creates the CUDA event handle on first record
-        a.record(); b.record()
-    launches0 = qb.kernel_launches()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    # ---- eager pass: every call launched from the host; the library brackets the dominant kernel
-    barrier()
-    e0.record()
-    for i in range(args.steps):
-        step(args.warmup + i, kev[i])
-    e1.record()
-    barrier()
-    launches = qb.kernel_launches() - launches0
-    eager_ms = e0.elapsed_time(e1)
-    dom_ms = statistics.mean(a.elapsed_time(b) for a, b, _ in kev)
-    ms = eager_ms
-    mode = "eager launches"
-    if not args.no_graph:
-        # ---- the same steps replayed as CUDA graphs (one graph per buffer set, one step each): the small
-        # adapter-side kernels are launch-bound when issued from the host one by one
+    ctx.barrier()
+    graphs = None
+    if not no_graph:
+        # the same steps as CUDA graphs (one graph per buffer set, one step each): the small adapter-side kernels
+        # are launch-bound when issued from the host one by one
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
         graphs = []
@@ -264,24 +286,77 @@ def run_gpu(args, wl, geom):
             with torch.cuda.graph(g, stream=side):
                 step(si)
             graphs.append(g)
-        for i in range(args.warmup):
+        for i in range(warmup):
             graphs[i % nsets].replay()
-        barrier()
+        ctx.barrier()
+
+    def run_steps(first):
+        for i in range(steps):
+            if graphs is not None:
+                graphs[(first + i) % nsets].replay()
+            else:
+                step(first + i)
+
+    sampler = ClockSampler(ctx.local)
+    sampler.start()
+    time.sleep(0.25)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    regions = []
+    done_s, k = 0.0, 0
+    while not regions or (done_s < min_region_s and len(regions) < 2000):
+        ctx.barrier()
         e0.record()
-        for i in range(args.steps):
-            graphs[(args.warmup + i) % nsets].replay()
+        run_steps(warmup + k * steps)
         e1.record()
-        barrier()
-        ms = e0.elapsed_time(e1)
-        mode = "CUDA-graph replay, one graph per buffer set"
+        ctx.barrier()
+        regions.append(e0.elapsed_time(e1))
+        done_s += regions[-1] * 1e-3
+        k += 1
+    # ---- one more region with every call launched from the host; the library brackets the dominant kernel of
+    # each step with an event pair (the chip is in the state the regions above left it in)
+    kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True), dom) for _ in range(steps)]
+    for a, b, _ in kev:          # torch creates the CUDA event handle on first record
+        a.record(); b.record()
+    launches0 = qb.kernel_launches()
+    ctx.barrier()
+    e0.record()
+    for i in range(steps):
+        step(warmup + i, kev[i])
+    e1.record()
+    ctx.barrier()
+    launches = qb.kernel_launches() - launches0
+    eager_ms = e0.elapsed_time(e1)
     clocks = sampler.stop()
+    dom_ms = statistics.mean(a.elapsed_time(b) for a, b, _ in kev)
+    if graphs is None:
+        regions.append(eager_ms)
     for spec, q2, ad, X, dY, Y, dX, dA, dB, wsf, wsb in sets[0]:
         assert qb.device_status(wsf) == qb.OK and qb.device_status(wsb) == qb.OK
-    if dist is not None:
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    value = flops_step * world * args.steps / (ms * 1e-3) / 1e12
+    ms = ctx.max_over_ranks(statistics.mean(regions))          # mean region of exactly `steps` steps, max over ranks
+    value = flops_step * ctx.world * steps / (ms * 1e-3) / 1e12
+    timed_s = sum(regions) * 1e-3 + eager_ms * 1e-3
+    sustained = timed_s >= BURST_REGION_S
+    peak = ctx.peaks["bf16_tflops_sustained"] if sustained else ctx.peaks["bf16_tflops"]
+    achieved = dom_flops / (dom_ms * 1e-3) / 1e12
+    traffic, traffic_note = measured_traffic(wl.name, geom.name)
+    res = {
+        "value": value, "ms_per_step": ms / steps, "steps": steps, "regions": len(regions),
+        "region_ms": {"mean": statistics.mean(regions), "min": min(regions), "max": max(regions)},
+        "timed_s": timed_s, "step_flops": flops_step, "clocks": clocks, "gpu_launches": int(launches),
+        "launch": "eager launches" if graphs is None else "CUDA-graph replay, one graph per buffer set",
+        "l2": f"rotating over {nsets} distinct buffer sets ({nsets * step_bytes / 2**20:.0f} MiB > 2x L2)",
+        "frac_of_peak": value / ctx.world / peak,
+        "roofline": {"bound": "tensor", "kernel": f"forward base contraction {dspec.name}[{dspec.d_out},{dspec.d_in}] T={T}",
+                     "achieved": achieved, "peak": peak,
+                     "peak_kind": (f"bf16 dense, {'sustained' if sustained else 'burst'}, {ctx.peaks['source']}: the kernel was timed inside "
+                                   f"{timed_s:.2f} s of back-to-back steps (burst figure below {BURST_REGION_S} s, sustained above)"),
+                     "unit": "TFLOP/s", "frac": achieved / peak,
+                     "frac_of_burst": achieved / ctx.peaks["bf16_tflops"], "frac_of_sustained": achieved / ctx.peaks["bf16_tflops_sustained"],
+                     "traffic": traffic, "traffic_note": traffic_note, "ms_per_launch": dom_ms},
+        "eager": {"ms_per_step": eager_ms / steps, "value": flops_step * steps / (eager_ms * 1e-3) / 1e12,
+                  "unit": "TFLOP/s", "note": "this rank, every call launched from the host"}}
+    if not want_e2e:
+        return res
 
     # ---- end to end: host (pinned) inputs in, results out, copies inside the timed region.  Up to three lanes
     # (stream + device buffer set + pinned host buffers each) take the steps in turn, so the copies of
@@ -289,7 +364,8 @@ def run_gpu(args, wl, geom):
     # its inputs and results.
     lanes = []
     h2d = d2h = 0
-    n_lanes = min(3, nsets)
+    lane_bytes = sum((X.numel() + dY.numel() + Y.numel() + dX.numel()) * 2 for _, _, _, X, dY, Y, dX, *_ in sets[0])
+    n_lanes = max(1, min(3, nsets, int(8e9 // max(lane_bytes, 1))))        # at most ~8 GB of pinned host memory
     for li_ in range(n_lanes):
         host = []
         for spec, q2, ad, X, dY, Y, dX, dA, dB, wsf, wsb in sets[li_]:
@@ -312,58 +388,73 @@ def run_gpu(args, wl, geom):
                 hY.copy_(Y, non_blocking=True); hdX.copy_(dX, non_blocking=True)
                 hdA.copy_(dA, non_blocking=True); hdB.copy_(dB, non_blocking=True)
 
-    e2e_steps = max(3, min(args.steps, 10))
+    e2e_steps = max(3, min(steps, 10))
     for i in range(n_lanes):
         e2e_step(i)
-    barrier()
+    ctx.barrier()
     t0 = time.perf_counter()
     for i in range(e2e_steps):
         e2e_step(i)
-    barrier()
-    e2e_s = time.perf_counter() - t0
-    if dist is not None:
-        t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e_val = flops_step * world * e2e_steps / e2e_s / 1e12
+    ctx.barrier()
+    e2e_s = ctx.max_over_ranks(time.perf_counter() - t0)
+    res["e2e"] = {"value": flops_step * ctx.world * e2e_steps / e2e_s / 1e12, "unit": "TFLOP/s",
+                  "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps, "lanes": n_lanes}
+    return res
 
-    line = {"metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+
+def ref_rows_for(wl, geom, requested):
+    """Token rows of one bounded oracle step: about 45 GF of fp64 work (10-15 s on a dozen host cores)."""
+    if requested:
+        return min(requested, wl.tokens)
+    per_row = sum(sum(linear_flops(1, s.d_out, s.d_in, wl.rank, geom)) for s in wl.linears)
+    return int(max(8, min(wl.tokens, 512, round(45e9 / per_row / 8) * 8)))
+
+
+def run_gpu(args, wl, geom):
+    ctx = GpuCtx()
+    torch, qb = ctx.torch, ctx.qb
+    m = measure_workload(ctx, wl, geom, args.steps, args.warmup, args.min_region_s, args.no_graph, want_e2e=True)
+    T, r = wl.tokens, wl.rank
+    line = {"metric": METRIC, "value": m["value"], "unit": "TFLOP/s", "n_gpus": ctx.world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": m["ms_per_step"], "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": wl.name, "scale_op": SCALE_OP, "geometry": f"{geom.name} (lambda_in={geom.lambda_in}, lambda_out={geom.lambda_out})",
                        "tokens": T, "linears": [f"{s.name}[{s.d_out},{s.d_in}]" for s in wl.linears], "rank": r,
                        "quant": "4-bit, block 64 along input, " + ("min-max" if wl.qfmt else "level table + absmax"),
-                       "parallelism": "replicas only" if world > 1 else "single GPU",
-                       "launch": mode,
-                       "l2": f"rotating over {nsets} distinct buffer sets ({nsets * step_bytes / 2**20:.0f} MiB > 2x L2)"},
-            "clocks": clocks, "gpu_launches": int(launches),
-            "e2e": {"value": e2e_val, "unit": "TFLOP/s", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
-                    "steps": e2e_steps, "lanes": n_lanes},
-            "roofline": {"bound": "tensor", "kernel": f"forward base contraction {dspec.name}[{dspec.d_out},{dspec.d_in}] T={T}",
-                         "achieved": dom_flops / (dom_ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops_sustained"],
-                         "peak_kind": f"bf16 dense, sustained, {peaks['source']}", "unit": "TFLOP/s",
-                         "frac": dom_flops / (dom_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
-                         "peak_burst": peaks["bf16_tflops"],
-                         "frac_of_burst": dom_flops / (dom_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
-                         "traffic": MEASURED_DRAM_TRAFFIC.get((wl.name, geom.name)), "ms_per_launch": dom_ms},
-            "step_flops": flops_step,
-            "eager": {"ms_per_step": eager_ms / args.steps, "value": flops_step * args.steps / (eager_ms * 1e-3) / 1e12,
-                      "unit": "TFLOP/s", "note": "this rank, every call launched from the host"}}
-
-    if rank == 0 and not args.no_extras:
-        line["lowbit"] = lowbit_extras(qb, torch, dev, peaks, l2_bytes, args.lowbit_shapes.split(","),
+                       "parallelism": "replicas only" if ctx.world > 1 else "single GPU",
+                       "launch": m["launch"], "l2": m["l2"],
+                       "timing": f"{m['regions']} timed regions of exactly {args.steps} steps each ({m['timed_s']:.2f} s of timed work); "
+                                 "value = steps x flops / mean region"},
+            "regions": m["regions"], "region_ms": m["region_ms"], "frac_of_peak": m["frac_of_peak"],
+            "clocks": m["clocks"], "gpu_launches": m["gpu_launches"], "e2e": m["e2e"], "roofline": m["roofline"],
+            "step_flops": m["step_flops"], "eager": m["eager"]}
+    # ---- the other fine-tuning configurations, each for about a second of timed work (rank 0 reports its own)
+    if ctx.world == 1 and args.configs:
+        line["configs"] = {}
+        for name in [c for c in args.configs.split(",") if c and c != wl.name]:
+            torch.cuda.empty_cache()
+            w2 = synth.WORKLOADS[name]
+            m2 = measure_workload(ctx, w2, geom, args.steps, args.warmup, args.min_region_s_configs, args.no_graph, want_e2e=False)
+            line["configs"][name if name != "C5" else "C5 shapes as a fine-tuning step"] = {
+                "tokens": w2.tokens, "linears": [f"{s.name}[{s.d_out},{s.d_in}]" for s in w2.linears],
+                "ms_per_step": m2["ms_per_step"], "value": m2["value"], "unit": "TFLOP/s", "frac_of_peak": m2["frac_of_peak"],
+                "regions": m2["regions"], "timed_s": m2["timed_s"], "clocks": m2["clocks"],
+                "dominant_kernel": {k: m2["roofline"][k] for k in ("kernel", "achieved", "peak", "peak_kind", "frac", "frac_of_burst", "ms_per_launch")}}
+    torch.cuda.empty_cache()
+    if ctx.rank == 0 and not args.no_extras:
+        line["lowbit"] = lowbit_extras(qb, torch, ctx.dev, ctx.peaks, ctx.l2_bytes, args.lowbit_shapes.split(","),
                                        [int(t) for t in args.lowbit_tokens.split(",")])
-    if rank == 0 and not args.no_cpu_baseline and world == 1:
-        rows = args.ref_rows
+    if ctx.rank == 0 and not args.no_cpu_baseline and ctx.world == 1:
+        rows = ref_rows_for(wl, geom, args.ref_rows)
         cache = oracle_cache(wl, geom, rows)
         import oracle
         t, f = oracle_step(wl, geom, rows, cache)
         line["cpu_baseline"] = {"value": f / t / 1e12, "unit": "TFLOP/s", "cores": oracle.num_threads(), "kind": "oracle",
                                 "sample": f"{rows} of {T} token rows, all linears, fwd+bwd (dX, dA, dB), {t:.1f} s"}
-    if rank == 0:
+    if ctx.rank == 0:
         print(json.dumps(line), flush=True)
-    if dist is not None:
-        dist.destroy_process_group()
+    if ctx.dist is not None:
+        ctx.dist.destroy_process_group()
 
 
 def lowbit_extras(qb, torch, dev, peaks, l2_bytes, shapes=("q", "up"), tokens=(1, 16, 2048)):
@@ -423,7 +514,8 @@ def lowbit_extras(qb, torch, dev, peaks, l2_bytes, shapes=("q", "up"), tokens=(1
                 e.record(); torch.cuda.synchronize()
                 us = s.elapsed_time(e) / 10 * 1e3
                 tf = 2.0 * T * spec.d_in * spec.d_out / us / 1e6
-                out[f"{spec.name}/T{T}"] = {"us": us, "TFLOP/s": tf, "frac_bf16_sustained": tf / peaks["bf16_tflops_sustained"],
+                out[f"{spec.name}/T{T}"] = {"us": us, "TFLOP/s": tf, "frac_bf16_burst": tf / peaks["bf16_tflops"],
+                                            "peak_kind": "burst (ten launches, a few ms)", "frac_bf16_sustained": tf / peaks["bf16_tflops_sustained"],
                                             "status": qb.device_status(wsl)}
                 del Xl, Yl
                 continue
@@ -480,15 +572,19 @@ def lowbit_extras(qb, torch, dev, peaks, l2_bytes, shapes=("q", "up"), tokens=(1
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="gpu", choices=["gpu", "reference"])
-    ap.add_argument("--workload", default="C2", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--workload", default="C4", choices=sorted(synth.WORKLOADS),
+                    help="headline workload (default: the largest single-GPU configuration)")
+    ap.add_argument("--configs", default="C2,C3,C5", help="other fine-tuning configurations reported beside the headline ('' = none)")
+    ap.add_argument("--min-region-s", type=float, default=1.5, help="repeat the K-step timed region until this much timed work has run")
+    ap.add_argument("--min-region-s-configs", type=float, default=1.0)
     ap.add_argument("--geometry", default="GA", choices=["GA", "GB"])
     ap.add_argument("--scale-op", type=int, default=0, choices=[0, 1, 2],
                     help="adapter operator pair: 0 AvgPool & repeat_interleave (the method), 1 truncation & zero padding, "
                          "2 interval sampling & zero fill (Sec. 4 ablation)")
-    ap.add_argument("--ref-rows", type=int, default=512, help="token rows per oracle step (bounded sample)")
+    ap.add_argument("--ref-rows", type=int, default=0, help="token rows per oracle step (bounded sample; 0 = sized for about 45 GF per step)")
     ap.add_argument("--ref-max-steps", type=int, default=3)
     ap.add_argument("--no-extras", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -108,7 +108,7 @@ size_t ws_bytes_impl(int op, const QwView& q, const AdView* ad, int64_t T) {
     case QBLORA_OP_MERGE_DENSE: return merge_dense_ws_bytes(q, ad);
     case QBLORA_OP_LOWBIT_GEMM:
       if (gemv_supported(q, T)) return gemv_ws_bytes(q, T);
-      if (!force_general() && tc_supported(q, nullptr, T)) return tc_ws_bytes(QBLORA_OP_LINEAR_FWD, q, nullptr, T);
+      if (!force_general() && tc_supported(q, nullptr, T)) return tc_lowbit_ws_bytes(q, T);
       return simt_ws_bytes(QBLORA_OP_LINEAR_FWD, q, nullptr, T);
     default: return 0;
   }
@@ -333,7 +333,7 @@ int qablora_lowbit_gemm(const qblora_qweight* qw, const void* X, int64_t tokens,
   rc = reset_status(ws, st);
   if (rc) return rc;
   if (!force_general() && tc_supported(q, nullptr, tokens))
-    return tc_linear_fwd(q, nullptr, Xb, tokens, Y, y_dtype, static_cast<char*>(ws), st);
+    return tc_lowbit_gemm(q, Xb, tokens, Y, y_dtype, static_cast<char*>(ws), st);
   return simt_linear_fwd(q, nullptr, Xb, tokens, Y, y_dtype, static_cast<char*>(ws), st);
 }
 

@@ -89,6 +89,9 @@ bool tc_supported(const QwView& qw, const AdView* ad, int64_t T);
 size_t tc_ws_bytes(int op, const QwView& qw, const AdView* ad, int64_t T);
 int tc_linear_fwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, int64_t T, void* Y,
                   int y_dtype, char* ws, cudaStream_t st);
+// Low-bit product on the tensor-core path (any token count; the caller sends small ones to the decode kernels).
+size_t tc_lowbit_ws_bytes(const QwView& qw, int64_t T);
+int tc_lowbit_gemm(const QwView& qw, const __nv_bfloat16* X, int64_t T, void* Y, int y_dtype, char* ws, cudaStream_t st);
 int tc_linear_bwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X,
                   const __nv_bfloat16* dY, int64_t T, void* dX, int dx_dtype, float* dA, float* dB,
                   char* ws, cudaStream_t st);

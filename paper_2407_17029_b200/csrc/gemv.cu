@@ -131,16 +131,19 @@ __device__ __forceinline__ float4 gv_ldsf4(uint32_t addr) {
   return v;
 }
 
-// Release of a shared-memory buffer to the producer.  The arrival names values computed from
-// everything the warp loaded from the buffer, so it cannot be issued before those loads have
-// returned: a load that is merely issued may still be in flight when the refill lands.
-__device__ __forceinline__ void gv_release(uint32_t bar, float d0, float d1, float d2, float d3) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];  // after %1 %2 %3 %4"
-               ::"r"(bar), "f"(d0), "f"(d1), "f"(d2), "f"(d3) : "memory");
+// Release of a shared-memory buffer to the producer: one mbarrier arrival per warp, issued by lane 0 after
+// __syncwarp().  What has to hold: every lane's ld.shared from the buffer has returned its data before the
+// arrival is performed, because the arrival (release) is what the producer's try_wait (acquire) pairs with
+// before it lets the async proxy (TMA / bulk copy) overwrite the buffer.  Program order alone does not give
+// that to the assembler -- a load that is merely issued may still be in flight -- so the arrival's address
+// operand is made to depend on `dep`, a value computed FROM the loaded registers (the sums they fed, see the
+// call sites) and and-ed with a kernel parameter that is zero at run time but unknown at compile time.  The
+// arrival therefore cannot issue before those registers are written, whatever the scheduling.
+__device__ __forceinline__ uint32_t gv_dep(float a, float b, float c, float d, uint32_t zero) {
+  return (__float_as_uint(a) ^ __float_as_uint(b) ^ __float_as_uint(c) ^ __float_as_uint(d)) & zero;
 }
-__device__ __forceinline__ void gv_release_u(uint32_t bar, uint32_t d0, uint32_t d1, float d2, float d3) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];  // after %1 %2 %3 %4"
-               ::"r"(bar), "r"(d0), "r"(d1), "f"(d2), "f"(d3) : "memory");
+__device__ __forceinline__ void gv_release(uint32_t bar, uint32_t dep) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar + dep) : "memory");
 }
 
 // Waits of this kernel pass a suspend-time hint so that a waiting warp sleeps in hardware until the
@@ -175,6 +178,7 @@ struct GtParams {
   int* status;
   // one-token kernel, split tail (see T1Walk): row blocks done whole, ways the rest is split, hand-over area
   int tail_first, tail_split;
+  uint32_t zero;             // always 0; unknown to the compiler (see gv_release)
   uint32_t epoch;            // value a hand-over flag takes in this launch (never 0, differs from launch to launch)
   float* tail_partial;       // [tail row block][part][32 rows] fp32
   uint32_t* tail_flags;      // [tail row block][part]
@@ -394,7 +398,8 @@ lowbit_gemv_t1_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
             }
           }
           __syncwarp();
-          if (lane == 0) gv_release(empty(s), y[0][0], y[0][1], y[1][0], y[1][1]);   // this warp is done reading the stage
+          // y[][] are sums over everything this lane loaded from the stage (codes through the MMAs, alpha, beta)
+          if (lane == 0) gv_release(empty(s), gv_dep(y[0][0], y[0][1], y[1][0], y[1][1], p.zero));
         }
         if (++s == STAGES) { s = 0; ph ^= 1u; }
       }
@@ -416,7 +421,7 @@ lowbit_gemv_t1_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
 #pragma unroll
         for (int ww = 0; ww < GT_WARPS; ++ww) a += red[ww * GT_ROWS + lane];
         __syncwarp();
-        if (lane == 0) gv_release(red_free, a, a, a, a);
+        if (lane == 0) gv_release(red_free, gv_dep(a, a, a, 0.0f, p.zero));
         if (walk.tail) {
           const int slot = (rb - p.tail_first) * p.tail_split;
           if (walk.part != 0) {
@@ -441,6 +446,11 @@ lowbit_gemv_t1_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
             if (seen != p.epoch) ok = false;
             __threadfence();
             a += __ldcg(p.tail_partial + (slot + part) * GT_ROWS + lane);
+            // Consumed: put the flag back to 0, which is never an epoch.  A launch replayed from a CUDA graph
+            // carries the epoch it was captured with, so without this the flag left by the previous replay
+            // would already match and the owner would read sums that are not there yet.  The next writer of
+            // this flag is a later launch, whose compute warps start only after this grid has completed.
+            if (lane == 0) atomicExch(p.tail_flags + slot + part, 0u);
           }
         }
         const int o = rb * GT_ROWS + lane;                // lane = row of the block
@@ -735,15 +745,22 @@ lowbit_gemv_ko_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
               }
             }
             __syncwarp();
-            if (lane == 0) gv_release(empty(s), y[j][0][0][0], y[j][0][0][2], y[j][0][1][0], y[j][0][1][2]);
+            // sums over everything this lane loaded from the stage: rows g (…[0]) and g + 8 (…[2]) of both row tiles
+            if (lane == 0) gv_release(empty(s), gv_dep(y[j][0][0][0], y[j][0][0][2], y[j][0][1][0], y[j][0][1][2], p.zero));
           }
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
-        // The fragment buffer is released only here, after the K tile's row blocks: releasing it right
-        // after the loads into registers (even with the release made to depend on the loaded values)
-        // produced rare wrong sums for the second token tile under stress.
+        // The fragment buffer is released here, after the K tile's row blocks.  The arrival depends on the
+        // first row block's sums of every token tile (they consumed f[n][0..7] through the MMAs and both
+        // sg[n][] entries) and, for a warp whose group lies beyond G and did no arithmetic, on the last loaded
+        // registers themselves.
         __syncwarp();
-        if (ok && lane == 0) gv_release_u(xempty(xb), f[0][7], f[NT - 1][7], sg[0][1].w, sg[NT - 1][1].w);
+        if (ok && lane == 0) {
+          uint32_t dep = __float_as_uint(sg[0][1].w) ^ __float_as_uint(sg[NT - 1][1].w) ^ f[0][7] ^ f[NT - 1][7];
+#pragma unroll
+          for (int n = 0; n < NT; ++n) dep ^= __float_as_uint(y[0][n][0][0]) ^ __float_as_uint(y[0][n][0][1]);
+          gv_release(xempty(xb), dep & p.zero);
+        }
       }
       // ---- end of the pass: the RB row blocks are summed over the warps one after the other
 #pragma unroll
@@ -771,7 +788,7 @@ lowbit_gemv_ko_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
 #pragma unroll
           for (int ww = 0; ww < GT_WARPS; ++ww) a += red[(ww * NTOK + t) * GT_ROWS + (lane ^ (((t >> 1) & 3) << 3))];
           __syncwarp();
-          if (lane == 0) gv_release(red_free, a, a, a, a);
+          if (lane == 0) gv_release(red_free, gv_dep(a, a, a, 0.0f, p.zero));
           const int o = rb * GT_ROWS + lane;                // lane = row of the block
           if (o < p.d_out) {
             if (p.y_dtype == QBLORA_BF16) reinterpret_cast<__nv_bfloat16*>(p.Y)[(int64_t)t * p.d_out + o] = __float2bfloat16_rn(a);

@@ -125,7 +125,7 @@ __global__ void __launch_bounds__(256) quantize_b64_kernel(const TIn* __restrict
       }
       if (live && part == 0) {
         alpha[b] = degenerate ? 0.0f : a;
-        beta[b] = mn;
+        beta[b] = mn == 0.0f ? 0.0f : mn;   // a zero minimum is stored as +0, whichever zeros the block holds
       }
     }
     if (live) reinterpret_cast<uint32_t*>(codes)[b * 8 + part] = packed;   // element 2k in the low nibble of byte k
@@ -159,7 +159,7 @@ __global__ void quantize_generic_kernel(const TIn* __restrict__ W, int d_out, in
     a = __fdiv_rn(d, tab.qmax);
     degenerate = (d == 0.0f) || (a == 0.0f);
     alpha[b] = degenerate ? 0.0f : a;
-    beta[b] = mn;
+    beta[b] = mn == 0.0f ? 0.0f : mn;   // a zero minimum is stored as +0
   }
   const float inv = __frcp_rn(a);
   for (int o = o0; o < o0 + block_out; ++o)

@@ -58,6 +58,13 @@ struct TcParams {
   const __nv_bfloat16* ex;  // adapter matrix feeding the extra K-blocks: forward B [r][Q], backward A [P][r]
   int ex_ld, ex_rows, lam;  // its leading dimension; the rank r; forward lambda_out, backward lambda_in
   int op, n_small;          // operator pair (qblora_scale_op) and the compressed size on that side (forward Q, backward P)
+  // Low-bit product (Sec. 3.3) only: the per-block offsets as their own K-blocks.  The weight tile then holds
+  // bf16(alpha * c + beta_c) with beta_c = -alpha * (mid code of the block), and the rest of the offset,
+  // gamma = beta' - beta_c, multiplies the group sums of x: three K-segments of ng_blocks K-blocks each,
+  // (gamma_hi, S_hi), (gamma_lo, S_hi), (gamma_hi, S_lo), with hi + lo the bf16 split of an fp32 value.
+  int kb_gamma, ng_blocks;
+  const __nv_bfloat16 *gam_h, *gam_l;   // [d_out][gam_ld], columns beyond G are zero
+  int gam_ld;
   void* out;                // forward Y [T][d_out]; backward dX [T][d_in]
   int out_dtype;
   int* status;
@@ -128,7 +135,8 @@ __device__ __forceinline__ void dequant_direct8(uint32_t w, int word, const floa
 template <int MODE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ CUtensorMap tm_bx,
-                  const __grid_constant__ CUtensorMap tm_p, const __grid_constant__ TcParams p) {
+                  const __grid_constant__ CUtensorMap tm_p, const __grid_constant__ CUtensorMap tm_s,
+                  const __grid_constant__ CUtensorMap tm_sl, const __grid_constant__ TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -166,7 +174,8 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
   const uint32_t tmem_base = *tmem_slot_g;
 
   const int num_tiles = p.m_tiles * p.n_tiles;
-  const int kb_total = p.kb_base + p.kb_extra;
+  const int kb_total = p.kb_base + p.kb_extra + p.kb_gamma;
+  const int kb_gamma0 = p.kb_base + p.kb_extra;   // first K-block of the offset term
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (one lane)
@@ -199,7 +208,12 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
               adapter_input_ready = true;
             }
             mbar_arrive_expect_tx(full(s), B_BYTES);
-            tma_load_2d(sB + s * B_BYTES, &tm_bx, full(s), (kb - p.kb_base) * BK, t0);
+            if (kb < kb_gamma0) {
+              tma_load_2d(sB + s * B_BYTES, &tm_bx, full(s), (kb - p.kb_base) * BK, t0);
+            } else {   // group sums of x: hi for the first two segments, lo for the third
+              const int kg = kb - kb_gamma0, seg = kg / p.ng_blocks, blk = kg - seg * p.ng_blocks;
+              tma_load_2d(sB + s * B_BYTES, seg == 2 ? &tm_sl : &tm_s, full(s), blk * BK, t0);
+            }
           }
         }
       }
@@ -233,7 +247,7 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
           tc_fence_after();
           // weight K-blocks: K-major tile in the forward, MN-major in the backward; the adapter
           // K-blocks are written the other way round (see the dequant warps)
-          const bool a_kmajor = (MODE == 0) == (kb < p.kb_base);
+          const bool a_kmajor = kb >= kb_gamma0 || (MODE == 0) == (kb < p.kb_base);
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k) {
             const uint64_t adesc = a_kmajor ? smem_desc(sA + s * A_BYTES + k * 32, 16, 1024)
@@ -267,7 +281,7 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
         // K-major tile: thread d owns row d (64 K elements = 128 bytes).  MN-major tile: thread d owns
         // K-row (d & 63) of the 64-row group (d >> 6).  Either way a 128-byte row whose 16-byte chunks
         // are XOR-swizzled with (d & 7).
-        const bool a_kmajor = (MODE == 0) == (kb < p.kb_base);
+        const bool a_kmajor = kb >= kb_gamma0 || (MODE == 0) == (kb < p.kb_base);
         const uint32_t dst = a_kmajor ? a_stage + d * 128 : a_stage + (d >> 6) * 8192 + (d & 63) * 128;
         const uint32_t xr = d & 7;
         if (kb < p.kb_base && p.direct) {
@@ -329,6 +343,19 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
             uint32_t o4[4];
             tab.lookup8(w[j], o4, k_m4, k_c3210);
             st_shared_v4(dst + (((uint32_t)j ^ xr) << 4), o4[0], o4[1], o4[2], o4[3]);
+          }
+        } else if (kb >= kb_gamma0) {
+          // offset term of the low-bit product: K-major tile A[m = o][k = group] = gamma_hi (segments 0, 2) or
+          // gamma_lo (segment 1); thread = output row o, reading 128 contiguous bytes of that row
+          if (!mbar_wait(empty(s), ph ^ 1u, p.status) || (rank != 0 && !mbar_wait(full(s), ph, p.status))) { ok = false; break; }
+          const int kg = kb - kb_gamma0, seg = kg / p.ng_blocks, g0 = (kg - seg * p.ng_blocks) * BK;
+          const int o = m0 + d;
+          const uint4* src = reinterpret_cast<const uint4*>((seg == 1 ? p.gam_l : p.gam_h) + (int64_t)(o < p.d_out ? o : 0) * p.gam_ld + g0);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (o < p.d_out && g0 + j * 8 < p.gam_ld) v = __ldg(src + j);
+            st_shared_v4(dst + (((uint32_t)j ^ xr) << 4), v.x, v.y, v.z, v.w);
           }
         } else {
           // adapter K-blocks carry no packed codes, but the other CTA still vouches for its token half
@@ -586,6 +613,41 @@ __global__ void sample_split_kernel(const __nv_bfloat16* __restrict__ src, int64
   store_split(scale * __bfloat162float(src[t * width + (int64_t)j * stride]), hi, lo, t * ld_out + j);
 }
 
+// Low-bit product, one thread per quantization block (64 codes = 32 bytes): splits the block's offset beta' into
+// beta_c = -alpha * c_mid, which stays inside the bf16 weight operand (c_mid = middle of the codes the block
+// uses, so alpha * c + beta_c is centred on zero and its bf16 rounding error is that of the weight's own spread,
+// whatever shift a merge has put into beta'), and gamma = beta' - beta_c, kept as a bf16 hi + lo pair for the
+// offset-term K-blocks.  The last block of a row also zeroes the row's padding columns.
+__global__ void __launch_bounds__(256) lowbit_center_kernel(const uint8_t* __restrict__ codes, const float* __restrict__ alpha,
+                                                           const float* __restrict__ beta, int64_t nblocks, int G, int ldg,
+                                                           float* __restrict__ beta_c, __nv_bfloat16* __restrict__ gam_h,
+                                                           __nv_bfloat16* __restrict__ gam_l) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= nblocks) return;
+  const uint4* src = reinterpret_cast<const uint4*>(codes + b * 32);
+  const uint4 q0 = __ldg(src), q1 = __ldg(src + 1);
+  const uint32_t w[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+  uint32_t mn = 0x0F0F0F0Fu, mx = 0u;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const uint32_t lo = w[j] & 0x0F0F0F0Fu, hi = (w[j] >> 4) & 0x0F0F0F0Fu;
+    mn = __vminu4(mn, __vminu4(lo, hi));
+    mx = __vmaxu4(mx, __vmaxu4(lo, hi));
+  }
+  mn = __vminu4(mn, mn >> 16); mn = __vminu4(mn, mn >> 8);
+  mx = __vmaxu4(mx, mx >> 16); mx = __vmaxu4(mx, mx >> 8);
+  const float c_mid = 0.5f * (float)((mn & 0xFFu) + (mx & 0xFFu));
+  const float bc = -__fmul_rn(__ldg(alpha + b), c_mid);
+  const float gm = __fsub_rn(__ldg(beta + b), bc);
+  beta_c[b] = bc;
+  const int64_t row = b / G;
+  const int g = (int)(b - row * G);
+  store_split(gm, gam_h, gam_l, row * ldg + g);
+  if (g == G - 1)
+    for (int k = G; k < ldg; ++k) { gam_h[row * ldg + k] = __float2bfloat16_rn(0.0f); gam_l[row * ldg + k] = __float2bfloat16_rn(0.0f); }
+}
+
 int num_sms() {
   static int n = []() {
     int dev = 0, v = 0;
@@ -635,8 +697,17 @@ bool overlap_adapter_prologue() {
 
 // Launches the fused-dequant GEMM.  Bop: X (forward) / dY (backward); Bx: the compressed adapter
 // activation [T][ldx] feeding the extra K-blocks (s * x' A forward, dv B^T / lambda_in backward).
+// Offset term of the low-bit product (see TcParams): per-block table offsets beta_c [d_out][G], gamma = beta' - beta_c
+// as bf16 hi / lo [d_out][ldg], and the group sums of x as bf16 hi / lo [T][ldg].
+struct LowbitTerm {
+  const float* beta_c;
+  const __nv_bfloat16 *gam_h, *gam_l, *s_h, *s_l;
+  int ldg;
+};
+
 int launch_main(int mode, const QwView& qw, const AdView* ad, const __nv_bfloat16* Bop, const __nv_bfloat16* Bx,
-                int ldx, int64_t T, void* out, int out_dtype, int* status, cudaStream_t st) {
+                int ldx, int64_t T, void* out, int out_dtype, int* status, cudaStream_t st,
+                const LowbitTerm* lb = nullptr) {
   static bool attr_set[2] = {false, false};
   if (!attr_set[mode]) {
     cudaError_t e = mode == 0
@@ -665,8 +736,14 @@ int launch_main(int mode, const QwView& qw, const AdView* ad, const __nv_bfloat1
   p.op = ad ? ad->op : 0;
   p.n_small = ad ? (mode == 0 ? ad->Q : ad->P) : 0;
   p.out = out; p.out_dtype = out_dtype; p.status = status;
+  if (lb) {
+    p.beta = lb->beta_c;
+    p.ng_blocks = (qw.G + BK - 1) / BK;
+    p.kb_gamma = 3 * p.ng_blocks;
+    p.gam_h = lb->gam_h; p.gam_l = lb->gam_l; p.gam_ld = lb->ldg;
+  }
 
-  CUtensorMap tm_b, tm_bx, tm_p;
+  CUtensorMap tm_b, tm_bx, tm_p, tm_s, tm_sl;
   int rc = make_tensor_map_2d(&tm_b, false, Bop, (uint64_t)Kq, (uint64_t)T, (uint64_t)Kq * 2, BK, BN_HALF, true);
   if (rc) return rc;
   if (ad) rc = make_tensor_map_2d(&tm_bx, false, Bx, (uint64_t)ad->r, (uint64_t)T, (uint64_t)ldx * 2, BK, BN_HALF, true);
@@ -675,6 +752,14 @@ int launch_main(int mode, const QwView& qw, const AdView* ad, const __nv_bfloat1
   if (mode == 0) rc = make_tensor_map_2d(&tm_p, true, qw.codes, (uint64_t)qw.d_in / 2, (uint64_t)qw.d_out, (uint64_t)qw.d_in / 2, BK / 2, BM, false);
   else rc = make_tensor_map_2d(&tm_p, true, qw.codes, (uint64_t)qw.d_in / 2, (uint64_t)qw.d_out, (uint64_t)qw.d_in / 2, BK / 2, BK, false);
   if (rc) return rc;
+  if (lb) {
+    rc = make_tensor_map_2d(&tm_s, false, lb->s_h, (uint64_t)qw.G, (uint64_t)T, (uint64_t)lb->ldg * 2, BK, BN_HALF, true);
+    if (rc) return rc;
+    rc = make_tensor_map_2d(&tm_sl, false, lb->s_l, (uint64_t)qw.G, (uint64_t)T, (uint64_t)lb->ldg * 2, BK, BN_HALF, true);
+    if (rc) return rc;
+  } else {
+    tm_s = tm_b; tm_sl = tm_b;
+  }
 
   const int tiles = p.m_tiles * p.n_tiles;                      // one tile per CTA pair
   const int pairs = num_sms() / 2;
@@ -688,12 +773,12 @@ int launch_main(int mode, const QwView& qw, const AdView* ad, const __nv_bfloat1
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr; cfg.numAttrs = (ad && overlap_adapter_prologue()) ? 1 : 0;
+  cfg.attrs = attr; cfg.numAttrs = ((ad || lb) && overlap_adapter_prologue()) ? 1 : 0;
   cudaError_t le;
   {
     DominantKernelTimer timer(st);
-    le = mode == 0 ? cudaLaunchKernelEx(&cfg, tc_dq_gemm_kernel<0>, tm_b, tm_bx, tm_p, p)
-                   : cudaLaunchKernelEx(&cfg, tc_dq_gemm_kernel<1>, tm_b, tm_bx, tm_p, p);
+    le = mode == 0 ? cudaLaunchKernelEx(&cfg, tc_dq_gemm_kernel<0>, tm_b, tm_bx, tm_p, tm_s, tm_sl, p)
+                   : cudaLaunchKernelEx(&cfg, tc_dq_gemm_kernel<1>, tm_b, tm_bx, tm_p, tm_s, tm_sl, p);
     count_launch();
   }
   QB_CUDA(le);
@@ -755,6 +840,54 @@ int tc_linear_fwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, in
     if (rc) return rc;
   }
   return launch_main(0, qw, ad, X, w.u16, w.ldr, T, Y, y_dtype, status, st);
+}
+
+// Low-bit product for more than a handful of tokens (Sec. 3.3), 64 x 1 blocks:
+//   Y[t][o] = sum_i x[t][i] bf16(alpha c + beta_c)[o][i] + sum_g gamma[o][g] S[t][g],  S[t][g] = sum of x over group g.
+// Keeping gamma (which carries the merged adapter's shift) out of the bf16 weight operand makes the merged
+// layer agree with the unmerged one to the accuracy of the base weight's own rounding (the merge identity).
+namespace {
+struct LowbitWs {
+  float* beta_c; __nv_bfloat16 *gam_h, *gam_l, *s_h, *s_l; int ldg; size_t bytes;
+};
+LowbitWs carve_lowbit(const QwView& qw, int64_t T, char* ws) {
+  LowbitWs w{};
+  w.ldg = round8(qw.G);
+  size_t off = kStatusBytes;
+  auto take = [&](size_t bytes) { char* ptr = ws ? ws + off : nullptr; off += align_up(bytes, 256); return ptr; };
+  w.beta_c = (float*)take((size_t)qw.d_out * qw.G * 4);
+  w.gam_h = (__nv_bfloat16*)take((size_t)qw.d_out * w.ldg * 2);
+  w.gam_l = (__nv_bfloat16*)take((size_t)qw.d_out * w.ldg * 2);
+  w.s_h = (__nv_bfloat16*)take((size_t)T * w.ldg * 2);
+  w.s_l = (__nv_bfloat16*)take((size_t)T * w.ldg * 2);
+  w.bytes = off;
+  return w;
+}
+}  // namespace
+
+bool tc_lowbit_split_offsets(const QwView& qw) {
+  return qw.qfmt == QBLORA_FMT_AFFINE_MINMAX && qw.block_in == BK && qw.block_out == 1;
+}
+size_t tc_lowbit_ws_bytes(const QwView& qw, int64_t T) {
+  return tc_lowbit_split_offsets(qw) ? carve_lowbit(qw, T, nullptr).bytes : tc_ws_bytes(QBLORA_OP_LINEAR_FWD, qw, nullptr, T);
+}
+int tc_lowbit_gemm(const QwView& qw, const __nv_bfloat16* X, int64_t T, void* Y, int y_dtype, char* ws, cudaStream_t st) {
+  int* status = reinterpret_cast<int*>(ws);
+  if (!tc_lowbit_split_offsets(qw)) return launch_main(0, qw, nullptr, X, nullptr, 0, T, Y, y_dtype, status, st);
+  const LowbitWs w = carve_lowbit(qw, T, ws);
+  const int64_t nblocks = (int64_t)qw.d_out * qw.G;
+  lowbit_center_kernel<<<(unsigned)((nblocks + 255) / 256), 256, 0, st>>>(qw.codes, qw.alpha, qw.beta, nblocks, qw.G, w.ldg,
+                                                                      w.beta_c, w.gam_h, w.gam_l);
+  count_launch();
+  QB_CUDA(cudaGetLastError());
+  // group sums of x (d_in is a multiple of 64 here, so the one-load-per-thread kernel applies)
+  const int64_t chunks = T * (qw.d_in / 8);
+  segsum_split_kernel<false><<<(unsigned)((chunks + 256 * SEGSUM_UNROLL - 1) / (256 * SEGSUM_UNROLL)), 256, 0, st>>>(
+      X, T, qw.d_in, BK, 1.0f, w.ldg, w.s_h, w.s_l);
+  count_launch();
+  QB_CUDA(cudaGetLastError());
+  const LowbitTerm lb{w.beta_c, w.gam_h, w.gam_l, w.s_h, w.s_l, w.ldg};
+  return launch_main(0, qw, nullptr, X, nullptr, 0, T, Y, y_dtype, status, st, &lb);
 }
 
 namespace {

@@ -36,11 +36,18 @@ def normal(seed: int, name: str, shape, std: float = 1.0) -> np.ndarray:
 
 
 def round_to_bf16(a: np.ndarray) -> np.ndarray:
-    """float32 array whose values are the bf16 round-to-nearest-even of ``a``."""
+    """float32 array whose values are the bf16 round-to-nearest-even of ``a`` (non-finite values keep
+    their class)."""
     a = np.ascontiguousarray(a, dtype=np.float32)
-    u = a.view(np.uint32).astype(np.uint64)
-    u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000
-    return u.astype(np.uint32).view(np.float32).reshape(a.shape)
+    u = a.view(np.uint32)
+    out = u + (np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1)))   # cannot wrap for finite values
+    out &= np.uint32(0xFFFF0000)
+    special = (u & np.uint32(0x7F800000)) == np.uint32(0x7F800000)
+    if special.any():
+        nan = special & ((u & np.uint32(0x007FFFFF)) != 0)
+        out[special] = u[special] & np.uint32(0xFFFF0000)
+        out[nan] |= np.uint32(0x00400000)
+    return out.view(np.float32).reshape(a.shape)
 
 
 def bf16_bits(a: np.ndarray) -> np.ndarray:

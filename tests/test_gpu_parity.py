@@ -51,6 +51,42 @@ def test_quantize_bit_exact(qb, qfmt, shape, bi, bo, dtype):
         assert got.beta is None
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_quantize_signed_zero_block_minimum(qb, dtype):
+    # blocks whose minimum is a zero, with zeros of both signs in every order (within a lane's eight elements,
+    # across lanes, across the halves of the block): beta comes out as +0 bit for bit, as in the oracle; also a
+    # block of zeros of mixed sign only, and both formats' codes for the signed zeros.
+    W = np.abs(synth.normal(34, "qz/pm0", (16, 256), 0.02)).astype(np.float32)
+    pz, nz = np.float32(0.0), np.float32(-0.0)
+    W[0, 0], W[0, 1] = pz, nz
+    W[1, 0], W[1, 1] = nz, pz
+    W[2, 3], W[2, 40] = pz, nz
+    W[3, 3], W[3, 40] = nz, pz
+    W[4, 64 + 63], W[4, 64] = nz, pz
+    W[5, 128:192] = pz; W[5, 128:192:2] = nz
+    W[6, 192:256] = nz
+    W[7, 7] = nz
+    if dtype == "bf16":
+        W = synth.round_to_bf16(W)
+        Wd = to_bf16_dev(W)
+    else:
+        Wd = to_dev(W)
+    for qfmt in (0, 1):
+        ref = oracle.quantize_blockwise(W, 64, 1, qfmt)
+        got = qb.quantize_blockwise(Wd, 64, 1, qfmt)
+        assert np.array_equal(got.codes.cpu().numpy(), ref.codes)
+        assert np.array_equal(got.alpha.cpu().numpy().view(np.uint32), ref.alpha.view(np.uint32))
+        if qfmt == 1:
+            gb = got.beta.cpu().numpy().view(np.uint32)
+            assert np.array_equal(gb, ref.beta.view(np.uint32))
+            assert gb[0, 0] == 0 and gb[1, 0] == 0 and gb[5, 2] == 0 and gb[6, 3] == 0 and gb[7, 0] == 0
+    # the general (any block shape) kernel takes the same decision
+    ref = oracle.quantize_blockwise(W, 8, 8, 1)
+    got = qb.quantize_blockwise(Wd, 8, 8, 1)
+    assert np.array_equal(got.beta.cpu().numpy().view(np.uint32), ref.beta.view(np.uint32))
+    assert np.array_equal(got.codes.cpu().numpy(), ref.codes)
+
+
 def test_quantize_round_trip_on_device(qb):
     # Q(D(Q(W))) == Q(W) on the level-table format, dequantizing with the oracle in between
     W = synth.normal(32, "qz/rt", (128, 512), 0.02)
@@ -172,13 +208,16 @@ def test_single_token_and_workspace_errors(qb):
 
 # ------------------------------------------------------------------------- merge + low-bit product
 @pytest.mark.parametrize("single", [False, True])
-@pytest.mark.parametrize("scaling", [1.0, 37.5])
-def test_merge_bit_exact_and_identity(qb, single, scaling):
+@pytest.mark.parametrize("scaling", [1.0, 37.5, "visible"])
+def test_merge_bit_exact_and_identity(qb, path, single, scaling):
+    # 333 token rows (three token tiles with a ragged tail), every row gated.  With P = 7 pooled inputs the
+    # adapter term varies strongly from token to token, so rows where it happens to be small are measured against
+    # a small row RMS: the low-bit product has to keep the merged shift out of its bf16-rounded operand to pass.
     d_out, d_in, r = 320, 448, 48
-    qw, ad, X, _ = make_case(51, 40, d_out, d_in, 64, 8, r, qfmt=1, ab_std=0.02)
+    qw, ad, X, _ = make_case(51, 333, d_out, d_in, 64, 8, r, qfmt=1, ab_std=0.02)
     if single:
         ad = oracle.Adapter(64, 8, 0, scaling, synth.round_to_bf16(synth.normal(51, "H", (d_in // 64, d_out // 8), 0.02)), None)
-    ad.scaling = scaling
+    ad.scaling = visible_scaling(oracle.dequantize(qw), ad, X) if scaling == "visible" else scaling
     ref = oracle.merge(qw, ad)
     dq, da = qweight_to_dev(qw), adapter_to_dev(ad)
     codes0, alpha0 = dq.codes.clone(), dq.alpha.clone()
@@ -190,6 +229,9 @@ def test_merge_bit_exact_and_identity(qb, single, scaling):
     Xd = to_bf16_dev(X)
     unmerged = oracle.linear_fwd(oracle.dequantize(qw), ad, X)
     gate_strict(to_np64(qb.lowbit_gemm(got, Xd, torch.float32)), unmerged, "merged low-bit vs unmerged fwd")
+    gate_bf16(to_np64(qb.lowbit_gemm(got, Xd, torch.bfloat16)), unmerged, "merged low-bit vs unmerged fwd, bf16")
+    for T in (1, 7, 16):      # the decode kernels on the same merged weight
+        gate_strict(to_np64(qb.lowbit_gemm(got, Xd[:T].contiguous(), torch.float32)), unmerged[:T], f"merged decode T={T}")
     if not single:
         gate_strict(to_np64(qb.linear_fwd(dq, da, Xd, torch.float32)), unmerged, "unmerged fwd")
     # in place
@@ -402,3 +444,70 @@ def test_cuda_graph_replay_equals_eager_calls(qb):
             assert torch.equal(Y, eager[k][0]) and torch.equal(dX, eager[k][1]), f"replay {it}"
             assert torch.equal(dA, eager[k][2]) and torch.equal(dB, eager[k][3]), f"replay {it}"
     assert qb.device_status(wf) == 0 and qb.device_status(wb) == 0
+
+
+@pytest.mark.parametrize("T", [9, 12, 16])
+def test_lowbit_decode_k_outer_alternating_inputs_stress(qb, T):
+    # The 2..16-token decode kernel hands shared-memory buffers (weight ring, token-fragment double buffer, row-block
+    # sums) back to its producers with mbarrier arrivals that must not overtake the loads from those buffers.
+    # 200 calls back to back with no host synchronisation, two inputs alternating through ONE workspace (so each
+    # call's fragment area is rewritten while the previous call may still drain); several K tiles (the fragment
+    # buffers are reused) and more than one pass of row blocks per CTA.  Every result equals the lone call's bit
+    # for bit, and the lone call matches the oracle.
+    d_out, d_in = 148 * 2 * 32 + 32 * 5 + 8, 64 * 16 * 5
+    qw, _, X0, _ = make_case(71, T, d_out, d_in, 64, 8, 16, qfmt=1)
+    X1 = synth.round_to_bf16(synth.normal(72, "stress/X1", (T, d_in)) * np.float32(3.0))
+    dq = qweight_to_dev(qw)
+    Xs = [to_bf16_dev(X0), to_bf16_dev(X1)]
+    ws = qb.alloc_workspace(qb.OP_LOWBIT_GEMM, dq, None, T)
+    alone = []
+    for k in range(2):
+        Y = qb.lowbit_gemm(dq, Xs[k], torch.float32, ws=ws)
+        torch.cuda.synchronize()
+        alone.append(Y.clone())
+    gate_strict(to_np64(alone[0]), oracle.lowbit_gemm(qw, X0), f"decode T={T}")
+    gate_strict(to_np64(alone[1]), oracle.lowbit_gemm(qw, X1), f"decode T={T}, second input")
+    assert not torch.equal(alone[0], alone[1])
+    outs = [torch.empty_like(alone[0]) for _ in range(200)]
+    for it in range(200):
+        qb.lowbit_gemm(dq, Xs[it & 1], ws=ws, out=outs[it])
+    torch.cuda.synchronize()
+    bad = [it for it in range(200) if not torch.equal(outs[it], alone[it & 1])]
+    assert not bad, f"calls {bad[:10]} differ from the lone result"
+    assert qb.device_status(ws) == qb.OK
+
+
+@pytest.mark.parametrize("d_out", [72, 4768])
+def test_lowbit_one_token_split_tail_graph_replay(qb, d_out):
+    # ONE one-token call on a split-tail shape captured into a CUDA graph and replayed on alternating inputs in a
+    # static buffer.  A replay carries the hand-over epoch it was captured with, so the owner of a row block must
+    # not take the flags left by the previous replay for this replay's: every replay equals the eager result.
+    qw, _, X0, _ = make_case(73, 1, d_out, 64 * 256, 64, 8, 16, qfmt=1)
+    X1 = synth.round_to_bf16(synth.normal(74, "tail/X1", (1, 64 * 256)) * np.float32(2.0))
+    dq = qweight_to_dev(qw)
+    ins = [to_bf16_dev(X0), to_bf16_dev(X1)]
+    ws = qb.alloc_workspace(qb.OP_LOWBIT_GEMM, dq, None, 1)
+    eager = []
+    for k in range(2):
+        Y = qb.lowbit_gemm(dq, ins[k], torch.float32, ws=ws)
+        torch.cuda.synchronize()
+        eager.append(Y.clone())
+    gate_strict(to_np64(eager[0]), oracle.lowbit_gemm(qw, X0), "split tail")
+    assert not torch.equal(eager[0], eager[1])
+    Xs = torch.empty_like(ins[0])
+    Y = torch.empty_like(eager[0])
+    st = torch.cuda.Stream()
+    with torch.cuda.stream(st):
+        Xs.copy_(ins[0])
+        qb.lowbit_gemm(dq, Xs, ws=ws, out=Y)
+        st.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=st):
+            qb.lowbit_gemm(dq, Xs, ws=ws, out=Y)
+        for it in range(50):
+            k = it & 1
+            Xs.copy_(ins[k])
+            g.replay()
+            st.synchronize()
+            assert torch.equal(Y, eager[k]), f"replay {it}"
+    assert qb.device_status(ws) == qb.OK
