@@ -10,11 +10,34 @@
  *
  * Ownership.  Every pointer in a struct or argument list marked DEVICE is a
  * CUDA device pointer owned by the caller, 16-byte aligned; the library never
- * allocates or frees device memory in these calls, keeps no per-call state, and
- * only enqueues work on the given stream (a cudaStream_t passed as void*,
- * NULL = default stream).  Pointers marked HOST are ordinary host memory read
- * during the call.  Scratch memory is the caller's `ws` buffer of at least
- * qblora_workspace_bytes(...) bytes; its contents are undefined after a call.
+ * allocates or frees device memory in these calls.  Pointers marked HOST are
+ * ordinary host memory read during the call.  Scratch memory is the caller's
+ * `ws` buffer of at least qblora_workspace_bytes(...) bytes; its contents are
+ * undefined after a call, and two calls that may run concurrently on the GPU
+ * need separate `ws` buffers.
+ *
+ * Streams.  Work is enqueued on the given stream (a cudaStream_t passed as
+ * void*, NULL = default stream), with ONE exception: qblora_linear_bwd runs its
+ * adapter-gradient chain on a second stream that the library creates on first
+ * use and keeps (one non-blocking stream and three events per host thread and
+ * device, never destroyed).  That stream is forked from `stream` at entry and
+ * joined back into it before the call returns -- also when the call returns an
+ * error after the fork -- so the caller sees ordinary stream semantics, inside a
+ * stream capture too.  All caller streams of one host thread share that second
+ * stream: do not capture qblora_linear_bwd on one stream while the same thread
+ * runs it un-captured on another.
+ *
+ * State the library keeps between calls (none of it per call):
+ *   - the second stream and events above (thread-local);
+ *   - per-kernel "shared-memory attribute set" flags and the SM count (atomic,
+ *     set once);
+ *   - the device address of the built-in scratch of qablora_merge_noalloc, per
+ *     device (atomic, set once);
+ *   - the launch counter and the armed event pair of the instrumentation calls,
+ *     and the values set by the qblora_debug_* test hooks (atomic / thread-local).
+ * Every entry point may be called from several host threads at once; calls that
+ * share a `ws` buffer, or qablora_merge_noalloc calls on one device, must be
+ * serialised by the caller.
  *
  * Errors.  Every call returns a qblora_status; nothing throws or aborts.
  * Argument checks are made on the host before any launch.  Device-side waits
@@ -128,6 +151,18 @@ int qblora_device_status(const void* ws, void* stream);
  * on the call's stream, then disarms.  Pass NULL, NULL to disarm.  The paper has no counterpart. */
 uint64_t qblora_kernel_launches(void);
 int qblora_set_timing_events(void* start_event, void* stop_event);
+
+/* Test hooks for the bounded device-side waits (process-wide host state; the paper has no counterpart).
+ * qblora_debug_set_wait_limit(cycles): kernels launched from now on give up a wait after `cycles` SM clock
+ *   cycles instead of the default 2 * 10^9 (0 restores the default).
+ * qblora_debug_drop_load(iteration): in the NEXT launch of the fused dequant contraction (qblora_linear_fwd /
+ *   qblora_linear_bwd / the large-token qablora_lowbit_gemm) the producer of every CTA announces the bytes of
+ *   its `iteration`-th weight K-block to the stage's barrier but issues no copy, so that barrier never
+ *   completes: every role of the kernel runs into its wait limit, the kernel stores QBLORA_ERR_TIMEOUT in the
+ *   status word, releases its tensor memory and returns by itself; the outputs of that call are undefined.
+ *   Negative = disarm.  Use together with a short wait limit. */
+int qblora_debug_set_wait_limit(int64_t cycles);
+int qblora_debug_drop_load(int32_t iteration);
 
 /*
  * Block-wise 4-bit quantization, Eq. 1 (Sec. 3.1).

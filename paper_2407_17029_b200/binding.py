@@ -31,7 +31,7 @@ EXPORTS = ["qblora_default_code_table", "qblora_workspace_bytes", "qblora_status
            "qblora_device_status", "qblora_quantize_blockwise", "qblora_linear_fwd",
            "qblora_linear_bwd", "qablora_merge", "qablora_lowbit_gemm", "qblora_kernel_launches",
            "qblora_set_timing_events", "qablora_merge_noalloc", "qblora_merge_dense",
-           "qblora_quantize_minmax_nbit"]
+           "qblora_quantize_minmax_nbit", "qblora_debug_set_wait_limit", "qblora_debug_drop_load"]
 
 
 class _CQWeight(ctypes.Structure):
@@ -82,6 +82,8 @@ _lib.qblora_merge_dense.restype = ctypes.c_int
 _lib.qblora_kernel_launches.restype = ctypes.c_uint64
 _lib.qblora_kernel_launches.argtypes = []
 _lib.qblora_set_timing_events.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
+_lib.qblora_debug_set_wait_limit.argtypes = [ctypes.c_int64]
+_lib.qblora_debug_drop_load.argtypes = [ctypes.c_int32]
 
 
 def kernel_launches() -> int:
@@ -94,6 +96,21 @@ def set_timing_events(start, stop) -> None:
         _lib.qblora_set_timing_events(None, None)
     else:
         _lib.qblora_set_timing_events(start.cuda_event, stop.cuda_event)
+
+
+def debug_set_wait_limit(cycles: int) -> None:
+    """Test hook: device-side waits of kernels launched from now on give up after `cycles` cycles (0 = default)."""
+    _check_plain(_lib.qblora_debug_set_wait_limit(int(cycles)))
+
+
+def debug_drop_load(iteration: int) -> None:
+    """Test hook: the next fused-contraction launch leaves out one weight load (see the header); negative = disarm."""
+    _check_plain(_lib.qblora_debug_drop_load(int(iteration)))
+
+
+def _check_plain(status: int):
+    if status != OK:
+        raise RuntimeError(f"status {status}")
 
 
 class QbloraError(RuntimeError):
@@ -278,11 +295,13 @@ def linear_bwd(qw: QWeight, ad: Optional[Adapter], X: Optional[torch.Tensor], dY
 
 
 def merge(qw: QWeight, ad: Adapter, in_place: bool = False, ws: Optional[torch.Tensor] = None,
-          stream=None) -> QWeight:
-    """QA-BLoRA merge: returns the weight with beta' (codes and alpha are shared, untouched)."""
+          stream=None, beta_out: Optional[torch.Tensor] = None) -> QWeight:
+    """QA-BLoRA merge: returns the weight with beta' (codes and alpha are shared, untouched).
+    `beta_out`: preallocated fp32 tensor of beta's shape to receive beta'."""
     if qw.beta is None:
         raise QbloraError(ERR_INVALID_ARG, "qablora_merge")
-    beta_out = qw.beta if in_place else torch.empty_like(qw.beta)
+    if beta_out is None:
+        beta_out = qw.beta if in_place else torch.empty_like(qw.beta)
     if ws is None:
         ws = alloc_workspace(OP_MERGE, qw, ad, 0)
     cq = qw.c_struct()

@@ -47,6 +47,12 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 // ---- instrumentation (instrument.cu) ------------------------------------------------------------
 void count_launch(int n = 1);
+// Device-side waits give up after this many cycles (~1 s: far beyond any legitimate wait) unless
+// qblora_debug_set_wait_limit has set another value; every launch passes the current value to its kernel.
+constexpr long long kDefaultWaitLimitCycles = 2000000000LL;
+long long wait_limit_cycles();
+// Test hook armed by qblora_debug_drop_load: returns the armed producer iteration once (then -1 again).
+int take_dropped_load();
 // Brackets the dominant kernel of a call with the armed event pair (if any), then disarms.
 struct DominantKernelTimer {
   cudaStream_t st; cudaEvent_t stop;

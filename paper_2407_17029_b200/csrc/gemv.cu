@@ -156,11 +156,11 @@ __device__ __forceinline__ bool gv_try_wait_hint(uint32_t bar, uint32_t parity) 
       : "=r"(ok) : "r"(bar), "r"(parity), "r"(100000u) : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ bool gv_wait(uint32_t bar, uint32_t parity, int* status) {
+__device__ __forceinline__ bool gv_wait(uint32_t bar, uint32_t parity, int* status, long long limit) {
   if (gv_try_wait_hint(bar, parity)) return true;
   const long long t0 = clock64();
   while (!gv_try_wait_hint(bar, parity)) {
-    if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+    if (clock64() - t0 > limit) {
       atomicExch(status, (int)QBLORA_ERR_TIMEOUT);
       return false;
     }
@@ -178,6 +178,7 @@ struct GtParams {
   int* status;
   // one-token kernel, split tail (see T1Walk): row blocks done whole, ways the rest is split, hand-over area
   int tail_first, tail_split;
+  long long wait_limit;      // cycles after which a device-side wait gives up
   uint32_t zero;             // always 0; unknown to the compiler (see gv_release)
   uint32_t epoch;            // value a hand-over flag takes in this launch (never 0, differs from launch to launch)
   float* tail_partial;       // [tail row block][part][32 rows] fp32
@@ -270,7 +271,7 @@ lowbit_gemv_t1_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
       while (ok && walk.next(p)) {
         const int rb = walk.rb;
         for (int kc = walk.kc0; kc < walk.kc1; ++kc, ++it) {
-          if (!gv_wait(empty(s), ph ^ 1u, p.status)) { ok = false; break; }
+          if (!gv_wait(empty(s), ph ^ 1u, p.status, p.wait_limit)) { ok = false; break; }
           const uint32_t st = base + s * GT_STAGE_BYTES;
           mbar_arrive_expect_tx(full(s), GT_STAGE_BYTES);
 #pragma unroll
@@ -283,7 +284,7 @@ lowbit_gemv_t1_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
       }
       if (!ok) {   // give copies already in flight a bounded chance to land before the CTA exits
         const uint32_t lo = it > (uint32_t)STAGES ? it - STAGES : 0;
-        for (uint32_t j = lo; j < it; ++j) gv_wait(full(j % STAGES), (j / STAGES) & 1u, p.status);
+        for (uint32_t j = lo; j < it; ++j) gv_wait(full(j % STAGES), (j / STAGES) & 1u, p.status, p.wait_limit);
       }
     }
   } else {
@@ -366,7 +367,7 @@ lowbit_gemv_t1_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
       const int rb = walk.rb;
       float y[2][2] = {{0.0f, 0.0f}, {0.0f, 0.0f}};    // [row tile][row g, row g + 8], token 0 (lanes tg == 0)
       for (int kc = walk.kc0; kc < walk.kc1; ++kc) {
-        if (ok && !gv_wait(full(s), ph, p.status)) ok = false;
+        if (ok && !gv_wait(full(s), ph, p.status, p.wait_limit)) ok = false;
         const int grp = kc * GT_GROUPS + warp;
         if (ok) {
           if (grp < p.G) {                                   // warp-uniform
@@ -407,7 +408,7 @@ lowbit_gemv_t1_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
       // slot (once the warp that summed the previous row block has let go of the buffer) and arrives
       // on red_done; the sixteen slots are then summed in slot order (deterministic) and stored by
       // warp (row block count) % 16, which is the only warp that waits for the others.
-      if (ok && !gv_wait(red_free, rph ^ 1u, p.status)) ok = false;
+      if (ok && !gv_wait(red_free, rph ^ 1u, p.status, p.wait_limit)) ok = false;
       float* my_red = red + warp * GT_ROWS;
       if (tg == 0) {
 #pragma unroll
@@ -416,7 +417,7 @@ lowbit_gemv_t1_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
       __syncwarp();
       if (lane == 0) mbar_arrive(red_done);
       if (warp == (int)(rcount & 15u)) {
-        if (ok && !gv_wait(red_done, rph, p.status)) ok = false;
+        if (ok && !gv_wait(red_done, rph, p.status, p.wait_limit)) ok = false;
         float a = 0.0f;
 #pragma unroll
         for (int ww = 0; ww < GT_WARPS; ++ww) a += red[ww * GT_ROWS + lane];
@@ -439,7 +440,7 @@ lowbit_gemv_t1_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
               const long long w0 = clock64();
               while ((seen = *reinterpret_cast<volatile uint32_t*>(p.tail_flags + slot + part)) != p.epoch) {
                 __nanosleep(100);
-                if (clock64() - w0 > WAIT_LIMIT_CYCLES) { atomicExch(p.status, (int)QBLORA_ERR_TIMEOUT); break; }
+                if (clock64() - w0 > p.wait_limit) { atomicExch(p.status, (int)QBLORA_ERR_TIMEOUT); break; }
               }
             }
             seen = __shfl_sync(0xFFFFFFFFu, seen, 0);
@@ -630,7 +631,7 @@ lowbit_gemv_ko_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
           for (int j = 0; j < RB; ++j) {
             const int rb = (pass * RB + j) * gridDim.x + blockIdx.x;
             if (rb >= p.n_rb) break;
-            if (!gv_wait(empty(s), ph ^ 1u, p.status)) { ok = false; break; }
+            if (!gv_wait(empty(s), ph ^ 1u, p.status, p.wait_limit)) { ok = false; break; }
             const uint32_t st = base + s * GT_STAGE_BYTES;
             mbar_arrive_expect_tx(full(s), GT_STAGE_BYTES);
 #pragma unroll
@@ -645,7 +646,7 @@ lowbit_gemv_ko_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
       }
       if (!ok) {   // give copies already in flight a bounded chance to land before the CTA exits
         const uint32_t lo = it > (uint32_t)STAGES ? it - STAGES : 0;
-        for (uint32_t j = lo; j < it; ++j) gv_wait(full(j % STAGES), (j / STAGES) & 1u, p.status);
+        for (uint32_t j = lo; j < it; ++j) gv_wait(full(j % STAGES), (j / STAGES) & 1u, p.status, p.wait_limit);
       }
     }
   } else if (warp == GT_WARPS + 1) {
@@ -658,14 +659,14 @@ lowbit_gemv_ko_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
         if (pass * RB * (int)gridDim.x + (int)blockIdx.x >= p.n_rb) break;
         for (int kc = 0; kc < p.n_kc; ++kc, ++xit) {
           const uint32_t xb = xit & 1u;
-          if (!gv_wait(xempty(xb), ((xit >> 1) & 1u) ^ 1u, p.status)) { ok = false; break; }
+          if (!gv_wait(xempty(xb), ((xit >> 1) & 1u) ^ 1u, p.status, p.wait_limit)) { ok = false; break; }
           mbar_arrive_expect_tx(xfull(xb), Cfg::KT_BYTES);
           gv_bulk_load(base + xbuf_off + xb * Cfg::KT_BYTES, xfrag + (size_t)kc * Cfg::KT_BYTES, Cfg::KT_BYTES, xfull(xb));
         }
       }
       if (!ok) {
         const uint32_t xlo = xit > 2u ? xit - 2u : 0u;
-        for (uint32_t j = xlo; j < xit; ++j) gv_wait(xfull(j & 1u), (j >> 1) & 1u, p.status);
+        for (uint32_t j = xlo; j < xit; ++j) gv_wait(xfull(j & 1u), (j >> 1) & 1u, p.status, p.wait_limit);
       }
     }
   } else {
@@ -695,7 +696,7 @@ lowbit_gemv_ko_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
       for (int kc = 0; kc < p.n_kc; ++kc, ++xit) {
         // ---- this warp's group of the K tile: fragments and offsets into registers, once for all row blocks
         const uint32_t xb = xit & 1u;
-        if (ok && !gv_wait(xfull(xb), (xit >> 1) & 1u, p.status)) ok = false;
+        if (ok && !gv_wait(xfull(xb), (xit >> 1) & 1u, p.status, p.wait_limit)) ok = false;
         uint32_t f[NT][8];
         float4 sg[NT][2];
 #pragma unroll
@@ -713,7 +714,7 @@ lowbit_gemv_ko_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
         for (int j = 0; j < RB; ++j) {
           const int rb = (pass * RB + j) * gridDim.x + blockIdx.x;
           if (rb >= p.n_rb) break;
-          if (ok && !gv_wait(full(s), ph, p.status)) ok = false;
+          if (ok && !gv_wait(full(s), ph, p.status, p.wait_limit)) ok = false;
           if (ok) {
             if (group_live) {
               const uint32_t sb = base + (uint32_t)s * GT_STAGE_BYTES;
@@ -767,7 +768,7 @@ lowbit_gemv_ko_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
       for (int j = 0; j < RB; ++j) {
         const int rb = (pass * RB + j) * gridDim.x + blockIdx.x;
         if (rb >= p.n_rb) break;
-        if (ok && !gv_wait(red_free, rph ^ 1u, p.status)) ok = false;
+        if (ok && !gv_wait(red_free, rph ^ 1u, p.status, p.wait_limit)) ok = false;
         float* my_red = red + warp * GT_ROWS * NTOK;
 #pragma unroll
         for (int n = 0; n < NT; ++n)
@@ -783,7 +784,7 @@ lowbit_gemv_ko_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_con
         if (lane == 0) mbar_arrive(red_done);
         const int t = (warp - (int)(rcount & 15u)) & 15;    // the token this warp sums (if it exists)
         if (t < p.T) {
-          if (ok && !gv_wait(red_done, rph, p.status)) ok = false;
+          if (ok && !gv_wait(red_done, rph, p.status, p.wait_limit)) ok = false;
           float a = 0.0f;
 #pragma unroll
           for (int ww = 0; ww < GT_WARPS; ++ww) a += red[(ww * NTOK + t) * GT_ROWS + (lane ^ (((t >> 1) & 3) << 3))];
@@ -860,6 +861,7 @@ int launch_lowbit_gemv(const QwView& qw, const __nv_bfloat16* X, int64_t T, void
   p.n_rb = (qw.d_out + GT_ROWS - 1) / GT_ROWS;
   p.n_kc = (qw.G + GT_GROUPS - 1) / GT_GROUPS;
   p.X = X; p.Y = Y; p.y_dtype = y_dtype; p.status = status;
+  p.wait_limit = wait_limit_cycles();
   CUtensorMap tm_c, tm_a, tm_b;
   // codes as 32-bit words: [d_out][d_in / 8], boxes of 32 words (four groups) x 32 rows, 128-byte swizzle
   int rc = make_tensor_map_2d_typed(&tm_c, TM_U32, qw.codes, (uint64_t)qw.d_in / 8, (uint64_t)qw.d_out,

@@ -9,7 +9,15 @@ namespace {
 std::atomic<uint64_t> g_launches{0};
 thread_local cudaEvent_t t_start = nullptr;
 thread_local cudaEvent_t t_stop = nullptr;
+std::atomic<long long> g_wait_limit{0};   // 0 = default
+std::atomic<int> g_drop_load{-1};
 }  // namespace
+
+long long wait_limit_cycles() {
+  const long long v = g_wait_limit.load(std::memory_order_relaxed);
+  return v > 0 ? v : kDefaultWaitLimitCycles;
+}
+int take_dropped_load() { return g_drop_load.exchange(-1, std::memory_order_relaxed); }
 
 void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 
@@ -25,6 +33,15 @@ DominantKernelTimer::~DominantKernelTimer() {
 
 extern "C" {
 uint64_t qblora_kernel_launches(void) { return qb::g_launches.load(std::memory_order_relaxed); }
+int qblora_debug_set_wait_limit(int64_t cycles) {
+  if (cycles < 0) return QBLORA_ERR_INVALID_ARG;
+  qb::g_wait_limit.store((long long)cycles, std::memory_order_relaxed);
+  return QBLORA_OK;
+}
+int qblora_debug_drop_load(int32_t iteration) {
+  qb::g_drop_load.store(iteration < 0 ? -1 : (int)iteration, std::memory_order_relaxed);
+  return QBLORA_OK;
+}
 int qblora_set_timing_events(void* start_event, void* stop_event) {
   qb::t_start = static_cast<cudaEvent_t>(start_event);
   qb::t_stop = static_cast<cudaEvent_t>(stop_event);

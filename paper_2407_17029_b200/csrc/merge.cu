@@ -1,5 +1,7 @@
 // QA-BLoRA merge (Sec. 3.3): fold the adapter into the per-block beta of the min-max format.
 // Two small kernels: H = A B in fp64 (P x Q values), then beta' = beta + s * H / lambda_in.
+#include <atomic>
+
 #include "common.cuh"
 
 namespace qb {
@@ -151,17 +153,18 @@ int64_t merge_noalloc_capacity() { return kStaticMergeElems; }
 // that device current) and cached; that lookup is the only set-up this path needs.
 int launch_merge_noalloc(const QwView& qw, const AdView& ad, bool single, float* beta_out, cudaStream_t st) {
   constexpr int kMaxDevices = 64;
-  static double* scratch_of_device[kMaxDevices] = {};
+  static std::atomic<double*> scratch_of_device[kMaxDevices];   // atomic: host threads may race to fill an entry (same value)
   int dev = -1;
   QB_CUDA(cudaGetDevice(&dev));
   if (dev < 0 || dev >= kMaxDevices) return QBLORA_ERR_UNSUPPORTED;
-  if (!scratch_of_device[dev]) {
+  double* H = scratch_of_device[dev].load(std::memory_order_acquire);
+  if (!H) {
     double* ptr = nullptr;
     QB_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_merge_scratch));
     if (!ptr) return QBLORA_ERR_CUDA;
-    scratch_of_device[dev] = ptr;
+    scratch_of_device[dev].store(ptr, std::memory_order_release);
+    H = ptr;
   }
-  double* H = scratch_of_device[dev];
   // every one of the P * Q entries read below is written first, so nothing has to be cleared
   int64_t n = (int64_t)ad.P * ad.Q;
   merge_h_kernel<<<(unsigned)((n + 127) / 128), 128, 0, st>>>(ad.A, ad.B, ad.P, ad.Q, ad.r, single, H);

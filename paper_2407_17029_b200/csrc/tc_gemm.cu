@@ -15,16 +15,18 @@
 // live in TMEM (2 x 256 columns, double-buffered so the epilogue of one tile overlaps the mainloop
 // of the next).
 //
-// Warp roles (448 threads per CTA): warp 0 TMA producer; warp 1 MMA issuer (leader CTA only) and
-// TMEM owner; warps 2-9 two dequant groups taking alternate K-blocks (those of the other CTA report
-// each finished stage to the leader's barrier); warps 10-13 epilogue.  Every mbarrier wait is bounded;
-// on expiry the kernel stores QBLORA_ERR_TIMEOUT in the workspace status word and every role
-// leaves its loop.
+// Warp roles: warp 0 TMA producer; warp 1 MMA issuer (leader CTA only) and TMEM owner; then the dequant
+// groups of four warps each, taking the K-blocks in turn (two groups in the forward, three in the backward;
+// those of the other CTA report each finished stage to the leader's barrier); the last four warps are the
+// epilogue.  Every mbarrier wait is bounded; on expiry the kernel stores QBLORA_ERR_TIMEOUT in the workspace
+// status word and every role leaves its loop.
 #include <cuda.h>
+
+#include <atomic>
+#include <cstdlib>
 
 #include "common.cuh"
 #include "simt_gemm.cuh"
-#include <cstdlib>
 #include "tc_ptx.cuh"
 #include "tc_small.cuh"
 
@@ -41,8 +43,22 @@ constexpr int STAGES = 6;
 constexpr int A_BYTES = BM * BK * 2;        // 16 KB dequantized weight tile
 constexpr int B_BYTES = BN_HALF * BK * 2;   // 16 KB: this CTA's half of the token tile
 constexpr int P_BYTES = BM * BK / 2;        // 4 KB packed codes
-constexpr int NUM_THREADS = 448;            // 14 warps, see roles above
 constexpr int SMEM_BYTES = STAGES * (A_BYTES + B_BYTES + P_BYTES) + 512 + 1024;
+static_assert(SMEM_BYTES <= 227 * 1024, "shared memory of the fused contraction");
+
+// Warp roles.  Dequant groups of 128 threads take the K-blocks in turn (group g: index % NG == g).  The forward
+// runs two groups; the backward three: its scale loads touch a new row of alpha / beta in every K-block (the
+// forward walks along a row and mostly hits the L1), so one of its groups spends longer per K-block and two of
+// them could not keep the tensor pipe fed (C4 shapes, kernel alone: backward 950 -> 1100 TFLOP/s with three
+// groups and the scales of a group's next K-block loaded one K-block ahead; the forward measured the same with
+// two or three groups and slower with the early load).
+template <int MODE>
+struct Roles {
+  static constexpr int NG = MODE == 0 ? 2 : 3;
+  static constexpr int EPI_WARP0 = 2 + 4 * NG;            // four epilogue warps behind the dequant warps
+  static constexpr int NUM_THREADS = (EPI_WARP0 + 4) * 32;
+  static constexpr bool SCALES_AHEAD = MODE == 1;
+};
 
 struct TcParams {
   int M;                    // output rows of the tile grid: d_out (forward) / d_in (backward)
@@ -68,6 +84,8 @@ struct TcParams {
   void* out;                // forward Y [T][d_out]; backward dX [T][d_in]
   int out_dtype;
   int* status;
+  long long wait_limit;     // cycles after which a device-side wait gives up
+  int drop_load;            // test hook: the producers leave out the loads of this K-block iteration (-1: none)
 };
 
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
@@ -133,10 +151,11 @@ __device__ __forceinline__ void dequant_direct8(uint32_t w, int word, const floa
 }
 
 template <int MODE>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(Roles<MODE>::NUM_THREADS, 1)
 tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ CUtensorMap tm_bx,
                   const __grid_constant__ CUtensorMap tm_p, const __grid_constant__ CUtensorMap tm_s,
                   const __grid_constant__ CUtensorMap tm_sl, const __grid_constant__ TcParams p) {
+  constexpr int NG = Roles<MODE>::NG, EPI_WARP0 = Roles<MODE>::EPI_WARP0;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -189,15 +208,19 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
         for (int kb = 0; kb < kb_total; ++kb, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1u;
-          if (!mbar_wait(empty(s), ph ^ 1u, p.status)) { ok = false; break; }
+          if (!mbar_wait(empty(s), ph ^ 1u, p.status, p.wait_limit)) { ok = false; break; }
           if (kb < p.kb_base) {
             mbar_arrive_expect_tx(full(s), B_BYTES + P_BYTES);
-            tma_load_2d(sB + s * B_BYTES, &tm_b, full(s), kb * BK, t0);
-            if (MODE == 0) {
-              tma_load_2d(sP + s * P_BYTES, &tm_p, full(s), kb * (BK / 2), m0);
-            } else {   // two boxes of 64 rows x 32 bytes: packed[ng][k][32 B]
-              tma_load_2d(sP + s * P_BYTES, &tm_p, full(s), m0 / 2, kb * BK);
-              tma_load_2d(sP + s * P_BYTES + P_BYTES / 2, &tm_p, full(s), m0 / 2 + 32, kb * BK);
+            // test hook (qblora_debug_drop_load): the bytes are announced and never sent, so this stage's
+            // barrier cannot complete and every role has to run into its wait limit and leave by itself
+            if ((int)it != p.drop_load) {
+              tma_load_2d(sB + s * B_BYTES, &tm_b, full(s), kb * BK, t0);
+              if (MODE == 0) {
+                tma_load_2d(sP + s * P_BYTES, &tm_p, full(s), kb * (BK / 2), m0);
+              } else {   // two boxes of 64 rows x 32 bytes: packed[ng][k][32 B]
+                tma_load_2d(sP + s * P_BYTES, &tm_p, full(s), m0 / 2, kb * BK);
+                tma_load_2d(sP + s * P_BYTES + P_BYTES / 2, &tm_p, full(s), m0 / 2 + 32, kb * BK);
+              }
             }
           } else {
             // The compressed adapter activation is written by the kernel launched just before this one.  With the
@@ -219,7 +242,7 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
       }
       if (!ok) {  // give copies already in flight a bounded chance to land before the CTA exits
         const uint32_t lo = it > (uint32_t)STAGES ? it - STAGES : 0;
-        for (uint32_t j = lo; j < it; ++j) mbar_wait(full(j % STAGES), (j / STAGES) & 1u, p.status);
+        for (uint32_t j = lo; j < it; ++j) mbar_wait(full(j % STAGES), (j / STAGES) & 1u, p.status, p.wait_limit);
       }
     }
   } else if (warp == 1) {
@@ -230,39 +253,51 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
       const uint32_t idesc_common = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) |
                                     ((uint32_t)((2 * BM) >> 4) << 24);
       const uint32_t idesc_kmajor = idesc_common, idesc_mnmajor = idesc_common | (1u << 15);
-      uint32_t it = 0;
+      // One thread issues every MMA of the pair, so its instruction count per K-block is on the critical path:
+      // the shared-memory descriptors are kept as running 64-bit values (constant upper half; the 14-bit start
+      // address field moves by 2 per 32 bytes), the stage index and phase are counters, and the weight and
+      // adapter K-blocks have loops of their own.
+      const uint64_t dhi_k = smem_desc(0, 16, 1024), dhi_mn = smem_desc(0, 8192, 1024);   // upper halves (address 0)
+      const uint32_t a_lo0 = (sA & 0x3FFFFu) >> 4, b_lo0 = (sB & 0x3FFFFu) >> 4;
       bool ok = true;
-      int lt = 0;
+      int lt = 0, s = 0;
+      uint32_t ph = 0;
       for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters, ++lt) {
         const int a = lt & 1;
         const uint32_t aph = (lt >> 1) & 1u;
-        if (!mbar_wait(accempty(a), aph ^ 1u, p.status)) { ok = false; break; }
+        if (!mbar_wait(accempty(a), aph ^ 1u, p.status, p.wait_limit)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(a * BN);
-        for (int kb = 0; kb < kb_total; ++kb, ++it) {
-          const int s = it % STAGES;
-          const uint32_t ph = (it / STAGES) & 1u;
-          if (!mbar_wait(full(s), ph, p.status) || !mbar_wait(aready(s), ph, p.status) ||
-              !mbar_wait(peer(s), ph, p.status)) { ok = false; break; }
-          tc_fence_after();
-          // weight K-blocks: K-major tile in the forward, MN-major in the backward; the adapter
-          // K-blocks are written the other way round (see the dequant warps)
-          const bool a_kmajor = kb >= kb_gamma0 || (MODE == 0) == (kb < p.kb_base);
+        uint32_t acc = 0;   // the first MMA of a tile overwrites the accumulator
+        // weight K-blocks [0, kb_base): K-major tile in the forward, MN-major in the backward; adapter K-blocks
+        // [kb_base, kb_gamma0): the other way round (see the dequant warps); offset-term K-blocks: K-major
+        for (int part = 0; part < 3 && ok; ++part) {
+          const int n_kb = part == 0 ? p.kb_base : part == 1 ? p.kb_extra : p.kb_gamma;
+          const bool a_kmajor = part == 2 || (MODE == 0) == (part == 0);
+          const uint64_t dhi_a = a_kmajor ? dhi_k : dhi_mn;
+          const uint32_t a_step = a_kmajor ? 2u : 128u;      // 32 bytes / 2048 bytes per K = 16, in 16-byte units
+          const uint32_t idesc = a_kmajor ? idesc_kmajor : idesc_mnmajor;
+          for (int kb = 0; kb < n_kb; ++kb) {
+            if (!mbar_wait(full(s), ph, p.status, p.wait_limit) || !mbar_wait(aready(s), ph, p.status, p.wait_limit) ||
+                !mbar_wait(peer(s), ph, p.status, p.wait_limit)) { ok = false; break; }
+            tc_fence_after();
+            const uint64_t adesc = dhi_a | (uint64_t)(a_lo0 + (uint32_t)s * (A_BYTES >> 4));
+            const uint64_t bdesc = dhi_k | (uint64_t)(b_lo0 + (uint32_t)s * (B_BYTES >> 4));
 #pragma unroll
-          for (int k = 0; k < BK / 16; ++k) {
-            const uint64_t adesc = a_kmajor ? smem_desc(sA + s * A_BYTES + k * 32, 16, 1024)
-                                            : smem_desc(sA + s * A_BYTES + k * 2048, 8192, 1024);
-            const uint64_t bdesc = smem_desc(sB + s * B_BYTES + k * 32, 16, 1024);
-            tc_mma_pair(d_tmem, adesc, bdesc, a_kmajor ? idesc_kmajor : idesc_mnmajor, (kb | k) != 0 ? 1u : 0u);
+            for (int k = 0; k < BK / 16; ++k) {
+              tc_mma_pair(d_tmem, adesc + (uint64_t)(k * a_step), bdesc + (uint64_t)(k * 2), idesc, acc);
+              acc = 1u;
+            }
+            tc_commit_pair(empty(s));
+            if (++s == STAGES) { s = 0; ph ^= 1u; }
           }
-          tc_commit_pair(empty(s));
         }
         if (ok) tc_commit_pair(accfull(a));
       }
     }
-  } else if (warp < 10) {
-    // ------------------------------------------------------------------ dequant warps: two groups of 128
-    // threads; group g fills the stages of K-blocks with (global index & 1) == g.  Thread d owns one
+  } else if (warp < EPI_WARP0) {
+    // ------------------------------------------------------------------ dequant warps: NG groups of 128
+    // threads; group g fills the stages of K-blocks with (global index % NG) == g.  Thread d owns one
     // quantization block (64 codes, one alpha/beta) of the tile per K-block.
     const int g = (warp - 2) >> 2;
     const int d = tid - 64 - 128 * g;
@@ -271,10 +306,29 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
     asm volatile("" : "+r"(k_m4), "+r"(k_c3210));
     bool ok = true;
     uint32_t it = 0;
+    float al_next = 0.0f, be_next = 0.0f;   // scale and offset of this group's next weight K-block of the tile,
+    bool have_next = false;                 // loaded one K-block ahead (the load's latency hides under the look-ups)
     for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
       const int m0 = (tile % p.m_tiles) * (2 * BM) + (int)rank * BM;
+      // (alpha, beta) of this thread's quantization block in weight K-block kb
+      auto load_scale = [&](int kb, float& al, float& be) {
+        al = 0.0f; be = 0.0f;
+        if (MODE == 0) {
+          const int row = m0 + d;
+          if (row < p.d_out) {
+            al = __ldg(p.alpha + (int64_t)row * p.G + kb);
+            if (p.beta) be = __ldg(p.beta + (int64_t)row * p.G + kb);
+          }
+        } else {
+          const int o = kb * BK + (d & 63), blk = (m0 >> 6) + (d >> 6);
+          if (o < p.d_out && blk < p.G) {
+            al = __ldg(p.alpha + (int64_t)o * p.G + blk);
+            if (p.beta) be = __ldg(p.beta + (int64_t)o * p.G + blk);
+          }
+        }
+      };
       for (int kb = 0; kb < kb_total; ++kb, ++it) {
-        if ((int)(it & 1u) != g) continue;
+        if ((int)(it % (uint32_t)NG) != g) continue;
         const int s = it % STAGES;
         const uint32_t ph = (it / STAGES) & 1u;
         const uint32_t a_stage = sA + s * A_BYTES;
@@ -304,11 +358,12 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
                 be[4 * k] = b4.x; be[4 * k + 1] = b4.y; be[4 * k + 2] = b4.z; be[4 * k + 3] = b4.w;
               }
           }
-          if (!mbar_wait(full(s), ph, p.status) || !mbar_wait(empty(s), ph ^ 1u, p.status)) { ok = false; break; }
+          if (!mbar_wait(full(s), ph, p.status, p.wait_limit)) { ok = false; break; }
           const uint8_t* src = gP + s * P_BYTES + d * 32;
           const uint4 q0 = *reinterpret_cast<const uint4*>(src);
           const uint4 q1 = *reinterpret_cast<const uint4*>(src + 16);
           const uint32_t w[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+          if (!mbar_wait(empty(s), ph ^ 1u, p.status, p.wait_limit)) { ok = false; break; }
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             uint32_t o4[4];
@@ -317,27 +372,18 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
             st_shared_v4(dst + (((uint32_t)j ^ xr) << 4), o4[0], o4[1], o4[2], o4[3]);
           }
         } else if (kb < p.kb_base) {
-          float al = 0.0f, be = 0.0f;
-          if (MODE == 0) {
-            const int row = m0 + d;
-            if (row < p.d_out) {
-              al = __ldg(p.alpha + (int64_t)row * p.G + kb);
-              if (p.beta) be = __ldg(p.beta + (int64_t)row * p.G + kb);
-            }
-          } else {
-            const int o = kb * BK + (d & 63), blk = (m0 >> 6) + (d >> 6);
-            if (o < p.d_out && blk < p.G) {
-              al = __ldg(p.alpha + (int64_t)o * p.G + blk);
-              if (p.beta) be = __ldg(p.beta + (int64_t)o * p.G + blk);
-            }
-          }
+          float al, be;
+          if (have_next) { al = al_next; be = be_next; } else load_scale(kb, al, be);
+          have_next = Roles<MODE>::SCALES_AHEAD && kb + NG < p.kb_base;
+          if (have_next) load_scale(kb + NG, al_next, be_next);
           BlockTable tab;
           tab.build(p.level, al, be);
-          if (!mbar_wait(full(s), ph, p.status) || !mbar_wait(empty(s), ph ^ 1u, p.status)) { ok = false; break; }
+          if (!mbar_wait(full(s), ph, p.status, p.wait_limit)) { ok = false; break; }
           const uint8_t* src = gP + s * P_BYTES + d * 32;
           const uint4 q0 = *reinterpret_cast<const uint4*>(src);
           const uint4 q1 = *reinterpret_cast<const uint4*>(src + 16);
           const uint32_t w[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+          if (!mbar_wait(empty(s), ph ^ 1u, p.status, p.wait_limit)) { ok = false; break; }
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             uint32_t o4[4];
@@ -346,52 +392,54 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
           }
         } else if (kb >= kb_gamma0) {
           // offset term of the low-bit product: K-major tile A[m = o][k = group] = gamma_hi (segments 0, 2) or
-          // gamma_lo (segment 1); thread = output row o, reading 128 contiguous bytes of that row
-          if (!mbar_wait(empty(s), ph ^ 1u, p.status) || (rank != 0 && !mbar_wait(full(s), ph, p.status))) { ok = false; break; }
+          // gamma_lo (segment 1); thread = output row o, reading 128 contiguous bytes of that row (the loads are
+          // issued before the wait for the slot, so their latency hides under it)
           const int kg = kb - kb_gamma0, seg = kg / p.ng_blocks, g0 = (kg - seg * p.ng_blocks) * BK;
           const int o = m0 + d;
           const uint4* src = reinterpret_cast<const uint4*>((seg == 1 ? p.gam_l : p.gam_h) + (int64_t)(o < p.d_out ? o : 0) * p.gam_ld + g0);
+          uint4 v[8];
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (o < p.d_out && g0 + j * 8 < p.gam_ld) v = __ldg(src + j);
-            st_shared_v4(dst + (((uint32_t)j ^ xr) << 4), v.x, v.y, v.z, v.w);
+            v[j] = make_uint4(0, 0, 0, 0);
+            if (o < p.d_out && g0 + j * 8 < p.gam_ld) v[j] = __ldg(src + j);
           }
+          if (!mbar_wait(empty(s), ph ^ 1u, p.status, p.wait_limit)) { ok = false; break; }
+#pragma unroll
+          for (int j = 0; j < 8; ++j) st_shared_v4(dst + (((uint32_t)j ^ xr) << 4), v[j].x, v[j].y, v[j].z, v[j].w);
         } else {
-          // adapter K-blocks carry no packed codes, but the other CTA still vouches for its token half
-          if (!mbar_wait(empty(s), ph ^ 1u, p.status) || (rank != 0 && !mbar_wait(full(s), ph, p.status))) { ok = false; break; }
+          // adapter K-blocks carry no packed codes
           const int kk = (kb - p.kb_base) * BK;
           if (MODE == 0) {
             // MN-major tile: A[m = o][k] = B[kk + k][o / lambda_out]; thread = (K-row, 64-wide output group),
-            // reading a contiguous run of row kk + k of B
+            // reading a contiguous run of row kk + k of B.  Loads first, then the wait for the slot, then the stores.
             const int krow = kk + (d & 63);
             const int o0 = m0 + (d >> 6) * 64;
             const unsigned short* src = reinterpret_cast<const unsigned short*>(p.ex) + (int64_t)krow * p.ex_ld;
             const bool live = krow < p.ex_rows;
+            uint4 v[8];
             if ((p.lam & 7) == 0 && p.op == QBLORA_SCALE_AVGPOOL_REPEAT) {   // a 16-byte chunk (8 outputs) repeats a single element of B
 #pragma unroll
               for (int j = 0; j < 8; ++j) {
                 const int o = o0 + j * 8;
-                uint32_t v = (live && o < p.d_out) ? (uint32_t)__ldg(src + o / p.lam) : 0u;
-                v |= v << 16;
-                st_shared_v4(dst + (((uint32_t)j ^ xr) << 4), v, v, v, v);
+                uint32_t e = (live && o < p.d_out) ? (uint32_t)__ldg(src + o / p.lam) : 0u;
+                e |= e << 16;
+                v[j] = make_uint4(e, e, e, e);
               }
             } else if (p.op == QBLORA_SCALE_TRUNCATE_ZEROPAD) {
               // the first Q outputs take B's row as it is (Q is a multiple of 8: whole aligned 16-byte chunks), the rest nothing
 #pragma unroll
               for (int j = 0; j < 8; ++j) {
                 const int o = o0 + j * 8;
-                uint4 v = make_uint4(0, 0, 0, 0);
-                if (live && o < p.n_small) v = __ldg(reinterpret_cast<const uint4*>(src + o));
-                st_shared_v4(dst + (((uint32_t)j ^ xr) << 4), v.x, v.y, v.z, v.w);
+                v[j] = make_uint4(0, 0, 0, 0);
+                if (live && o < p.n_small) v[j] = __ldg(reinterpret_cast<const uint4*>(src + o));
               }
             } else if ((p.lam & 7) == 0) {
               // zero fill with a factor that is a multiple of 8: only the first output of a chunk can be a sampled one
 #pragma unroll
               for (int j = 0; j < 8; ++j) {
                 const int o = o0 + j * 8;
-                const uint32_t v = (live && o < p.d_out && o % p.lam == 0) ? (uint32_t)__ldg(src + o / p.lam) : 0u;
-                st_shared_v4(dst + (((uint32_t)j ^ xr) << 4), v, 0u, 0u, 0u);
+                const uint32_t e = (live && o < p.d_out && o % p.lam == 0) ? (uint32_t)__ldg(src + o / p.lam) : 0u;
+                v[j] = make_uint4(e, 0u, 0u, 0u);
               }
             } else {
 #pragma unroll
@@ -406,23 +454,31 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
                   const uint32_t hi = (live && ob < p.d_out && qb_ >= 0) ? (uint32_t)__ldg(src + qb_) : 0u;
                   o4[e] = lo | (hi << 16);
                 }
-                st_shared_v4(dst + (((uint32_t)j ^ xr) << 4), o4[0], o4[1], o4[2], o4[3]);
+                v[j] = make_uint4(o4[0], o4[1], o4[2], o4[3]);
               }
             }
+            if (!mbar_wait(empty(s), ph ^ 1u, p.status, p.wait_limit)) { ok = false; break; }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) st_shared_v4(dst + (((uint32_t)j ^ xr) << 4), v[j].x, v[j].y, v[j].z, v[j].w);
           } else {
             // K-major tile: A[m = i][k] = A_adapter[i / lambda_in][kk + k]; thread = input column i,
             // reading 128 contiguous bytes of a row of A_adapter (rank is a multiple of 8)
             const int i = m0 + d;
             const int prow = i < p.d_in ? scale_src(p.op, i, p.lam, p.n_small) : -1;   // -1: input not seen by the adapter
             const uint4* src = reinterpret_cast<const uint4*>(p.ex + (int64_t)(prow < 0 ? 0 : prow) * p.ex_ld + kk);
+            uint4 v[8];
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-              uint4 v = make_uint4(0, 0, 0, 0);
-              if (prow >= 0 && kk + j * 8 < p.ex_rows) v = __ldg(src + j);
-              st_shared_v4(dst + (((uint32_t)j ^ xr) << 4), v.x, v.y, v.z, v.w);
+              v[j] = make_uint4(0, 0, 0, 0);
+              if (prow >= 0 && kk + j * 8 < p.ex_rows) v[j] = __ldg(src + j);
             }
+            if (!mbar_wait(empty(s), ph ^ 1u, p.status, p.wait_limit)) { ok = false; break; }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) st_shared_v4(dst + (((uint32_t)j ^ xr) << 4), v[j].x, v[j].y, v[j].z, v[j].w);
           }
         }
+        // the other CTA vouches for its token half of the stage as well as for its weight tile
+        if (rank != 0 && !mbar_wait(full(s), ph, p.status, p.wait_limit)) { ok = false; break; }
         fence_async_proxy();   // generic-proxy stores -> visible to the tensor core's async proxy
         if (rank == 0) {
           mbar_arrive(aready(s));
@@ -444,7 +500,7 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
       const uint32_t aph = (lt >> 1) & 1u;
       const int m = (tile % p.m_tiles) * (2 * BM) + (int)rank * BM + q * 32 + lane;
       const int t0 = (tile / p.m_tiles) * BN;
-      if (!mbar_wait(accfull(a), aph, p.status)) { ok = false; break; }
+      if (!mbar_wait(accfull(a), aph, p.status, p.wait_limit)) { ok = false; break; }
       tc_fence_after();
       for (int c = 0; c < BN / 32; ++c) {
         if (t0 + c * 32 >= p.T) break;
@@ -708,13 +764,18 @@ struct LowbitTerm {
 int launch_main(int mode, const QwView& qw, const AdView* ad, const __nv_bfloat16* Bop, const __nv_bfloat16* Bx,
                 int ldx, int64_t T, void* out, int out_dtype, int* status, cudaStream_t st,
                 const LowbitTerm* lb = nullptr) {
-  static bool attr_set[2] = {false, false};
-  if (!attr_set[mode]) {
+  // the shared-memory opt-in is a per-device function attribute: set once per device and kernel (the flags are
+  // atomic, so concurrent host threads at worst set it twice)
+  static std::atomic<bool> attr_set[64][2];
+  int dev = 0;
+  QB_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return QBLORA_ERR_UNSUPPORTED;
+  if (!attr_set[dev][mode].load(std::memory_order_acquire)) {
     cudaError_t e = mode == 0
         ? cudaFuncSetAttribute(tc_dq_gemm_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES)
         : cudaFuncSetAttribute(tc_dq_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return QBLORA_ERR_CUDA;
-    attr_set[mode] = true;
+    attr_set[dev][mode].store(true, std::memory_order_release);
   }
   TcParams p{};
   p.M = mode == 0 ? qw.d_out : qw.d_in;
@@ -736,6 +797,8 @@ int launch_main(int mode, const QwView& qw, const AdView* ad, const __nv_bfloat1
   p.op = ad ? ad->op : 0;
   p.n_small = ad ? (mode == 0 ? ad->Q : ad->P) : 0;
   p.out = out; p.out_dtype = out_dtype; p.status = status;
+  p.wait_limit = wait_limit_cycles();
+  p.drop_load = take_dropped_load();
   if (lb) {
     p.beta = lb->beta_c;
     p.ng_blocks = (qw.G + BK - 1) / BK;
@@ -769,7 +832,7 @@ int launch_main(int mode, const QwView& qw, const AdView* ad, const __nv_bfloat1
   // while that product finishes (the producer warp waits for it before the first adapter K-block).  Without an
   // adapter the predecessor is the caller's own work and the launch is an ordinary one.
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(NUM_THREADS); cfg.dynamicSmemBytes = SMEM_BYTES; cfg.stream = st;
+  cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(mode == 0 ? Roles<0>::NUM_THREADS : Roles<1>::NUM_THREADS); cfg.dynamicSmemBytes = SMEM_BYTES; cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -922,18 +985,21 @@ int tc_linear_bwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, co
                   void* dX, int dx_dtype, float* dA, float* dB, char* ws, cudaStream_t st) {
   TcWs w = carve(QBLORA_OP_LINEAR_BWD, ad, T, ws);
   int* status = reinterpret_cast<int*>(ws);
-  int rc;
-  if (ad) {
-    // Two chains: (a) dv -> du, which the dX contraction needs; (b) pooled x -> u -> dB, dA, which
-    // nothing else needs.  With a side lane (b) runs on it: it starts together with (a), waits for du
-    // before the gradient products, and is joined at the end; the caller's stream goes straight from
-    // (a) to the dX contraction.
-    SideLane* lane = (dX && (dA || dB)) ? side_lane() : nullptr;
-    cudaStream_t sb = lane ? lane->stream : st;
-    if (lane) {
-      QB_CUDA(cudaEventRecord(lane->fork, st));
-      QB_CUDA(cudaStreamWaitEvent(lane->stream, lane->fork, 0));
-    }
+  if (!ad) return dX ? launch_main(1, qw, ad, dY, w.du16, w.ldr, T, dX, dx_dtype, status, st) : QBLORA_OK;
+  // Two chains: (a) dv -> du, which the dX contraction needs; (b) pooled x -> u -> dB, dA, which
+  // nothing else needs.  With a side lane (b) runs on it: it starts together with (a), waits for du
+  // before the gradient products, and is joined at the end; the caller's stream goes straight from
+  // (a) to the dX contraction.
+  SideLane* lane = (dX && (dA || dB)) ? side_lane() : nullptr;
+  cudaStream_t sb = lane ? lane->stream : st;
+  if (lane) {
+    QB_CUDA(cudaEventRecord(lane->fork, st));
+    QB_CUDA(cudaStreamWaitEvent(lane->stream, lane->fork, 0));
+  }
+  // From here on the side lane may hold work of this call (and, inside a stream capture, is part of the capture):
+  // whatever happens below, it is joined back into the caller's stream before the call returns.
+  const int rc = [&]() -> int {
+    int rc;
     const int64_t n = T * ad->Q;
     if (ad->op != QBLORA_SCALE_AVGPOOL_REPEAT) {
       sample_split_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(
@@ -985,15 +1051,14 @@ int tc_linear_bwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, co
       rc = small_gemm(ad->P, ad->r, segs, 3, out, status, sb, w.partial);
       if (rc) return rc;
     }
-    if (lane) {
-      QB_CUDA(cudaEventRecord(lane->join, lane->stream));
-      rc = dX ? launch_main(1, qw, ad, dY, w.du16, w.ldr, T, dX, dx_dtype, status, st) : QBLORA_OK;
-      QB_CUDA(cudaStreamWaitEvent(st, lane->join, 0));   // the call's work is complete when st is
-      return rc;
-    }
+    return dX ? launch_main(1, qw, ad, dY, w.du16, w.ldr, T, dX, dx_dtype, status, st) : QBLORA_OK;
+  }();
+  if (lane) {   // the call's work is complete when st is; on an error path this also closes a capture's fork
+    const bool joined = cudaEventRecord(lane->join, lane->stream) == cudaSuccess &&
+                        cudaStreamWaitEvent(st, lane->join, 0) == cudaSuccess;
+    if (!joined && rc == QBLORA_OK) return QBLORA_ERR_CUDA;
   }
-  if (!dX) return QBLORA_OK;
-  return launch_main(1, qw, ad, dY, w.du16, w.ldr, T, dX, dx_dtype, status, st);
+  return rc;
 }
 
 }  // namespace qb

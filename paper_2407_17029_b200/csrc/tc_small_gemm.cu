@@ -2,6 +2,8 @@
 // CTA (bn <= 256), cta_group::1, four TMA-fed stages; warp 0 TMA producer, warp 1 MMA issuer and
 // TMEM owner, warps 2-5 epilogue.  Operands may be K-contiguous (K-major) or MN-contiguous
 // (MN-major); both are staged in the canonical 128-byte-swizzled layout by TMA.
+#include <atomic>
+
 #include "tc_ptx.cuh"
 #include "tc_small.cuh"
 
@@ -32,6 +34,7 @@ struct SgParams {
   int a_kmajor, b_kmajor;
   SgOut out;
   int* status;
+  long long wait_limit;     // cycles after which a device-side wait gives up
 };
 
 __global__ void __launch_bounds__(SG_THREADS, 1)
@@ -79,7 +82,7 @@ small_gemm_kernel(const __grid_constant__ SgMaps maps, const __grid_constant__ S
         for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % SG_STAGES;
           const uint32_t ph = (it / SG_STAGES) & 1u;
-          if (!mbar_wait(empty(s), ph ^ 1u, p.status)) { ok = false; break; }
+          if (!mbar_wait(empty(s), ph ^ 1u, p.status, p.wait_limit)) { ok = false; break; }
           mbar_arrive_expect_tx(full(s), stage_bytes);
           const uint32_t a_dst = sA + s * SG_A_BYTES, b_dst = sB + s * SG_B_BYTES;
           if (p.a_kmajor) {
@@ -98,7 +101,7 @@ small_gemm_kernel(const __grid_constant__ SgMaps maps, const __grid_constant__ S
       }
       if (!ok) {
         const uint32_t lo = it > (uint32_t)SG_STAGES ? it - SG_STAGES : 0;
-        for (uint32_t j = lo; j < it; ++j) mbar_wait(full(j % SG_STAGES), (j / SG_STAGES) & 1u, p.status);
+        for (uint32_t j = lo; j < it; ++j) mbar_wait(full(j % SG_STAGES), (j / SG_STAGES) & 1u, p.status, p.wait_limit);
       }
     }
   } else if (warp == 1) {
@@ -116,7 +119,7 @@ small_gemm_kernel(const __grid_constant__ SgMaps maps, const __grid_constant__ S
         for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % SG_STAGES;
           const uint32_t ph = (it / SG_STAGES) & 1u;
-          if (!mbar_wait(full(s), ph, p.status)) { ok = false; break; }
+          if (!mbar_wait(full(s), ph, p.status, p.wait_limit)) { ok = false; break; }
           tc_fence_after();
 #pragma unroll
           for (int k = 0; k < SG_BK / 16; ++k) {
@@ -141,7 +144,7 @@ small_gemm_kernel(const __grid_constant__ SgMaps maps, const __grid_constant__ S
       const int kb0 = (int)blockIdx.z * per, kb1 = min(kb0 + per, p.kblocks[g]);
       my_kblocks += max(kb1 - kb0, 0);
     }
-    if (mbar_wait(accfull, 0, p.status)) {
+    if (mbar_wait(accfull, 0, p.status, p.wait_limit)) {
       tc_fence_after();
       for (int c = 0; c < p.bn / 32; ++c) {
         const int nb = n0 + c * 32;
@@ -286,10 +289,13 @@ int small_gemm_splits(int M, int N, int K) {
 int small_gemm(int M, int N, const SgSegment* segs, int nseg, const SgOut& out, int* status, cudaStream_t st,
                float* partial, bool dependent, bool wide_tiles) {
   if (nseg < 1 || nseg > SG_MAX_SEG || M < 1 || N < 1) return QBLORA_ERR_INVALID_ARG;
-  static bool attr_set = false;
-  if (!attr_set) {
+  static std::atomic<bool> attr_set[64];   // per device; atomic: concurrent host threads at worst set it twice
+  int dev = 0;
+  QB_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return QBLORA_ERR_UNSUPPORTED;
+  if (!attr_set[dev].load(std::memory_order_acquire)) {
     QB_CUDA(cudaFuncSetAttribute(small_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SG_SMEM));
-    attr_set = true;
+    attr_set[dev].store(true, std::memory_order_release);
   }
   SgMaps maps;
   SgParams p{};
@@ -313,6 +319,7 @@ int small_gemm(int M, int N, const SgSegment* segs, int nseg, const SgOut& out, 
   for (int g = nseg; g < SG_MAX_SEG; ++g) { maps.a[g] = maps.a[0]; maps.b[g] = maps.b[0]; p.kblocks[g] = 0; }
   p.out = out;
   p.status = status;
+  p.wait_limit = wait_limit_cycles();
   p.splits = 1;
   p.split_stride = 0;
   if (partial) {   // split the contraction; only the fp32 output is supported in this mode

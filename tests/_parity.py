@@ -88,3 +88,80 @@ def sample_rows(seed: int, T: int, n: int) -> np.ndarray:
         return np.arange(T)
     g = np.random.Generator(np.random.Philox(key=seed + 977))
     return np.sort(g.choice(T, size=n, replace=False))
+
+
+# ------------------------------------------------------------------------------------------------ guard bands
+# Every output and workspace buffer of a guarded call sits between two 4 KiB bands of a known byte pattern that
+# are checked after the call: a store past either end of Y, dX, dA, dB, beta', the codes, the scales or the
+# workspace fails the test even when all values inside the buffer are right.
+GUARD_BYTES = 4096
+GUARD_PATTERN = 0xA5
+
+
+class Guarded:
+    def __init__(self):
+        self.bufs = []
+
+    def alloc(self, shape, dtype):
+        shape = tuple(int(x) for x in shape)
+        n = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+        raw = torch.full((n + 2 * GUARD_BYTES,), GUARD_PATTERN, dtype=torch.uint8, device=DEV)
+        self.bufs.append((raw, n))
+        return raw[GUARD_BYTES:GUARD_BYTES + n].view(dtype).view(shape)
+
+    def workspace(self, op, qw, ad, tokens):
+        return self.alloc((max(qb.workspace_bytes(op, qw, ad, tokens), 256),), torch.uint8)
+
+    def check(self, what=""):
+        torch.cuda.synchronize()
+        for raw, n in self.bufs:
+            lo, hi = raw[:GUARD_BYTES], raw[GUARD_BYTES + n:]
+            assert bool((lo == GUARD_PATTERN).all()), f"{what}: bytes in front of a {n}-byte buffer were overwritten"
+            assert bool((hi == GUARD_PATTERN).all()), f"{what}: bytes behind a {n}-byte buffer were overwritten"
+
+
+def g_linear_fwd(dq, da, Xd, dtype):
+    g = Guarded()
+    Y = g.alloc((Xd.shape[0], dq.d_out), dtype)
+    ws = g.workspace(qb.OP_LINEAR_FWD, dq, da, Xd.shape[0])
+    qb.linear_fwd(dq, da, Xd, ws=ws, out=Y)
+    g.check("linear_fwd")
+    assert qb.device_status(ws) == qb.OK
+    return Y
+
+
+def g_linear_bwd(dq, da, Xd, dYd, dtype, need_dx=True, need_da=True, need_db=True):
+    g = Guarded()
+    T = dYd.shape[0]
+    dX = g.alloc((T, dq.d_in), dtype) if need_dx else None
+    dA = g.alloc(tuple(da.A.shape), torch.float32) if (da is not None and need_da) else None
+    dB = g.alloc(tuple(da.B.shape), torch.float32) if (da is not None and da.B is not None and need_db) else None
+    ws = g.workspace(qb.OP_LINEAR_BWD, dq, da, T)
+    qb.linear_bwd(dq, da, Xd, dYd, ws=ws, outs=(dX, dA, dB))
+    g.check("linear_bwd")
+    assert qb.device_status(ws) == qb.OK
+    return dX, dA, dB
+
+
+def g_lowbit_gemm(dq, Xd, dtype):
+    g = Guarded()
+    Y = g.alloc((Xd.shape[0], dq.d_out), dtype)
+    ws = g.workspace(qb.OP_LOWBIT_GEMM, dq, None, Xd.shape[0])
+    qb.lowbit_gemm(dq, Xd, ws=ws, out=Y)
+    g.check("lowbit_gemm")
+    assert qb.device_status(ws) == qb.OK
+    return Y
+
+
+def g_quantize(Wd, bi, bo, qfmt, code=None):
+    g = Guarded()
+    d_out, d_in = Wd.shape
+    codes = g.alloc((d_out, d_in // 2), torch.uint8)
+    alpha = g.alloc((d_out // bo, d_in // bi), torch.float32)
+    beta = g.alloc((d_out // bo, d_in // bi), torch.float32) if qfmt == qb.FMT_AFFINE_MINMAX else None
+    if qfmt == qb.FMT_CODEBOOK_ABSMAX and code is None:
+        code = qb.default_code_table()
+    out = qb.QWeight(d_out, d_in, bi, bo, qfmt, list(code) if code is not None else [0.0] * 16, codes, alpha, beta)
+    got = qb.quantize_blockwise(Wd, bi, bo, qfmt, code, out=out)
+    g.check("quantize_blockwise")
+    return got

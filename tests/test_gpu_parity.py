@@ -6,8 +6,8 @@ import torch
 
 import oracle
 from paper_2407_17029_b200 import synth
-from tests._parity import (DEV, adapter_to_dev, gate_bf16, gate_strict, qweight_to_dev, rms, to_bf16_dev,
-                           to_dev, to_np64, visible_scaling)
+from tests._parity import (DEV, Guarded, adapter_to_dev, g_linear_bwd, g_linear_fwd, g_lowbit_gemm, g_quantize, gate_bf16,
+                           gate_strict, qweight_to_dev, rms, to_bf16_dev, to_dev, to_np64, visible_scaling)
 
 pytestmark = pytest.mark.gpu
 
@@ -42,7 +42,7 @@ def test_quantize_bit_exact(qb, qfmt, shape, bi, bo, dtype):
     else:
         Wd = to_dev(W)
     ref = oracle.quantize_blockwise(W, bi, bo, qfmt)
-    got = qb.quantize_blockwise(Wd, bi, bo, qfmt)
+    got = g_quantize(Wd, bi, bo, qfmt)              # outputs between guard bands
     assert np.array_equal(got.codes.cpu().numpy(), ref.codes)
     assert np.array_equal(got.alpha.cpu().numpy().view(np.uint32), ref.alpha.view(np.uint32))
     if qfmt == 1:
@@ -139,8 +139,8 @@ def test_linear_fwd_parity(qb, path, case, qfmt, visible):
         ad.scaling = visible_scaling(Wt, ad, X)
     ref = oracle.linear_fwd(Wt, ad, X)
     dq, da, Xd = qweight_to_dev(qw), adapter_to_dev(ad), to_bf16_dev(X)
-    gate_strict(to_np64(qb.linear_fwd(dq, da, Xd, torch.float32)), ref, "Y f32")
-    gate_bf16(to_np64(qb.linear_fwd(dq, da, Xd, torch.bfloat16)), ref, "Y bf16")
+    gate_strict(to_np64(g_linear_fwd(dq, da, Xd, torch.float32)), ref, "Y f32")         # guarded: outputs and workspace
+    gate_bf16(to_np64(g_linear_fwd(dq, da, Xd, torch.bfloat16)), ref, "Y bf16")          # sit between guard bands
     if visible:
         base = oracle.linear_fwd(Wt, None, X)
         assert rms(ref - base) > 0.5 * rms(base)          # the adapter really is half of the output
@@ -157,11 +157,11 @@ def test_linear_bwd_parity(qb, path, case, qfmt, visible):
         ad.scaling = visible_scaling(Wt, ad, X)
     rdX, rdA, rdB = oracle.linear_bwd(Wt, ad, X, dY)
     dq, da, Xd, dYd = qweight_to_dev(qw), adapter_to_dev(ad), to_bf16_dev(X), to_bf16_dev(dY)
-    dX, dA, dB = qb.linear_bwd(dq, da, Xd, dYd, torch.float32)
+    dX, dA, dB = g_linear_bwd(dq, da, Xd, dYd, torch.float32)
     gate_strict(to_np64(dX), rdX, "dX f32")
     gate_strict(to_np64(dA), rdA, "dA", per_row=False)
     gate_strict(to_np64(dB), rdB, "dB", per_row=False)
-    dXb, _, _ = qb.linear_bwd(dq, da, Xd, dYd, torch.bfloat16, need_da=False, need_db=False)
+    dXb, _, _ = g_linear_bwd(dq, da, Xd, dYd, torch.bfloat16, need_da=False, need_db=False)
     gate_bf16(to_np64(dXb), rdX, "dX bf16")
     # skipping outputs leaves the others unchanged (bit for bit: the library is deterministic)
     _, dA2, dB2 = qb.linear_bwd(dq, da, Xd, dYd, need_dx=False)
@@ -221,7 +221,9 @@ def test_merge_bit_exact_and_identity(qb, path, single, scaling):
     ref = oracle.merge(qw, ad)
     dq, da = qweight_to_dev(qw), adapter_to_dev(ad)
     codes0, alpha0 = dq.codes.clone(), dq.alpha.clone()
-    got = qb.merge(dq, da)
+    g = Guarded()
+    got = qb.merge(dq, da, ws=g.workspace(qb.OP_MERGE, dq, da, 0), beta_out=g.alloc(tuple(dq.beta.shape), torch.float32))
+    g.check("merge")
     assert np.array_equal(got.beta.cpu().numpy().view(np.uint32), ref.beta.view(np.uint32))
     assert torch.equal(dq.codes, codes0) and torch.equal(dq.alpha, alpha0)          # untouched
     assert got.codes.data_ptr() == dq.codes.data_ptr()
@@ -251,8 +253,8 @@ def test_lowbit_gemm_parity(qb, path, T):
     qw, _, X, _ = make_case(53, T, 328, 448, 64, 8, 16, qfmt=1)
     ref = oracle.lowbit_gemm(qw, X)
     dq, Xd = qweight_to_dev(qw), to_bf16_dev(X)
-    gate_strict(to_np64(qb.lowbit_gemm(dq, Xd, torch.float32)), ref, f"lowbit T={T} f32")
-    gate_bf16(to_np64(qb.lowbit_gemm(dq, Xd, torch.bfloat16)), ref, f"lowbit T={T} bf16")
+    gate_strict(to_np64(g_lowbit_gemm(dq, Xd, torch.float32)), ref, f"lowbit T={T} f32")
+    gate_bf16(to_np64(g_lowbit_gemm(dq, Xd, torch.bfloat16)), ref, f"lowbit T={T} bf16")
 
 
 @pytest.mark.parametrize("T", [1, 3, 16])
@@ -278,7 +280,7 @@ def test_lowbit_decode_wide_input(qb, T):
     qw, _, X, _ = make_case(58, T, 72, 896 * 64, 64, 8, 16, qfmt=1)
     ref = oracle.lowbit_gemm(qw, X)
     dq, Xd = qweight_to_dev(qw), to_bf16_dev(X)
-    gate_strict(to_np64(qb.lowbit_gemm(dq, Xd, torch.float32)), ref, f"lowbit wide T={T}")
+    gate_strict(to_np64(g_lowbit_gemm(dq, Xd, torch.float32)), ref, f"lowbit wide T={T}")
 
 
 @pytest.mark.parametrize("case", [(300, 320, 448, 64, 8), (150, 128, 512, 8, 8), (77, 136, 192, 4, 4)])
@@ -294,11 +296,11 @@ def test_single_matrix_adapter_fwd_bwd(qb, path, case, visible):
     if visible:
         ad.scaling = visible_scaling(Wt, ad, X)
     dq, da, Xd, dYd = qweight_to_dev(qw), adapter_to_dev(ad), to_bf16_dev(X), to_bf16_dev(dY)
-    gate_strict(to_np64(qb.linear_fwd(dq, da, Xd, torch.float32)), oracle.linear_fwd(Wt, ad, X), "Y single matrix")
+    gate_strict(to_np64(g_linear_fwd(dq, da, Xd, torch.float32)), oracle.linear_fwd(Wt, ad, X), "Y single matrix")
     gate_bf16(to_np64(qb.linear_fwd(dq, da, Xd, torch.bfloat16)), oracle.linear_fwd(Wt, ad, X), "Y single matrix bf16")
     rdX, rdH, rdB = oracle.linear_bwd(Wt, ad, X, dY)
     assert rdB is None
-    dX, dH, dB = qb.linear_bwd(dq, da, Xd, dYd, torch.float32)
+    dX, dH, dB = g_linear_bwd(dq, da, Xd, dYd, torch.float32)
     assert dB is None and tuple(dH.shape) == H.shape
     gate_strict(to_np64(dX), rdX, "dX single matrix")
     gate_strict(to_np64(dH), rdH, "dH", per_row=False)
@@ -325,7 +327,7 @@ def test_lowbit_decode_tiny_shapes(qb, T, d_out, d_in):
     qw, _, X, _ = make_case(62, T, d_out, d_in, 64, 8, 8, qfmt=1)
     ref = oracle.lowbit_gemm(qw, X)
     dq, Xd = qweight_to_dev(qw), to_bf16_dev(X)
-    gate_strict(to_np64(qb.lowbit_gemm(dq, Xd, torch.float32)), ref, f"lowbit tiny {d_out}x{d_in} T={T}")
+    gate_strict(to_np64(g_lowbit_gemm(dq, Xd, torch.float32)), ref, f"lowbit tiny {d_out}x{d_in} T={T}")
 
 
 @pytest.mark.parametrize("bi,bo", [(8, 8), (4, 8), (8, 1), (4, 2)])
@@ -339,9 +341,9 @@ def test_two_dimensional_blocks_fwd_bwd(qb, path, bi, bo, visible):
     if visible:
         ad.scaling = visible_scaling(Wt, ad, X)
     dq, da, Xd, dYd = qweight_to_dev(qw), adapter_to_dev(ad), to_bf16_dev(X), to_bf16_dev(dY)
-    gate_strict(to_np64(qb.linear_fwd(dq, da, Xd, torch.float32)), oracle.linear_fwd(Wt, ad, X), f"Y blocks {bi}x{bo}")
+    gate_strict(to_np64(g_linear_fwd(dq, da, Xd, torch.float32)), oracle.linear_fwd(Wt, ad, X), f"Y blocks {bi}x{bo}")
     rdX, rdA, rdB = oracle.linear_bwd(Wt, ad, X, dY)
-    dX, dA, dB = qb.linear_bwd(dq, da, Xd, dYd, torch.float32)
+    dX, dA, dB = g_linear_bwd(dq, da, Xd, dYd, torch.float32)
     gate_strict(to_np64(dX), rdX, f"dX blocks {bi}x{bo}")
     gate_strict(to_np64(dA), rdA, "dA", per_row=False)
     gate_strict(to_np64(dB), rdB, "dB", per_row=False)
@@ -363,7 +365,11 @@ def test_dense_16bit_merge(qb, case):
     ad.scaling = visible_scaling(Wt, ad, X)
     ref = Wt + ad.scaling * oracle.dense_delta_w(d_out, d_in, ad)
     dq, da = qweight_to_dev(qw), adapter_to_dev(ad)
-    got = to_np64(qb.merge_dense(dq, da))
+    g = Guarded()
+    Wg = g.alloc((d_out, d_in), torch.bfloat16)
+    qb.merge_dense(dq, da, out=Wg, ws=g.workspace(qb.OP_MERGE_DENSE, dq, da, 0))
+    g.check("merge_dense")
+    got = to_np64(Wg)
     assert np.all(np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref) + 1e-30)          # one bf16 rounding
     base = to_np64(qb.merge_dense(dq, None))
     assert np.all(np.abs(base - Wt) <= 2.0 ** -8 * np.abs(Wt) + 1e-30)
