@@ -444,6 +444,8 @@ def run_gpu(args, wl, geom):
     if ctx.rank == 0 and not args.no_extras:
         line["lowbit"] = lowbit_extras(qb, torch, ctx.dev, ctx.peaks, ctx.l2_bytes, args.lowbit_shapes.split(","),
                                        [int(t) for t in args.lowbit_tokens.split(",")])
+        torch.cuda.empty_cache()
+        line["dense_16bit"] = dense_extras(qb, torch, ctx.dev, ctx.peaks)
     if ctx.rank == 0 and not args.no_cpu_baseline and ctx.world == 1:
         rows = ref_rows_for(wl, geom, args.ref_rows)
         cache = oracle_cache(wl, geom, rows)
@@ -566,6 +568,49 @@ def lowbit_extras(qb, torch, dev, peaks, l2_bytes, shapes=("q", "up"), tokens=(1
                                         "status": qb.device_status(ws)}
     out["peak_hbm_gbs"] = peaks["hbm_gbs"]
     out["peak_kind"] = peaks["source"]
+    return out
+
+
+def dense_extras(qb, torch, dev, peaks):
+    """The other deployment (Sec. 3.1 / 3.2): merge the adapter into a dense bf16 weight, then serve it with the
+    library's plain bf16 tensor-core GEMM.  TFLOP/s against the burst bf16 peak (ten launches, a few ms)."""
+    out = {}
+
+    def bf(a):
+        return torch.from_numpy(synth.bf16_bits(a).view(np.int16).copy()).to(dev).view(torch.bfloat16)
+
+    for wname, lname in (("C2", "attn_proj"), ("C4", "gate")):
+        wl = synth.WORKLOADS[wname]
+        spec = [sp for sp in wl.linears if sp.name == lname][0]
+        T = wl.tokens
+        li = synth.make_linear_inputs(wl, spec, synth.GEOM_A, seed=0, tokens=T)
+        dq = qb.quantize_blockwise(torch.from_numpy(li.W).to(dev), 64, 1, wl.qfmt)
+        li.W = None
+        ad = qb.Adapter(64, 8, wl.rank, wl.scaling, bf(li.A), bf(li.B))
+        Wm = torch.empty((spec.d_out, spec.d_in), dtype=torch.bfloat16, device=dev)
+        wsm = qb.alloc_workspace(qb.OP_MERGE_DENSE, dq, ad, 0)
+        s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        qb.merge_dense(dq, ad, out=Wm, ws=wsm)
+        s.record()
+        for _ in range(5):
+            qb.merge_dense(dq, ad, out=Wm, ws=wsm)
+        e.record(); torch.cuda.synchronize()
+        merge_us = s.elapsed_time(e) / 5 * 1e3
+        X = bf(li.X)
+        Y = torch.empty((T, spec.d_out), dtype=torch.bfloat16, device=dev)
+        ws = torch.empty(256, dtype=torch.uint8, device=dev)
+        for _ in range(3):
+            qb.dense_gemm(Wm, X, ws=ws, out=Y)
+        s.record()
+        for _ in range(10):
+            qb.dense_gemm(Wm, X, ws=ws, out=Y)
+        e.record(); torch.cuda.synchronize()
+        us = s.elapsed_time(e) / 10 * 1e3
+        tf = 2.0 * T * spec.d_in * spec.d_out / us / 1e6
+        out[f"{wname}/{lname}[{spec.d_out},{spec.d_in}] T={T}"] = {
+            "merge_dense_us": merge_us, "dense_gemm_us": us, "TFLOP/s": tf, "frac_bf16_burst": tf / peaks["bf16_tflops"],
+            "peak_kind": "burst (ten launches, a few ms)", "status": qb.device_status(ws)}
+        del Wm, X, Y, dq
     return out
 
 

@@ -250,11 +250,21 @@ int qablora_merge(const qblora_qweight* qw, const qblora_adapter* adapter, float
  *   W_out[o][i] = alpha * level[code] + beta  +  s * dW[o][i]   (A B in fp64, the sum in fp32, then bf16).
  *   W_out DEVICE out bf16 [d_out][d_in] (16-byte aligned, d_in % 8 == 0).  Either format, any block
  *   shape, any (lambda_in, lambda_out).  adapter may be NULL (plain dequantization) and may be the
- *   single matrix H (B == NULL).  The merged weight is then served by any plain bf16 GEMM.
+ *   single matrix H (B == NULL).  The merged weight is then served by qblora_dense_gemm (or any plain bf16 GEMM).
  *   ws: qblora_workspace_bytes(QBLORA_OP_MERGE_DENSE, ...) bytes.
  */
 int qblora_merge_dense(const qblora_qweight* qw, const qblora_adapter* adapter, void* W_out, void* ws,
                        size_t ws_bytes, void* stream);
+
+/*
+ * Serving product for the 16-bit deployment (Sec. 3.1: the fine-tuned adapter is merged into the weight, W' = W + s A B,
+ * "for inference"; Sec. 3.2, "Merging Q-BLoRA": the merged model has no inference overhead):
+ *   Y[t][o] = sum_i X[t][i] * W[o][i],  W DEVICE bf16 [d_out][d_in] as written by qblora_merge_dense.
+ * A plain bf16 tensor-core GEMM with fp32 accumulation.  X DEVICE bf16 [tokens][d_in]; Y DEVICE out [tokens][d_out],
+ * BF16 or F32.  Requires d_in % 8 == 0.  ws: at least 256 bytes (status word only).
+ */
+int qblora_dense_gemm(const void* W, int32_t d_out, int32_t d_in, const void* X, int64_t tokens, void* Y,
+                      int y_dtype, void* ws, size_t ws_bytes, void* stream);
 
 /*
  * The same merge for callers that cannot give the library a workspace.  (The paper has no

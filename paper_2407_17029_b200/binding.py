@@ -31,7 +31,7 @@ EXPORTS = ["qblora_default_code_table", "qblora_workspace_bytes", "qblora_status
            "qblora_device_status", "qblora_quantize_blockwise", "qblora_linear_fwd",
            "qblora_linear_bwd", "qablora_merge", "qablora_lowbit_gemm", "qblora_kernel_launches",
            "qblora_set_timing_events", "qablora_merge_noalloc", "qblora_merge_dense",
-           "qblora_quantize_minmax_nbit", "qblora_debug_set_wait_limit", "qblora_debug_drop_load"]
+           "qblora_quantize_minmax_nbit", "qblora_debug_set_wait_limit", "qblora_debug_drop_load", "qblora_dense_gemm"]
 
 
 class _CQWeight(ctypes.Structure):
@@ -82,6 +82,8 @@ _lib.qblora_merge_dense.restype = ctypes.c_int
 _lib.qblora_kernel_launches.restype = ctypes.c_uint64
 _lib.qblora_kernel_launches.argtypes = []
 _lib.qblora_set_timing_events.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
+_lib.qblora_dense_gemm.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p,
+                                   ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
 _lib.qblora_debug_set_wait_limit.argtypes = [ctypes.c_int64]
 _lib.qblora_debug_drop_load.argtypes = [ctypes.c_int32]
 
@@ -351,4 +353,20 @@ def lowbit_gemm(qw: QWeight, X: torch.Tensor, out_dtype=torch.bfloat16, ws: Opti
     st = _lib.qablora_lowbit_gemm(ctypes.byref(cq), X.data_ptr(), T, Y.data_ptr(), _dt(Y.dtype),
                                   ws.data_ptr(), ws.numel(), _stream_ptr(stream))
     _check(st, "qablora_lowbit_gemm")
+    return Y
+
+
+def dense_gemm(W: torch.Tensor, X: torch.Tensor, out_dtype=torch.bfloat16, ws: Optional[torch.Tensor] = None,
+               out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """qblora_dense_gemm: Y = X W^T for a dense bf16 weight [d_out][d_in] (the merged 16-bit deployment)."""
+    assert W.is_cuda and W.is_contiguous() and W.dtype == torch.bfloat16 and W.dim() == 2
+    assert X.is_cuda and X.is_contiguous() and X.dtype == torch.bfloat16 and X.shape[1] == W.shape[1]
+    T = X.shape[0]
+    d_out, d_in = W.shape
+    Y = out if out is not None else torch.empty((T, d_out), dtype=out_dtype, device=X.device)
+    if ws is None:
+        ws = torch.empty(256, dtype=torch.uint8, device=X.device)
+    st = _lib.qblora_dense_gemm(W.data_ptr(), d_out, d_in, X.data_ptr(), T, Y.data_ptr(), _dt(Y.dtype), ws.data_ptr(),
+                                ws.numel(), _stream_ptr(stream))
+    _check(st, "qblora_dense_gemm")
     return Y

@@ -306,6 +306,18 @@ int qblora_merge_dense(const qblora_qweight* qw, const qblora_adapter* adapter, 
                             static_cast<char*>(ws), st);
 }
 
+int qblora_dense_gemm(const void* W, int32_t d_out, int32_t d_in, const void* X, int64_t tokens, void* Y, int y_dtype,
+                      void* ws, size_t ws_bytes, void* stream) {
+  if (!W || !X || !Y || !aligned16(W) || !aligned16(X) || !aligned16(Y)) return QBLORA_ERR_INVALID_ARG;
+  if (d_out < 1 || d_in < 8 || d_in % 8 || tokens < 1 || tokens >= ((int64_t)1 << 31) || !dtype_ok(y_dtype)) return QBLORA_ERR_INVALID_ARG;
+  if (!ws || !aligned16(ws) || ws_bytes < dense_gemm_ws_bytes()) return QBLORA_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int rc = reset_status(ws, st);
+  if (rc) return rc;
+  return launch_dense_gemm(static_cast<const __nv_bfloat16*>(W), d_out, d_in, static_cast<const __nv_bfloat16*>(X), tokens, Y,
+                           y_dtype, static_cast<int*>(ws), st);
+}
+
 int qablora_merge_noalloc(const qblora_qweight* qw, const qblora_adapter* adapter, float* beta_out,
                           void* stream) {
   QwView q; int rc = make_qw(qw, &q);

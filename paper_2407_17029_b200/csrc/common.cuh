@@ -90,6 +90,11 @@ size_t gemv_ws_bytes(const QwView& qw, int64_t T);   // status word + (T > 1) to
 int launch_lowbit_gemv(const QwView& qw, const __nv_bfloat16* X, int64_t T, void* Y, int y_dtype,
                        int* status, cudaStream_t st);
 
+// Plain bf16 tcgen05 GEMM serving a dense merged weight: Y = X W^T, W bf16 [d_out][d_in] (d_in % 8 == 0).
+size_t dense_gemm_ws_bytes();
+int launch_dense_gemm(const __nv_bfloat16* W, int d_out, int d_in, const __nv_bfloat16* X, int64_t T, void* Y,
+                      int y_dtype, int* status, cudaStream_t st);
+
 // Tensor-core path (tcgen05 / TMEM / TMA): block_in == 64, block_out == 1.
 bool tc_supported(const QwView& qw, const AdView* ad, int64_t T);
 size_t tc_ws_bytes(int op, const QwView& qw, const AdView* ad, int64_t T);

@@ -373,7 +373,11 @@ def test_dense_16bit_merge(qb, case):
     assert np.all(np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref) + 1e-30)          # one bf16 rounding
     base = to_np64(qb.merge_dense(dq, None))
     assert np.all(np.abs(base - Wt) <= 2.0 ** -8 * np.abs(Wt) + 1e-30)
-    Y = torch.matmul(to_bf16_dev(X).float(), qb.merge_dense(dq, da).float().t())
+    # served by the library's own bf16 GEMM, outputs and workspace between guard bands
+    g = Guarded()
+    Y = g.alloc((X.shape[0], d_out), torch.float32)
+    qb.dense_gemm(Wg, to_bf16_dev(X), ws=g.alloc((256,), torch.uint8), out=Y)
+    g.check("dense_gemm")
     gate_strict(to_np64(Y), oracle.linear_fwd(Wt, ad, X), "X W'^T vs adapted forward")
 
 
@@ -517,3 +521,22 @@ def test_lowbit_one_token_split_tail_graph_replay(qb, d_out):
             st.synchronize()
             assert torch.equal(Y, eager[k]), f"replay {it}"
     assert qb.device_status(ws) == qb.OK
+
+
+@pytest.mark.parametrize("T,d_out,d_in", [(300, 320, 448), (515, 264, 72), (1, 8, 64), (77, 1000, 1096)])
+def test_dense_gemm_parity(qb, T, d_out, d_in):
+    # the serving GEMM of the 16-bit deployment on its own: ragged tiles in every dimension, K not a multiple of 64
+    W = synth.round_to_bf16(synth.normal(66, f"dg/W/{d_out}x{d_in}", (d_out, d_in), 0.02))
+    X = synth.round_to_bf16(synth.normal(66, f"dg/X/{T}", (T, d_in)))
+    ref = X.astype(np.float64) @ W.astype(np.float64).T
+    Wd, Xd = to_bf16_dev(W), to_bf16_dev(X)
+    for dt, gate in ((torch.float32, gate_strict), (torch.bfloat16, gate_bf16)):
+        g = Guarded()
+        Y = g.alloc((T, d_out), dt)
+        ws = g.alloc((256,), torch.uint8)
+        qb.dense_gemm(Wd, Xd, ws=ws, out=Y)
+        g.check("dense_gemm")
+        assert qb.device_status(ws) == qb.OK
+        gate(to_np64(Y), ref, f"dense gemm {T}x{d_out}x{d_in}")
+    # fp32 accumulation of exact bf16 products: far tighter than the gate
+    assert np.abs(to_np64(qb.dense_gemm(Wd, Xd, torch.float32)) - ref).max() <= 1e-5 * np.sqrt(d_in)
