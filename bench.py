@@ -484,7 +484,18 @@ def lowbit_extras(qb, torch, dev, peaks, l2_bytes, shapes=("q", "up"), tokens=(1
         q_bytes = Wd.numel() * 4 + packed_bytes(spec.d_out, spec.d_in)
         out[f"{spec.name}/quantize"] = {"us": q_us, "GB/s": q_bytes / q_us / 1e3, "frac_hbm": q_bytes / q_us / 1e3 / peaks["hbm_gbs"],
                                         "bytes": q_bytes, "note": "fp32 in (larger than L2), outputs preallocated"}
-        del Wd
+        # the same weight in the level-table format (the format of the fine-tuning configurations)
+        dq0 = qb.quantize_blockwise(Wd, 64, 1, qb.FMT_CODEBOOK_ABSMAX)
+        s.record()
+        for _ in range(5):
+            qb.quantize_blockwise(Wd, 64, 1, qb.FMT_CODEBOOK_ABSMAX, out=dq0)
+        e.record(); torch.cuda.synchronize()
+        q0_us = s.elapsed_time(e) / 5 * 1e3
+        q0_bytes = Wd.numel() * 4 + packed_bytes(spec.d_out, spec.d_in, with_beta=False)
+        out[f"{spec.name}/quantize_level_table"] = {"us": q0_us, "GB/s": q0_bytes / q0_us / 1e3,
+                                                    "frac_hbm": q0_bytes / q0_us / 1e3 / peaks["hbm_gbs"], "bytes": q0_bytes,
+                                                    "note": "fp32 in (larger than L2), outputs preallocated"}
+        del Wd, dq0
         ad = qb.Adapter(64, 8, wl.rank, 1.0, bf(li.A), bf(li.B))
         nbytes = packed_bytes(spec.d_out, spec.d_in)
         ncopies = int(np.ceil(2.0 * l2_bytes / nbytes)) + 1

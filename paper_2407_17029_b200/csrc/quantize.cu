@@ -10,7 +10,22 @@ struct QuantTable {
   float mid[15];  // fl32 midpoints between adjacent levels
   int zero_idx;   // index of the level closest to 0 (used for all-zero blocks)
   float qmax;     // largest code of the min-max grid: 2^N - 1 (15 for the 4-bit weight)
+  int use_lut;    // level table: midpoints far enough apart for the bucket table of code_of_level_lut
 };
+
+// Bucket table of the level-table format.  [-1, 1] is covered by 129 equal buckets centred on the multiples of 1/64
+// (the table has 256 entries so that any 8-bit index is in range); when adjacent midpoints
+// are farther apart than a bucket (plus margins), a bucket, widened by LUT_MARGIN on both sides, sees at most one
+// midpoint m, and for every v in it  #{ j : v > mid_j } = base + (v > m),  base = number of midpoints below m (or
+// below the bucket when it sees none; m is then a huge value).  An entry is ONE 32-bit word: the float m with its
+// four lowest mantissa bits replaced by base.  That moves m by less than 16 ulp < 1e-6, and a value closer than
+// LUT_NEAR = 2e-6 to the stored m is decided by the exact quotient anyway, so the comparison with the stored m gives
+// the same answer as with m itself everywhere else.  One 4-byte shared-memory load replaces the search.
+constexpr int LUT_BUCKETS = 256;
+constexpr float LUT_SCALE = 64.0f;       // buckets per unit: bucket of v = round(v * 64 + 64)
+constexpr float LUT_NEAR = 2e-6f;        // closer to the stored midpoint than this: the exact quotient decides
+constexpr float LUT_MARGIN = 8e-6f;      // > LUT_NEAR + 16 ulp + rounding of the bucket index (1.2e-7)
+constexpr float LUT_NONE = 3.0e38f;      // "no midpoint in this bucket"
 
 __device__ __forceinline__ float load_w(const float* W, int64_t i) { return W[i]; }
 __device__ __forceinline__ float load_w(const __nv_bfloat16* W, int64_t i) {
@@ -39,6 +54,20 @@ __device__ __forceinline__ int code_of_level_fast(float w, float absmax, float i
   k += (va > s_mid[k + 1]) ? 1 : 0;
   const float lo = s_mid[k], hi = s_mid[k + 1];
   if ((__fsub_rn(va, lo) > 1e-6f) && (__fsub_rn(hi, va) > 1e-6f)) return k;
+  return code_of_level(__fdiv_rn(w, absmax), t);
+}
+
+// The same decision through the bucket table (see LUT_BUCKETS): va lands in bucket round(va * 64 + 64), read off the
+// low mantissa bits after adding 2^23 (no conversion instruction, no clamp: |va| <= 1 up to rounding, and a
+// non-finite va still gives an index inside the table) -- or, when it sits within rounding of a bucket edge, in
+// the neighbour, whose widened range still covers it -- and the code is
+// base + (va > m) unless va is within LUT_NEAR of the stored m, where the exact quotient decides as before.
+__device__ __forceinline__ int code_of_level_lut(float w, float absmax, float inv, const uint32_t* s_lut, const QuantTable& t) {
+  const float va = __fmul_rn(w, inv);
+  const uint32_t b = __float_as_uint(fmaf(va, LUT_SCALE, 8388608.0f + LUT_SCALE)) & (uint32_t)(LUT_BUCKETS - 1);
+  const uint32_t e = s_lut[b];
+  const float m = __uint_as_float(e);
+  if (fabsf(__fsub_rn(va, m)) > LUT_NEAR) return (int)(e & 15u) + (va > m ? 1 : 0);
   return code_of_level(__fdiv_rn(w, absmax), t);
 }
 
@@ -71,8 +100,20 @@ __global__ void __launch_bounds__(256) quantize_b64_kernel(const TIn* __restrict
                                                            float* __restrict__ alpha,
                                                            float* __restrict__ beta) {
   __shared__ float s_mid[17];
+  __shared__ uint32_t s_lut[LUT_BUCKETS];
   if (threadIdx.x < 17)
     s_mid[threadIdx.x] = threadIdx.x == 0 ? -INFINITY : threadIdx.x == 16 ? INFINITY : tab.mid[min(max((int)threadIdx.x, 1), 15) - 1];
+  if (tab.use_lut && threadIdx.x < LUT_BUCKETS) {
+    const float lo = ((float)threadIdx.x - 0.5f) / LUT_SCALE - 1.0f, hi = ((float)threadIdx.x + 0.5f) / LUT_SCALE - 1.0f;   // exact
+    float m = LUT_NONE;
+    int base = 0, below = 0;
+#pragma unroll
+    for (int j = 0; j < 15; ++j) {
+      if (tab.mid[j] >= lo - LUT_MARGIN && tab.mid[j] < hi + LUT_MARGIN) { m = tab.mid[j]; base = j; }
+      below += tab.mid[j] < lo - LUT_MARGIN ? 1 : 0;
+    }
+    s_lut[threadIdx.x] = (__float_as_uint(m) & ~15u) | (uint32_t)(m == LUT_NONE ? below : base);
+  }
   __syncthreads();
   const int lane = threadIdx.x & 31, sub = lane >> 3, part = lane & 7;
   const int64_t warps_per_grid = (int64_t)gridDim.x * (blockDim.x >> 5);
@@ -109,7 +150,8 @@ __global__ void __launch_bounds__(256) quantize_b64_kernel(const TIn* __restrict
       const float inv = __frcp_rn(am);
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
-        const int c = am != 0.0f ? code_of_level_fast(v[e], am, inv, s_mid, tab) : tab.zero_idx;
+        const int c = am == 0.0f ? tab.zero_idx
+                      : tab.use_lut ? code_of_level_lut(v[e], am, inv, s_lut, tab) : code_of_level_fast(v[e], am, inv, s_mid, tab);
         packed |= (uint32_t)c << (4 * e);
       }
       if (live && part == 0) alpha[b] = am;
@@ -184,6 +226,7 @@ int launch_quantize(const void* W, int w_dtype, int d_out, int d_in, int block_i
                     cudaStream_t st) {
   QuantTable tab;
   tab.zero_idx = 0;
+  tab.use_lut = 0;
   tab.qmax = (float)((1 << bits) - 1);
   for (int j = 0; j < 15; ++j) tab.mid[j] = 0.0f;
   if (qfmt == QBLORA_FMT_CODEBOOK_ABSMAX) {
@@ -191,6 +234,12 @@ int launch_quantize(const void* W, int w_dtype, int d_out, int d_in, int block_i
       tab.mid[j] = (float)(((double)level[j] + (double)level[j + 1]) / 2.0);
     for (int j = 1; j < 16; ++j)
       if (fabs((double)level[j]) < fabs((double)level[tab.zero_idx])) tab.zero_idx = j;
+    // bucket table: every pair of adjacent midpoints farther apart than one widened bucket
+    tab.use_lut = 1;
+    for (int j = 0; j + 1 < 15; ++j)
+      if (!(tab.mid[j + 1] - tab.mid[j] > 1.0f / LUT_SCALE + 4.0f * LUT_MARGIN)) tab.use_lut = 0;
+    // (midpoints lie strictly inside (-1, 1): the levels are ascending and the caller's table spans [-1, 1])
+    for (int j = 0; j < 15; ++j) if (!(fabsf(tab.mid[j]) < 1.0f)) tab.use_lut = 0;
   }
   if (block_in == 64 && block_out == 1) {
     int64_t nblocks = (int64_t)d_out * (d_in / 64);

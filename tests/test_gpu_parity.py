@@ -106,6 +106,44 @@ def test_quantize_custom_table(qb):
     assert np.array_equal(got.codes.cpu().numpy(), ref.codes)
 
 
+def test_quantize_level_table_midpoints_on_bucket_edges_and_tight_tables(qb):
+    # The level-table quantizer finds a code through a table of 128 equal buckets over [-1, 1).  (a) A level table whose
+    # midpoints are multiples of 1/16 puts every midpoint exactly on a bucket edge; the block holds the midpoints
+    # themselves, their neighbours up to three ulps away and values a few 1e-7 .. 1e-5 beside them, at absmax 1 (the
+    # scaled value is the weight itself) and at an absmax that makes every quotient inexact.  (b) A table with two levels
+    # 0.002 apart cannot use the buckets and takes the search.  Codes and alpha equal the oracle's bit for bit.
+    table = np.array([-1, -0.875, -0.75, -0.625, -0.5, -0.375, -0.25, -0.125, 0, 0.125, 0.25, 0.375, 0.5, 0.625, 0.75, 1.0],
+                     dtype=np.float32)
+    mids = ((table[:-1].astype(np.float64) + table[1:].astype(np.float64)) / 2).astype(np.float32)
+    vals = [mids]
+    for k in (1, 2, 3):
+        up, dn = mids.copy(), mids.copy()
+        for _ in range(k):
+            up, dn = np.nextafter(up, np.float32(2)), np.nextafter(dn, np.float32(-2))
+        vals += [up, dn]
+    for off in (3e-7, 9e-7, 1.1e-6, 3e-6, 5e-6, 1e-5):
+        vals += [(mids + np.float32(off)).astype(np.float32), (mids - np.float32(off)).astype(np.float32)]
+    vals = np.concatenate(vals)                       # 19 x 15 = 285 values
+    rows = []
+    for scale in (1.0, 0.3, 1.7e-3):
+        v = (vals * np.float32(scale)).astype(np.float32)
+        v = np.concatenate([v, np.zeros((-len(v)) % 63, np.float32)]).reshape(-1, 63)
+        blk = np.concatenate([np.full((v.shape[0], 1), scale, np.float32), v], axis=1)     # absmax element first
+        rows.append(blk.reshape(1, -1))
+    W = np.concatenate(rows, axis=0)
+    assert W.shape[1] % 64 == 0
+    ref = oracle.quantize_blockwise(W, 64, 1, 0, table)
+    got = g_quantize(to_dev(W), 64, 1, 0, [float(x) for x in table])
+    assert np.array_equal(got.codes.cpu().numpy(), ref.codes)
+    assert np.array_equal(got.alpha.cpu().numpy().view(np.uint32), ref.alpha.view(np.uint32))
+    tight = np.linspace(-1.0, 1.0, 16).astype(np.float32)
+    tight[8] = tight[7] + np.float32(0.002)
+    Wr = synth.normal(35, "qz/tight", (64, 512), 0.5)
+    ref = oracle.quantize_blockwise(Wr, 64, 1, 0, tight)
+    got = g_quantize(to_dev(Wr), 64, 1, 0, [float(x) for x in tight])
+    assert np.array_equal(got.codes.cpu().numpy(), ref.codes)
+
+
 # --------------------------------------------------------------------------- forward / backward
 def make_case(seed, T, d_out, d_in, l1, l2, r, qfmt=0, ab_std=0.01, bi=64, bo=1, outliers=0.0):
     tag = f"case/{seed}"
