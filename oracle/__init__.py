@@ -118,6 +118,28 @@ def quantize_blockwise(W, block_in=64, block_out=1, qfmt=FMT_CODEBOOK_ABSMAX, co
     return QWeight(d_out, d_in, block_in, block_out, qfmt, code, codes, alpha, beta)
 
 
+def packed_row_bytes(d_in: int, nbits: int) -> int:
+    return d_in * nbits // 8
+
+
+def pack_codes(codes: np.ndarray, d_in: int, nbits: int) -> np.ndarray:
+    """Nibble-stored codes [d_out][d_in/2] -> dense N-bit storage [d_out][d_in*N/8], N = 2 or 3."""
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    d_out = codes.shape[0]
+    out = np.zeros((d_out, packed_row_bytes(d_in, nbits)), dtype=np.uint8)
+    _check(_L().orc_pack_codes(_p(codes, ctypes.c_uint8), d_out, d_in, int(nbits), _p(out, ctypes.c_uint8)), "pack_codes")
+    return out
+
+
+def unpack_codes(packed: np.ndarray, d_in: int, nbits: int) -> np.ndarray:
+    """Dense N-bit storage -> nibble-stored codes [d_out][d_in/2]."""
+    packed = np.ascontiguousarray(packed, dtype=np.uint8)
+    d_out = packed.shape[0]
+    out = np.zeros((d_out, d_in // 2), dtype=np.uint8)
+    _check(_L().orc_unpack_codes(_p(packed, ctypes.c_uint8), d_out, d_in, int(nbits), _p(out, ctypes.c_uint8)), "unpack_codes")
+    return out
+
+
 def dequantize(qw: QWeight) -> np.ndarray:
     Wt = np.zeros((qw.d_out, qw.d_in), dtype=np.float64)
     rc = _L().orc_dequantize(_p(qw.codes, ctypes.c_uint8), _p(qw.alpha, ctypes.c_float),

@@ -20,7 +20,8 @@
  * identity (Eq. 2 and the paragraph after it); finite differences and adjoint
  * identity for the backward pass; merge identity (Sec. 3.3); for the alternative
  * scale operators of the Sec. 4 ablation: slicing / zero-padding restatements,
- * the dense equivalent update, untouched outputs and finite differences.
+ * the dense equivalent update, untouched outputs and finite differences; dense
+ * N-bit packing: hand-written bit patterns, sizes and the round trip.
  * Parity unpinned: only two *conventions* -- the choice of the built-in 16-level
  * table (the paper cites NF4 without printing it) and which (lambda1, lambda2)
  * a benchmark config means.  Everything computed downstream of them is pinned.
@@ -160,6 +161,46 @@ int orc_quantize_blockwise(const float* W, int d_out, int d_in, int block_in,
       }
     }
   }
+  return ORC_OK;
+}
+
+/*
+ * Dense storage of N-bit codes, N = 2 or 3 (Eq. 1 is stated for N bits; the paper
+ * fixes no byte layout, so this one is the library's and is stated here in full):
+ *   N = 2: byte k of a row holds codes 4k .. 4k+3, code 4k+j in bits 2j .. 2j+1;
+ *          a row takes d_in / 4 bytes.
+ *   N = 3: codes 8k .. 8k+7 form the 24-bit number sum_j code(8k+j) << 3j, stored
+ *          little-endian in bytes 3k, 3k+1, 3k+2; a row takes 3 d_in / 8 bytes.
+ * `nibble` is the one-code-per-nibble layout used everywhere else ([d_out][d_in/2],
+ * low nibble = even column).  pack refuses a code that does not fit in N bits.
+ */
+static size_t packed_row_bytes(int d_in, int nbits) { return (size_t)d_in * (size_t)nbits / 8; }
+int orc_pack_codes(const uint8_t* nibble, int d_out, int d_in, int nbits, uint8_t* packed) {
+  if ((nbits != 2 && nbits != 3) || d_in % 8) return ORC_BAD;
+  const size_t rb = packed_row_bytes(d_in, nbits);
+  memset(packed, 0, rb * (size_t)d_out);
+  for (int o = 0; o < d_out; ++o)
+    for (int i = 0; i < d_in; ++i) {
+      int c = get_code(nibble, d_in, o, i);
+      if (c >> nbits) return ORC_BAD;
+      size_t bit = (size_t)i * (size_t)nbits;          /* position in the row's bit string, LSB first */
+      for (int b = 0; b < nbits; ++b, ++bit)
+        if ((c >> b) & 1) packed[(size_t)o * rb + bit / 8] |= (uint8_t)(1u << (bit % 8));
+    }
+  return ORC_OK;
+}
+int orc_unpack_codes(const uint8_t* packed, int d_out, int d_in, int nbits, uint8_t* nibble) {
+  if ((nbits != 2 && nbits != 3) || d_in % 8) return ORC_BAD;
+  const size_t rb = packed_row_bytes(d_in, nbits);
+  memset(nibble, 0, (size_t)d_out * (size_t)(d_in / 2));
+  for (int o = 0; o < d_out; ++o)
+    for (int i = 0; i < d_in; ++i) {
+      size_t bit = (size_t)i * (size_t)nbits;
+      int c = 0;
+      for (int b = 0; b < nbits; ++b, ++bit)
+        c |= ((packed[(size_t)o * rb + bit / 8] >> (bit % 8)) & 1) << b;
+      set_code(nibble, d_in, o, i, c);
+    }
   return ORC_OK;
 }
 

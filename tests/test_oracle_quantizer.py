@@ -265,3 +265,49 @@ def test_nbit_four_is_the_default_and_round_trip_is_stable():
         oracle.quantize_blockwise(W, 64, 1, oracle.FMT_AFFINE_MINMAX, nbits=5)
     with pytest.raises(ValueError):
         oracle.quantize_blockwise(W, 64, 1, oracle.FMT_CODEBOOK_ABSMAX, nbits=3)
+
+
+# ----------------------------------------------------------------- dense N-bit storage (N = 2, 3)
+def test_pack_two_bit_layout_by_hand():
+    # codes 0,1,2,3 in one byte: code j in bits 2j..2j+1 -> 0b11_10_01_00
+    nib = np.array([[0x10, 0x32, 0x03, 0x21]], dtype=np.uint8)     # codes 0,1,2,3,3,0,1,2 (low nibble = even column)
+    packed = oracle.pack_codes(nib, 8, 2)
+    assert packed.shape == (1, 2)
+    assert packed[0, 0] == 0b11100100 and packed[0, 1] == 0b10010011
+
+
+def test_pack_three_bit_layout_by_hand():
+    # codes 0..7 -> the 24-bit number sum_j j << 3j = 0o76543210, little-endian in three bytes
+    nib = np.array([[0x10, 0x32, 0x54, 0x76]], dtype=np.uint8)
+    packed = oracle.pack_codes(nib, 8, 3)
+    assert packed.shape == (1, 3)
+    value = int("76543210", 8)
+    assert [int(b) for b in packed[0]] == [value & 0xFF, (value >> 8) & 0xFF, (value >> 16) & 0xFF]
+    # a second group lands in the next three bytes and does not touch the first
+    nib2 = np.array([[0x10, 0x32, 0x54, 0x76, 0x77, 0x77, 0x77, 0x77]], dtype=np.uint8)
+    p2 = oracle.pack_codes(nib2, 16, 3)
+    assert np.array_equal(p2[0, :3], packed[0]) and [int(b) for b in p2[0, 3:]] == [0xFF, 0xFF, 0xFF]
+
+
+@pytest.mark.parametrize("nbits", [2, 3])
+def test_pack_round_trip_sizes_and_refusals(nbits):
+    rng = np.random.default_rng(5)
+    d_out, d_in = 7, 192
+    c = rng.integers(0, 1 << nbits, size=(d_out, d_in), dtype=np.uint8)
+    nib = (c[:, 0::2] | (c[:, 1::2] << 4)).astype(np.uint8)
+    packed = oracle.pack_codes(nib, d_in, nbits)
+    assert packed.shape == (d_out, d_in * nbits // 8)                 # N/8 bytes per weight
+    assert np.array_equal(oracle.unpack_codes(packed, d_in, nbits), nib)
+    # independent restatement: the row's bit string, least significant bit first
+    bits = ((c[:, :, None] >> np.arange(nbits)[None, None, :]) & 1).reshape(d_out, -1)
+    assert np.array_equal(np.packbits(bits, axis=1, bitorder="little"), packed)
+    # a code that needs more than N bits is refused
+    bad = nib.copy()
+    bad[0, 0] = 0x0F
+    with pytest.raises(ValueError):
+        oracle.pack_codes(bad, d_in, nbits)
+    # the quantizer's N-bit grid fits, and dequantizing the round-tripped codes changes nothing
+    W = np.random.default_rng(6).standard_normal((4, 128)).astype(np.float32)
+    qw = oracle.quantize_blockwise(W, 64, 1, oracle.FMT_AFFINE_MINMAX, nbits=nbits)
+    rt = oracle.unpack_codes(oracle.pack_codes(qw.codes, 128, nbits), 128, nbits)
+    assert np.array_equal(rt, qw.codes)
