@@ -96,6 +96,15 @@ typedef struct {
                                   high nibble = code(o,2k+1) */
   const float* alpha;          /* DEVICE [d_out/block_out][d_in/block_in] */
   const float* beta;           /* DEVICE same shape; NULL for the code-table format */
+  int32_t code_bits;           /* storage of `codes`: 0 or 4 = one code per nibble, as described above;
+                                  2 or 3 = dense N-bit storage (min-max format only, d_in % 32 == 0, every code < 2^N;
+                                  Eq. 1 is stated for N bits), written by qblora_pack_codes:
+                                    2: DEVICE [d_out][d_in/4],   byte k of row o: code(o,4k+j) in bits 2j..2j+1;
+                                    3: DEVICE [d_out][3*d_in/8], codes 8k..8k+7 of row o as the 24-bit number
+                                       sum_j code(o,8k+j) << 3j, little-endian in bytes 3k..3k+2.
+                                  Calls that read the codes expand such a weight to one code per nibble inside `ws` first
+                                  (qblora_workspace_bytes includes the d_out*d_in/2 bytes): the saving is in the memory the
+                                  weight occupies at rest, not in the bytes a product streams. */
 } qblora_qweight;
 
 /* The parameter-free operator pair that compresses the adapter's input and restores its output
@@ -187,14 +196,27 @@ int qblora_quantize_blockwise(const void* W, int w_dtype, int32_t d_out, int32_t
  *   beta = min; alpha = (max - min) / (2^N - 1); code = clamp(rint((w - beta) / alpha), 0, 2^N - 1), ties to even;
  *   constant block: alpha = 0, code = 0.  Same single-rounding fp32 arithmetic as above; bits = 4 gives exactly
  *   qblora_quantize_blockwise's min-max result.
- * Storage is unchanged: one code per nibble, codes uint8 [d_out][d_in/2] (no packing denser than 4 bits), so
- * the result is an ordinary QBLORA_FMT_AFFINE_MINMAX weight for every other call of this library (forward,
- * backward, both merges, low-bit product); what changes is the number of levels a weight can take.
+ * The codes come out one per nibble, codes uint8 [d_out][d_in/2], so the result is an ordinary
+ * QBLORA_FMT_AFFINE_MINMAX weight for every other call of this library (forward, backward, both merges, low-bit
+ * product); qblora_pack_codes turns 2- and 3-bit codes into dense storage (code_bits of qblora_qweight).
  * Arguments and requirements as for qblora_quantize_blockwise; beta must not be NULL.
  */
 int qblora_quantize_minmax_nbit(const void* W, int w_dtype, int32_t d_out, int32_t d_in,
                                 int32_t block_in, int32_t block_out, int32_t bits,
                                 uint8_t* codes, float* alpha, float* beta, void* stream);
+
+/*
+ * Dense storage for N-bit weights, N = bits in {2, 3} (Eq. 1 is stated for N bits; the paper fixes no byte layout --
+ * the layout is the one given at qblora_qweight.code_bits).
+ *   qblora_pack_codes:   codes DEVICE uint8 [d_out][d_in/2] (one per nibble, e.g. from qblora_quantize_minmax_nbit)
+ *                        -> packed DEVICE uint8 [d_out][d_in*bits/8].  ws: at least 256 bytes; qblora_device_status(ws)
+ *                        returns QBLORA_ERR_INVALID_ARG afterwards if some code did not fit in `bits` bits.
+ *   qblora_unpack_codes: the inverse.
+ * Requires d_in % 32 == 0; both buffers 16-byte aligned.
+ */
+int qblora_pack_codes(const uint8_t* codes, int32_t d_out, int32_t d_in, int32_t bits, uint8_t* packed, void* ws,
+                      size_t ws_bytes, void* stream);
+int qblora_unpack_codes(const uint8_t* packed, int32_t d_out, int32_t d_in, int32_t bits, uint8_t* codes, void* stream);
 
 /*
  * Forward of the adapted quantized linear (Sec. 3.1 combined formula with the Sec. 3.2 adapter;

@@ -31,14 +31,15 @@ EXPORTS = ["qblora_default_code_table", "qblora_workspace_bytes", "qblora_status
            "qblora_device_status", "qblora_quantize_blockwise", "qblora_linear_fwd",
            "qblora_linear_bwd", "qablora_merge", "qablora_lowbit_gemm", "qblora_kernel_launches",
            "qblora_set_timing_events", "qablora_merge_noalloc", "qblora_merge_dense",
-           "qblora_quantize_minmax_nbit", "qblora_debug_set_wait_limit", "qblora_debug_drop_load", "qblora_dense_gemm"]
+           "qblora_quantize_minmax_nbit", "qblora_debug_set_wait_limit", "qblora_debug_drop_load", "qblora_dense_gemm", "qblora_pack_codes", "qblora_unpack_codes"]
 
 
 class _CQWeight(ctypes.Structure):
     _fields_ = [("d_in", ctypes.c_int32), ("d_out", ctypes.c_int32),
                 ("block_in", ctypes.c_int32), ("block_out", ctypes.c_int32),
                 ("qfmt", ctypes.c_int32), ("code", ctypes.c_float * 16),
-                ("codes", ctypes.c_void_p), ("alpha", ctypes.c_void_p), ("beta", ctypes.c_void_p)]
+                ("codes", ctypes.c_void_p), ("alpha", ctypes.c_void_p), ("beta", ctypes.c_void_p),
+                ("code_bits", ctypes.c_int32)]
 
 
 class _CAdapter(ctypes.Structure):
@@ -84,6 +85,9 @@ _lib.qblora_kernel_launches.argtypes = []
 _lib.qblora_set_timing_events.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
 _lib.qblora_dense_gemm.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p,
                                    ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+_lib.qblora_pack_codes.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
+                                   ctypes.c_size_t, ctypes.c_void_p]
+_lib.qblora_unpack_codes.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]
 _lib.qblora_debug_set_wait_limit.argtypes = [ctypes.c_int64]
 _lib.qblora_debug_drop_load.argtypes = [ctypes.c_int32]
 
@@ -148,6 +152,7 @@ class QWeight:
     codes: torch.Tensor
     alpha: torch.Tensor
     beta: Optional[torch.Tensor]
+    code_bits: int = 4          # 4: codes one per nibble [d_out][d_in/2]; 2 / 3: dense storage [d_out][d_in*bits/8]
 
     def c_struct(self) -> _CQWeight:
         c = _CQWeight()
@@ -157,6 +162,7 @@ class QWeight:
         c.codes = self.codes.data_ptr()
         c.alpha = self.alpha.data_ptr()
         c.beta = self.beta.data_ptr() if self.beta is not None else None
+        c.code_bits = int(self.code_bits)
         return c
 
 
@@ -311,7 +317,7 @@ def merge(qw: QWeight, ad: Adapter, in_place: bool = False, ws: Optional[torch.T
     st = _lib.qablora_merge(ctypes.byref(cq), ctypes.byref(ca), beta_out.data_ptr(), ws.data_ptr(),
                             ws.numel(), _stream_ptr(stream))
     _check(st, "qablora_merge")
-    return QWeight(qw.d_out, qw.d_in, qw.block_in, qw.block_out, qw.qfmt, qw.code, qw.codes, qw.alpha, beta_out)
+    return QWeight(qw.d_out, qw.d_in, qw.block_in, qw.block_out, qw.qfmt, qw.code, qw.codes, qw.alpha, beta_out, qw.code_bits)
 
 
 def merge_dense(qw: QWeight, ad: Optional[Adapter], out: Optional[torch.Tensor] = None,
@@ -339,7 +345,7 @@ def merge_noalloc(qw: QWeight, ad: Adapter, beta_out: torch.Tensor, stream=None)
     ca = ad.c_struct()
     st = _lib.qablora_merge_noalloc(ctypes.byref(cq), ctypes.byref(ca), beta_out.data_ptr(), _stream_ptr(stream))
     _check(st, "qablora_merge_noalloc")
-    return QWeight(qw.d_out, qw.d_in, qw.block_in, qw.block_out, qw.qfmt, qw.code, qw.codes, qw.alpha, beta_out)
+    return QWeight(qw.d_out, qw.d_in, qw.block_in, qw.block_out, qw.qfmt, qw.code, qw.codes, qw.alpha, beta_out, qw.code_bits)
 
 
 def lowbit_gemm(qw: QWeight, X: torch.Tensor, out_dtype=torch.bfloat16, ws: Optional[torch.Tensor] = None,
@@ -370,3 +376,24 @@ def dense_gemm(W: torch.Tensor, X: torch.Tensor, out_dtype=torch.bfloat16, ws: O
                                 ws.numel(), _stream_ptr(stream))
     _check(st, "qblora_dense_gemm")
     return Y
+
+
+def pack_codes(qw: QWeight, bits: int, stream=None) -> QWeight:
+    """qblora_pack_codes: the same weight with its codes in dense `bits`-bit storage (bits = 2 or 3)."""
+    assert qw.code_bits == 4
+    packed = torch.empty((qw.d_out, qw.d_in * bits // 8), dtype=torch.uint8, device=qw.codes.device)
+    ws = torch.empty(256, dtype=torch.uint8, device=qw.codes.device)
+    st = _lib.qblora_pack_codes(qw.codes.data_ptr(), qw.d_out, qw.d_in, int(bits), packed.data_ptr(), ws.data_ptr(), ws.numel(),
+                                _stream_ptr(stream))
+    _check(st, "qblora_pack_codes")
+    _check(device_status(ws, stream), "qblora_pack_codes (a code does not fit)")
+    return QWeight(qw.d_out, qw.d_in, qw.block_in, qw.block_out, qw.qfmt, qw.code, packed, qw.alpha, qw.beta, int(bits))
+
+
+def unpack_codes(qw: QWeight, stream=None) -> QWeight:
+    """qblora_unpack_codes: dense storage back to one code per nibble."""
+    assert qw.code_bits in (2, 3)
+    codes = torch.empty((qw.d_out, qw.d_in // 2), dtype=torch.uint8, device=qw.codes.device)
+    st = _lib.qblora_unpack_codes(qw.codes.data_ptr(), qw.d_out, qw.d_in, int(qw.code_bits), codes.data_ptr(), _stream_ptr(stream))
+    _check(st, "qblora_unpack_codes")
+    return QWeight(qw.d_out, qw.d_in, qw.block_in, qw.block_out, qw.qfmt, qw.code, codes, qw.alpha, qw.beta, 4)

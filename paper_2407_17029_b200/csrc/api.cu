@@ -30,6 +30,12 @@ bool force_general() {
   return e && e[0] == '1';
 }
 
+// code_bits: 0 or 4 = one code per nibble; 2 or 3 = dense storage (min-max format, d_in a multiple of 32)
+bool code_bits_ok(const qblora_qweight* q) {
+  if (q->code_bits == 0 || q->code_bits == 4) return true;
+  return (q->code_bits == 2 || q->code_bits == 3) && q->qfmt == QBLORA_FMT_AFFINE_MINMAX && q->d_in % 32 == 0;
+}
+
 int make_qw(const qblora_qweight* q, QwView* v) {
   if (!q) return QBLORA_ERR_INVALID_ARG;
   if (q->d_in <= 0 || q->d_out <= 0 || q->block_in <= 0 || q->block_out <= 0) return QBLORA_ERR_INVALID_ARG;
@@ -37,6 +43,8 @@ int make_qw(const qblora_qweight* q, QwView* v) {
   if (q->qfmt != QBLORA_FMT_CODEBOOK_ABSMAX && q->qfmt != QBLORA_FMT_AFFINE_MINMAX) return QBLORA_ERR_INVALID_ARG;
   if (!q->codes || !q->alpha || !aligned16(q->codes) || !aligned16(q->alpha)) return QBLORA_ERR_INVALID_ARG;
   if (q->qfmt == QBLORA_FMT_AFFINE_MINMAX && (!q->beta || !aligned16(q->beta))) return QBLORA_ERR_INVALID_ARG;
+  if (!code_bits_ok(q)) return QBLORA_ERR_INVALID_ARG;
+  v->code_bits = q->code_bits == 0 ? 4 : q->code_bits;
   v->d_in = q->d_in; v->d_out = q->d_out; v->block_in = q->block_in; v->block_out = q->block_out;
   v->qfmt = q->qfmt; v->G = q->d_in / q->block_in;
   v->codes = q->codes; v->alpha = q->alpha;
@@ -49,9 +57,11 @@ int make_qw(const qblora_qweight* q, QwView* v) {
 bool make_qw_geom(const qblora_qweight* q, QwView* v) {
   if (!q || q->d_in <= 0 || q->d_out <= 0 || q->block_in <= 0 || q->block_out <= 0) return false;
   if (q->d_in % 2 || q->d_in % q->block_in || q->d_out % q->block_out) return false;
+  if (!code_bits_ok(q)) return false;
   std::memset(v, 0, sizeof(*v));
   v->d_in = q->d_in; v->d_out = q->d_out; v->block_in = q->block_in; v->block_out = q->block_out;
   v->qfmt = q->qfmt; v->G = q->d_in / q->block_in;
+  v->code_bits = q->code_bits == 0 ? 4 : q->code_bits;
   return true;
 }
 
@@ -89,6 +99,20 @@ AdView single_as_factored(const AdView& ad, const __nv_bfloat16* identity) {
   f.B = ad.A;          // H
   f.A = identity;
   return f;
+}
+
+// Densely stored codes (code_bits 2 or 3) are expanded to one code per nibble behind the op's own scratch.
+size_t expand_bytes(const QwView& q) { return q.code_bits < 4 ? align_up((size_t)q.d_out * q.d_in / 2, 256) : 0; }
+size_t with_expansion(size_t need, const QwView& q) { return q.code_bits < 4 ? align_up(need, 256) + expand_bytes(q) : need; }
+// Expands into ws + align_up(need, 256) and points the view at the expanded codes.
+int expand_codes(QwView* q, size_t need, void* ws, cudaStream_t st) {
+  if (q->code_bits >= 4) return QBLORA_OK;
+  uint8_t* dst = static_cast<uint8_t*>(ws) + align_up(need, 256);
+  const int rc = launch_unpack_codes(q->codes, q->d_out, q->d_in, q->code_bits, dst, st);
+  if (rc) return rc;
+  q->codes = dst;
+  q->code_bits = 4;
+  return QBLORA_OK;
 }
 
 size_t ws_bytes_impl(int op, const QwView& q, const AdView* ad, int64_t T);
@@ -152,9 +176,12 @@ size_t qblora_workspace_bytes(int op, const qblora_qweight* qw, const qblora_ada
     adp = &ad;
   }
   if (op != QBLORA_OP_MERGE && op != QBLORA_OP_MERGE_DENSE && op != QBLORA_OP_QUANTIZE && tokens < 1) return 0;
-  if (adp && !adapter->B && (op == QBLORA_OP_LINEAR_FWD || op == QBLORA_OP_LINEAR_BWD))
-    return ws_bytes_single(op, q, ad, tokens);
-  return ws_bytes_impl(op, q, adp, tokens);
+  const bool reads_codes = op == QBLORA_OP_LINEAR_FWD || op == QBLORA_OP_LINEAR_BWD || op == QBLORA_OP_MERGE_DENSE ||
+                           op == QBLORA_OP_LOWBIT_GEMM;
+  size_t need;
+  if (adp && !adapter->B && (op == QBLORA_OP_LINEAR_FWD || op == QBLORA_OP_LINEAR_BWD)) need = ws_bytes_single(op, q, ad, tokens);
+  else need = ws_bytes_impl(op, q, adp, tokens);
+  return reads_codes ? with_expansion(need, q) : need;
 }
 
 int qblora_device_status(const void* ws, void* stream) {
@@ -211,9 +238,11 @@ int qblora_linear_fwd(const qblora_qweight* qw, const qblora_adapter* adapter, c
   const bool single = adapter && !adapter->B;
   const size_t need = single ? ws_bytes_single(QBLORA_OP_LINEAR_FWD, q, ad, tokens)
                              : ws_bytes_impl(QBLORA_OP_LINEAR_FWD, q, adp, tokens);
-  if (!ws || !aligned16(ws) || ws_bytes < need) return QBLORA_ERR_WORKSPACE;
+  if (!ws || !aligned16(ws) || ws_bytes < with_expansion(need, q)) return QBLORA_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   rc = reset_status(ws, st);
+  if (rc) return rc;
+  rc = expand_codes(&q, need, ws, st);
   if (rc) return rc;
   if (single) {
     __nv_bfloat16* eye = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(ws) + need - single_identity_bytes(ad));
@@ -249,10 +278,14 @@ int qblora_linear_bwd(const qblora_qweight* qw, const qblora_adapter* adapter, c
   const bool single = adapter && !adapter->B;
   const size_t need = single ? ws_bytes_single(QBLORA_OP_LINEAR_BWD, q, ad, tokens)
                              : ws_bytes_impl(QBLORA_OP_LINEAR_BWD, q, adp, tokens);
-  if (!ws || !aligned16(ws) || ws_bytes < need) return QBLORA_ERR_WORKSPACE;
+  if (!ws || !aligned16(ws) || ws_bytes < with_expansion(need, q)) return QBLORA_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   rc = reset_status(ws, st);
   if (rc) return rc;
+  if (dX) {   // only the dX contraction reads the codes
+    rc = expand_codes(&q, need, ws, st);
+    if (rc) return rc;
+  }
   if (single) {
     __nv_bfloat16* eye = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(ws) + need - single_identity_bytes(ad));
     rc = launch_identity(eye, ad.P, st);
@@ -298,12 +331,31 @@ int qblora_merge_dense(const qblora_qweight* qw, const qblora_adapter* adapter, 
     adp = &ad;
   }
   const size_t need = merge_dense_ws_bytes(q, adp);
-  if (!ws || !aligned16(ws) || ws_bytes < need) return QBLORA_ERR_WORKSPACE;
+  if (!ws || !aligned16(ws) || ws_bytes < with_expansion(need, q)) return QBLORA_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   rc = reset_status(ws, st);
   if (rc) return rc;
+  rc = expand_codes(&q, need, ws, st);
+  if (rc) return rc;
   return launch_merge_dense(q, adp, adapter && adapter->B == nullptr, static_cast<__nv_bfloat16*>(W_out),
                             static_cast<char*>(ws), st);
+}
+
+int qblora_pack_codes(const uint8_t* codes, int32_t d_out, int32_t d_in, int32_t bits, uint8_t* packed, void* ws,
+                      size_t ws_bytes, void* stream) {
+  if (!codes || !packed || !aligned16(codes) || !aligned16(packed)) return QBLORA_ERR_INVALID_ARG;
+  if ((bits != 2 && bits != 3) || d_out < 1 || d_in < 32 || d_in % 32) return QBLORA_ERR_INVALID_ARG;
+  if (!ws || !aligned16(ws) || ws_bytes < kStatusBytes) return QBLORA_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int rc = reset_status(ws, st);
+  if (rc) return rc;
+  return launch_pack_codes(codes, d_out, d_in, bits, packed, static_cast<int*>(ws), st);
+}
+
+int qblora_unpack_codes(const uint8_t* packed, int32_t d_out, int32_t d_in, int32_t bits, uint8_t* codes, void* stream) {
+  if (!codes || !packed || !aligned16(codes) || !aligned16(packed)) return QBLORA_ERR_INVALID_ARG;
+  if ((bits != 2 && bits != 3) || d_out < 1 || d_in < 32 || d_in % 32) return QBLORA_ERR_INVALID_ARG;
+  return launch_unpack_codes(packed, d_out, d_in, bits, codes, static_cast<cudaStream_t>(stream));
 }
 
 int qblora_dense_gemm(const void* W, int32_t d_out, int32_t d_in, const void* X, int64_t tokens, void* Y, int y_dtype,
@@ -337,11 +389,15 @@ int qablora_lowbit_gemm(const qblora_qweight* qw, const void* X, int64_t tokens,
   if (q.qfmt != QBLORA_FMT_AFFINE_MINMAX) return QBLORA_ERR_INVALID_ARG;
   if (!X || !Y || !aligned16(X) || !aligned16(Y) || tokens < 1 || !dtype_ok(y_dtype)) return QBLORA_ERR_INVALID_ARG;
   const size_t need = ws_bytes_impl(QBLORA_OP_LOWBIT_GEMM, q, nullptr, tokens);
-  if (!ws || !aligned16(ws) || ws_bytes < need) return QBLORA_ERR_WORKSPACE;
+  if (!ws || !aligned16(ws) || ws_bytes < with_expansion(need, q)) return QBLORA_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const __nv_bfloat16* Xb = static_cast<const __nv_bfloat16*>(X);
-  // the decode kernel clears the status word itself: one launch per call
-  if (gemv_supported(q, tokens)) return launch_lowbit_gemv(q, Xb, tokens, Y, y_dtype, static_cast<int*>(ws), st);
+  const bool expanded = q.code_bits < 4;
+  rc = expand_codes(&q, need, ws, st);
+  if (rc) return rc;
+  // the decode kernel clears the status word itself: one launch per call (it is chained to its predecessor as a
+  // programmatic dependent unless that predecessor has just written the codes)
+  if (gemv_supported(q, tokens)) return launch_lowbit_gemv(q, Xb, tokens, Y, y_dtype, static_cast<int*>(ws), st, !expanded);
   rc = reset_status(ws, st);
   if (rc) return rc;
   if (!force_general() && tc_supported(q, nullptr, tokens))

@@ -16,6 +16,7 @@ namespace qb {
 // Device-side view of a frozen quantized weight (pointers are device pointers).
 struct QwView {
   int d_in, d_out, block_in, block_out, qfmt, G;  // G = d_in / block_in
+  int code_bits;   // storage of the codes: 4 = one per nibble; 2, 3 = dense (pack.cu), expanded into the workspace before use
   const uint8_t* codes;
   const float* alpha;
   const float* beta;
@@ -88,7 +89,11 @@ int launch_identity(__nv_bfloat16* out, int n, cudaStream_t st);   // bf16 ident
 bool gemv_supported(const QwView& qw, int64_t T);
 size_t gemv_ws_bytes(const QwView& qw, int64_t T);   // status word + (T > 1) token fragments
 int launch_lowbit_gemv(const QwView& qw, const __nv_bfloat16* X, int64_t T, void* Y, int y_dtype,
-                       int* status, cudaStream_t st);
+                       int* status, cudaStream_t st, bool chain = true);
+
+// Dense 2- / 3-bit code storage (pack.cu); d_in % 32 == 0.
+int launch_pack_codes(const uint8_t* nibble, int64_t d_out, int64_t d_in, int bits, uint8_t* packed, int* bad, cudaStream_t st);
+int launch_unpack_codes(const uint8_t* packed, int64_t d_out, int64_t d_in, int bits, uint8_t* nibble, cudaStream_t st);
 
 // Plain bf16 tcgen05 GEMM serving a dense merged weight: Y = X W^T, W bf16 [d_out][d_in] (d_in % 8 == 0).
 size_t dense_gemm_ws_bytes();

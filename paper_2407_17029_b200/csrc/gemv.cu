@@ -478,7 +478,7 @@ int t1_stages(int G) {   // ring depth that fits; 0 if fewer than six stages wou
   return n < T1_MAX_STAGES ? n : T1_MAX_STAGES;
 }
 int t1_launch(const CUtensorMap& tm_c, const CUtensorMap& tm_a, const CUtensorMap& tm_b, GtParams p, int grid,
-              cudaStream_t st) {
+              cudaStream_t st, bool chain) {
   p.stages = t1_stages(p.G);
   const size_t smem = t1_fixed_smem(p.G) + (size_t)p.stages * GT_STAGE_BYTES;
   QB_CUDA(cudaFuncSetAttribute(lowbit_gemv_t1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -487,7 +487,7 @@ int t1_launch(const CUtensorMap& tm_c, const CUtensorMap& tm_a, const CUtensorMa
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr; cfg.numAttrs = 1;
+  cfg.attrs = attr; cfg.numAttrs = chain ? 1 : 0;
   QB_CUDA(cudaLaunchKernelEx(&cfg, lowbit_gemv_t1_kernel, tm_c, tm_a, tm_b, p));
   return QBLORA_OK;
 }
@@ -811,7 +811,7 @@ int ko_stages() {
 }
 template <int NT>
 int ko_launch(const CUtensorMap& tm_c, const CUtensorMap& tm_a, const CUtensorMap& tm_b, GtParams p, int grid,
-              uint8_t* xfrag, cudaStream_t st) {
+              uint8_t* xfrag, cudaStream_t st, bool chain) {
   p.stages = ko_stages<NT>();
   const int items = p.n_kc * GT_GROUPS * KoCfg<NT>::NTOK * 4;
   cudaLaunchAttribute attr[1];
@@ -820,7 +820,7 @@ int ko_launch(const CUtensorMap& tm_c, const CUtensorMap& tm_a, const CUtensorMa
   {
     cudaLaunchConfig_t pc{};
     pc.gridDim = dim3((unsigned)((items + 255) / 256)); pc.blockDim = dim3(256); pc.dynamicSmemBytes = 0; pc.stream = st;
-    pc.attrs = attr; pc.numAttrs = 1;
+    pc.attrs = attr; pc.numAttrs = chain ? 1 : 0;
     QB_CUDA(cudaLaunchKernelEx(&pc, x_prepare_kernel<NT>, p.X, p.T, p.d_in, p.G, p.n_kc, xfrag));
   }
   count_launch();
@@ -828,7 +828,7 @@ int ko_launch(const CUtensorMap& tm_c, const CUtensorMap& tm_a, const CUtensorMa
   QB_CUDA(cudaFuncSetAttribute(lowbit_gemv_ko_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(KO_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = st;
-  cfg.attrs = attr; cfg.numAttrs = 1;
+  cfg.attrs = attr; cfg.numAttrs = chain ? 1 : 0;
   const uint8_t* xf = xfrag;
   QB_CUDA(cudaLaunchKernelEx(&cfg, lowbit_gemv_ko_kernel<NT>, tm_c, tm_a, tm_b, p, xf));
   return QBLORA_OK;
@@ -853,8 +853,10 @@ size_t gemv_ws_bytes(const QwView& qw, int64_t T) {
   return kStatusBytes + (frag > T1_TAIL_BYTES ? frag : T1_TAIL_BYTES);
 }
 
+// `chain`: launch as programmatic dependents (the weight stream starts while the predecessor drains).  false when the
+// weight itself was written by the kernel in front (densely stored codes just expanded into the workspace).
 int launch_lowbit_gemv(const QwView& qw, const __nv_bfloat16* X, int64_t T, void* Y, int y_dtype, int* status,
-                       cudaStream_t st) {
+                       cudaStream_t st, bool chain) {
   uint8_t* xfrag = reinterpret_cast<uint8_t*>(status) + kStatusBytes;   // fragments of x (see gemv_ws_bytes)
   GtParams p{};
   p.d_in = qw.d_in; p.d_out = qw.d_out; p.G = qw.G; p.T = (int)T;
@@ -901,9 +903,9 @@ int launch_lowbit_gemv(const QwView& qw, const __nv_bfloat16* X, int64_t T, void
   {
     DominantKernelTimer timer(st);
     count_launch();
-    if (one_token) rc = t1_launch(tm_c, tm_a, tm_b, p, grid, st);
-    else if (T <= 8) rc = ko_launch<1>(tm_c, tm_a, tm_b, p, grid, xfrag, st);
-    else rc = ko_launch<2>(tm_c, tm_a, tm_b, p, grid, xfrag, st);
+    if (one_token) rc = t1_launch(tm_c, tm_a, tm_b, p, grid, st, chain);
+    else if (T <= 8) rc = ko_launch<1>(tm_c, tm_a, tm_b, p, grid, xfrag, st, chain);
+    else rc = ko_launch<2>(tm_c, tm_a, tm_b, p, grid, xfrag, st, chain);
     if (rc) return rc;
   }
   QB_CUDA(cudaGetLastError());

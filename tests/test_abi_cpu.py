@@ -102,7 +102,7 @@ def test_binding_struct_layouts_match_the_header(tmp_path):
     # the header is plain C: compile a probe against it and compare sizes and member offsets with the ctypes mirrors
     import subprocess
     from paper_2407_17029_b200 import binding
-    members = {"qblora_qweight": ["d_in", "d_out", "block_in", "block_out", "qfmt", "code", "codes", "alpha", "beta"],
+    members = {"qblora_qweight": ["d_in", "d_out", "block_in", "block_out", "qfmt", "code", "codes", "alpha", "beta", "code_bits"],
                "qblora_adapter": ["lambda_in", "lambda_out", "rank", "scaling", "A", "B", "scale_op"]}
     lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "qblora.h"', 'int main(void) {']
     for s, ms in members.items():

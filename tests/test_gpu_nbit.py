@@ -130,3 +130,77 @@ def test_quantize_level_table_near_midpoints_bit_exact(qb):
     v = W.astype(np.float64) / ref.alpha.astype(np.float64)
     near = np.abs(v[..., None] - mids.astype(np.float64)).min(axis=-1) < 1e-6
     assert near.mean() > 0.5
+
+
+# ------------------------------------------------------------------------ dense 2- / 3-bit storage
+@pytest.mark.parametrize("bits", [2, 3])
+@pytest.mark.parametrize("shape", [(200, 192), (64, 1024), (1, 32)])
+def test_pack_codes_bit_exact_and_round_trip(qb, bits, shape):
+    from tests._parity import Guarded
+    d_out, d_in = shape
+    rng = np.random.default_rng(11)
+    c = rng.integers(0, 1 << bits, size=(d_out, d_in), dtype=np.uint8)
+    nib = (c[:, 0::2] | (c[:, 1::2] << 4)).astype(np.uint8)
+    ref = oracle.pack_codes(nib, d_in, bits)
+    alpha = torch.ones((d_out, max(d_in // 32, 1)), device="cuda:0")
+    qw = qb.QWeight(d_out, d_in, 32, 1, qb.FMT_AFFINE_MINMAX, [0.0] * 16, to_dev(nib), alpha, alpha.clone())
+    packed = qb.pack_codes(qw, bits)
+    assert packed.code_bits == bits and tuple(packed.codes.shape) == (d_out, d_in * bits // 8)
+    assert np.array_equal(packed.codes.cpu().numpy(), ref)
+    assert torch.equal(qb.unpack_codes(packed).codes, qw.codes)
+    # outputs between guard bands (the kernels work on 32-code units)
+    g = Guarded()
+    out = g.alloc((d_out, d_in * bits // 8), torch.uint8)
+    ws = g.alloc((256,), torch.uint8)
+    assert qb._lib.qblora_pack_codes(qw.codes.data_ptr(), d_out, d_in, bits, out.data_ptr(), ws.data_ptr(), 256, None) == qb.OK
+    g.check("pack_codes")
+    assert torch.equal(out, packed.codes)
+    # a code that needs more than `bits` bits is reported through the status word
+    bad = qw.codes.clone()
+    bad[0, 0] = 0x0F
+    qbad = qb.QWeight(d_out, d_in, 32, 1, qb.FMT_AFFINE_MINMAX, [0.0] * 16, bad, alpha, alpha.clone())
+    with pytest.raises(qb.QbloraError) as e:
+        qb.pack_codes(qbad, bits)
+    assert e.value.status == qb.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("bits", [2, 3])
+def test_densely_stored_weight_through_every_call(qb, bits):
+    # the same 2- / 3-bit weight stored one code per nibble and densely: every call that reads the codes gives the
+    # same result bit for bit (the dense codes are expanded inside the workspace), and that result matches the oracle
+    # computed from the oracle's own pack / unpack of the oracle's quantization
+    from tests._parity import g_linear_bwd, g_linear_fwd, g_lowbit_gemm
+    T, d_out, d_in, l1, l2, r = 300, 320, 512, 64, 8, 48
+    W = synth.normal(83, "nbit/dense/W", (d_out, d_in), 0.02)
+    X, _ = synth.make_activations(83, "nbit/dense/X", T, d_in, 0.0)
+    dY = synth.round_to_bf16(synth.normal(83, "nbit/dense/dY", (T, d_out)))
+    A = synth.round_to_bf16(synth.normal(83, "nbit/dense/A", (d_in // l1, r), 0.01))
+    B = synth.round_to_bf16(synth.normal(83, "nbit/dense/B", (r, d_out // l2), 0.01))
+    qw = oracle.quantize_blockwise(W, 64, 1, oracle.FMT_AFFINE_MINMAX, nbits=bits)
+    qw.codes = oracle.unpack_codes(oracle.pack_codes(qw.codes, d_in, bits), d_in, bits)
+    Wt = oracle.dequantize(qw)
+    ad = oracle.Adapter(l1, l2, r, 1.0, A, B)
+    ad.scaling = visible_scaling(Wt, ad, X)
+    nib = qb.quantize_minmax_nbit(to_dev(W), bits)
+    dense = qb.pack_codes(nib, bits)
+    assert dense.codes.numel() * 8 == d_out * d_in * bits
+    assert qb.workspace_bytes(qb.OP_LINEAR_FWD, dense, None, T) >= qb.workspace_bytes(qb.OP_LINEAR_FWD, nib, None, T) + d_out * d_in // 2
+    da, Xd, dYd = adapter_to_dev(ad), to_bf16_dev(X), to_bf16_dev(dY)
+    Y = g_linear_fwd(dense, da, Xd, torch.float32)
+    assert torch.equal(Y, qb.linear_fwd(nib, da, Xd, torch.float32))
+    gate_strict(to_np64(Y), oracle.linear_fwd(Wt, ad, X), "Y from dense codes")
+    dX, dA, dB = g_linear_bwd(dense, da, Xd, dYd, torch.float32)
+    nX, nA, nB = qb.linear_bwd(nib, da, Xd, dYd, torch.float32)
+    assert torch.equal(dX, nX) and torch.equal(dA, nA) and torch.equal(dB, nB)
+    gate_strict(to_np64(dX), oracle.linear_bwd(Wt, ad, X, dY)[0], "dX from dense codes")
+    # offset merge keeps the dense codes; the merged dense weight serves the low-bit product at every token count
+    merged = qb.merge(dense, da)
+    assert merged.code_bits == bits and merged.codes.data_ptr() == dense.codes.data_ptr()
+    assert np.array_equal(merged.beta.cpu().numpy().view(np.uint32), oracle.merge(qw, ad).beta.view(np.uint32))
+    unmerged = oracle.linear_fwd(Wt, ad, X)
+    for Tn in (1, 5, 16, T):
+        Yl = g_lowbit_gemm(merged, Xd[:Tn].contiguous(), torch.float32)
+        gate_strict(to_np64(Yl), unmerged[:Tn], f"low-bit product from dense codes, T={Tn}")
+    # dense 16-bit merge
+    Wm = qb.merge_dense(dense, da)
+    assert torch.equal(Wm, qb.merge_dense(nib, da))
