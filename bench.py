@@ -445,7 +445,8 @@ def run_gpu(args, wl, geom):
         line["lowbit"] = lowbit_extras(qb, torch, ctx.dev, ctx.peaks, ctx.l2_bytes, args.lowbit_shapes.split(","),
                                        [int(t) for t in args.lowbit_tokens.split(",")])
         torch.cuda.empty_cache()
-        line["dense_16bit"] = dense_extras(qb, torch, ctx.dev, ctx.peaks)
+        if not args.no_dense:
+            line["dense_16bit"] = dense_extras(qb, torch, ctx.dev, ctx.peaks)
     if ctx.rank == 0 and not args.no_cpu_baseline and ctx.world == 1:
         rows = ref_rows_for(wl, geom, args.ref_rows)
         cache = oracle_cache(wl, geom, rows)
@@ -642,7 +643,8 @@ def main():
                          "2 interval sampling & zero fill (Sec. 4 ablation)")
     ap.add_argument("--ref-rows", type=int, default=0, help="token rows per oracle step (bounded sample; 0 = sized for about 45 GF per step)")
     ap.add_argument("--ref-max-steps", type=int, default=3)
-    ap.add_argument("--no-extras", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the deploy-path blocks (lowbit, dense_16bit)")
+    ap.add_argument("--no-dense", action="store_true", help="skip the dense_16bit block only")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of graph replay")
     ap.add_argument("--lowbit-shapes", default="q,up", help="linears of C5 timed in the lowbit extras")
