@@ -489,7 +489,7 @@ def lowbit_extras(qb, torch, dev, peaks, l2_bytes, shapes=("q", "up"), tokens=(1
         dq0 = qb.quantize_blockwise(Wd, 64, 1, qb.FMT_CODEBOOK_ABSMAX)
         s.record()
         for _ in range(5):
-            qb.quantize_blockwise(Wd, 64, 1, qb.FMT_CODEBOOK_ABSMAX, out=dq0)
+            qb.quantize_blockwise(Wd, 64, 1, qb.FMT_CODEBOOK_ABSMAX, code=dq0.code, out=dq0)   # (table passed in: building the default one costs host time)
         e.record(); torch.cuda.synchronize()
         q0_us = s.elapsed_time(e) / 5 * 1e3
         q0_bytes = Wd.numel() * 4 + packed_bytes(spec.d_out, spec.d_in, with_beta=False)

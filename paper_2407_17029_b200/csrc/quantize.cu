@@ -20,7 +20,10 @@ struct QuantTable {
 // below the bucket when it sees none; m is then a huge value).  An entry is ONE 32-bit word: the float m with its
 // four lowest mantissa bits replaced by base.  That moves m by less than 16 ulp < 1e-6, and a value closer than
 // LUT_NEAR = 2e-6 to the stored m is decided by the exact quotient anyway, so the comparison with the stored m gives
-// the same answer as with m itself everywhere else.  One 4-byte shared-memory load replaces the search.
+// the same answer as with m itself everywhere else.  One 4-byte shared-memory load replaces the search.  The bucket
+// of v is round(v * 64 + 64), read off the low mantissa bits after adding 2^23 (no conversion instruction, no clamp:
+// |v| <= 1 up to rounding, and a non-finite v still gives an index inside the table); a v within rounding of a
+// bucket edge may land in the neighbour, whose widened range still covers it.
 constexpr int LUT_BUCKETS = 256;
 constexpr float LUT_SCALE = 64.0f;       // buckets per unit: bucket of v = round(v * 64 + 64)
 constexpr float LUT_NEAR = 2e-6f;        // closer to the stored midpoint than this: the exact quotient decides
@@ -54,20 +57,6 @@ __device__ __forceinline__ int code_of_level_fast(float w, float absmax, float i
   k += (va > s_mid[k + 1]) ? 1 : 0;
   const float lo = s_mid[k], hi = s_mid[k + 1];
   if ((__fsub_rn(va, lo) > 1e-6f) && (__fsub_rn(hi, va) > 1e-6f)) return k;
-  return code_of_level(__fdiv_rn(w, absmax), t);
-}
-
-// The same decision through the bucket table (see LUT_BUCKETS): va lands in bucket round(va * 64 + 64), read off the
-// low mantissa bits after adding 2^23 (no conversion instruction, no clamp: |va| <= 1 up to rounding, and a
-// non-finite va still gives an index inside the table) -- or, when it sits within rounding of a bucket edge, in
-// the neighbour, whose widened range still covers it -- and the code is
-// base + (va > m) unless va is within LUT_NEAR of the stored m, where the exact quotient decides as before.
-__device__ __forceinline__ int code_of_level_lut(float w, float absmax, float inv, const uint32_t* s_lut, const QuantTable& t) {
-  const float va = __fmul_rn(w, inv);
-  const uint32_t b = __float_as_uint(fmaf(va, LUT_SCALE, 8388608.0f + LUT_SCALE)) & (uint32_t)(LUT_BUCKETS - 1);
-  const uint32_t e = s_lut[b];
-  const float m = __uint_as_float(e);
-  if (fabsf(__fsub_rn(va, m)) > LUT_NEAR) return (int)(e & 15u) + (va > m ? 1 : 0);
   return code_of_level(__fdiv_rn(w, absmax), t);
 }
 
@@ -148,11 +137,32 @@ __global__ void __launch_bounds__(256) quantize_b64_kernel(const TIn* __restrict
     uint32_t packed = 0;
     if (qfmt == QBLORA_FMT_CODEBOOK_ABSMAX) {
       const float inv = __frcp_rn(am);
+      if (tab.use_lut) {
+        // bucket table, no branch per element: the eight codes are formed unconditionally while the smallest distance
+        // to a stored midpoint is tracked; a lane that came closer than LUT_NEAR to one (about one lane in 10^4)
+        // redoes its eight codes with the exact quotient
+        float nearest = INFINITY;
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        const int c = am == 0.0f ? tab.zero_idx
-                      : tab.use_lut ? code_of_level_lut(v[e], am, inv, s_lut, tab) : code_of_level_fast(v[e], am, inv, s_mid, tab);
-        packed |= (uint32_t)c << (4 * e);
+        for (int e = 0; e < 8; ++e) {
+          const float va = __fmul_rn(v[e], inv);
+          const uint32_t b = __float_as_uint(fmaf(va, LUT_SCALE, 8388608.0f + LUT_SCALE)) & (uint32_t)(LUT_BUCKETS - 1);
+          const uint32_t en = s_lut[b];
+          const float m = __uint_as_float(en);
+          nearest = fminf(nearest, fabsf(__fsub_rn(va, m)));
+          packed += ((en & 15u) + (va > m ? 1u : 0u)) << (4 * e);
+        }
+        if (!(nearest > LUT_NEAR) || !(am > 0.0f) || !(inv > 0.0f)) {   // also the all-zero block (va would be NaN) and an absmax whose reciprocal is not finite
+          packed = 0;
+#pragma unroll
+          for (int e = 0; e < 8; ++e)
+            packed |= (uint32_t)(am != 0.0f ? code_of_level(__fdiv_rn(v[e], am), tab) : tab.zero_idx) << (4 * e);
+        }
+      } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const int c = am != 0.0f ? code_of_level_fast(v[e], am, inv, s_mid, tab) : tab.zero_idx;
+          packed |= (uint32_t)c << (4 * e);
+        }
       }
       if (live && part == 0) alpha[b] = am;
     } else {
