@@ -87,6 +87,32 @@ def test_quantize_signed_zero_block_minimum(qb, dtype):
     assert np.array_equal(got.codes.cpu().numpy(), ref.codes)
 
 
+@pytest.mark.parametrize("qfmt", [0, 1])
+def test_quantize_non_finite_weights_stay_inside_their_block(qb, qfmt):
+    # NaN / Inf weights are outside the method (Eq. 1 has no value for them): the call must neither fault nor let them
+    # leak -- every block that holds only finite weights still comes out bit for bit as in the oracle, and every code of
+    # a poisoned block is a valid 4-bit code.
+    W = synth.normal(36, "qz/nonfinite", (32, 512), 0.02)
+    clean = W.copy()
+    W[3, 70] = np.nan
+    W[5, 128] = np.inf
+    W[5, 129] = -np.inf
+    W[9, 0] = np.inf
+    got = g_quantize(to_dev(W), 64, 1, qfmt)
+    ref = oracle.quantize_blockwise(clean, 64, 1, qfmt)
+    codes, alpha = got.codes.cpu().numpy(), got.alpha.cpu().numpy()
+    poisoned = {(3, 1), (5, 2), (9, 0)}
+    for o in range(32):
+        for b in range(8):
+            if (o, b) in poisoned:
+                continue
+            assert np.array_equal(codes[o, 32 * b:32 * b + 32], ref.codes[o, 32 * b:32 * b + 32])
+            assert alpha[o, b].view(np.uint32) == ref.alpha[o, b].view(np.uint32)
+            if qfmt == 1:
+                assert got.beta.cpu().numpy()[o, b].view(np.uint32) == ref.beta[o, b].view(np.uint32)
+    torch.cuda.synchronize()
+
+
 def test_quantize_round_trip_on_device(qb):
     # Q(D(Q(W))) == Q(W) on the level-table format, dequantizing with the oracle in between
     W = synth.normal(32, "qz/rt", (128, 512), 0.02)
