@@ -304,6 +304,9 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
     const uint32_t leader_peer = map_to_cta(peer(0), 0);
     uint32_t k_m4 = 0x44444444u, k_c3210 = 0x32103210u;   // constants of lookup8, pinned to registers
     asm volatile("" : "+r"(k_m4), "+r"(k_c3210));
+    // low-bit product: the per-block table offsets (and gamma) come from the kernel launched just before this one,
+    // which may still be running when this grid starts as its programmatic dependent
+    if (p.kb_gamma) asm volatile("griddepcontrol.wait;" ::: "memory");
     bool ok = true;
     uint32_t it = 0;
     float al_next = 0.0f, be_next = 0.0f;   // scale and offset of this group's next weight K-block of the tile,
@@ -555,10 +558,9 @@ __device__ __forceinline__ void store_split(float x, __nv_bfloat16* hi, __nv_bfl
 // launched as a programmatic dependent further down the chain, can move in while the last CTAs here drain.
 constexpr int SEGSUM_UNROLL = 2;
 template <bool DIVIDE>
-__global__ void __launch_bounds__(256, 8) segsum_split_kernel(const __nv_bfloat16* __restrict__ src, int64_t rows, int width,
-                                                           int lam, float scale, int ld_out,
-                                                           __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the small product that follows may set up now
+__device__ __forceinline__ void segsum_split_body(int64_t block, const __nv_bfloat16* __restrict__ src, int64_t rows, int width,
+                                                  int lam, float scale, int ld_out,
+                                                  __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
   constexpr int UNROLL = SEGSUM_UNROLL;   // 16-byte loads in flight per thread (the kernel is a pure stream)
   const int chunks_per_row = width >> 3;
   const int64_t total = rows * chunks_per_row;
@@ -566,7 +568,7 @@ __global__ void __launch_bounds__(256, 8) segsum_split_kernel(const __nv_bfloat1
   int64_t tt[UNROLL]; int cc[UNROLL]; bool lv[UNROLL];
 #pragma unroll
   for (int k = 0; k < UNROLL; ++k) {
-    const int64_t idx = ((int64_t)blockIdx.x * UNROLL + k) * blockDim.x + threadIdx.x;
+    const int64_t idx = (block * UNROLL + k) * blockDim.x + threadIdx.x;
     lv[k] = idx < total;
     tt[k] = 0; cc[k] = 0;
     q4[k] = make_uint4(0, 0, 0, 0);
@@ -604,6 +606,13 @@ __global__ void __launch_bounds__(256, 8) segsum_split_kernel(const __nv_bfloat1
       }
     }
   }
+}
+template <bool DIVIDE>
+__global__ void __launch_bounds__(256, 8) segsum_split_kernel(const __nv_bfloat16* __restrict__ src, int64_t rows, int width,
+                                                           int lam, float scale, int ld_out,
+                                                           __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the small product that follows may set up now
+  segsum_split_body<DIVIDE>(blockIdx.x, src, rows, width, lam, scale, ld_out, hi, lo);
 }
 inline bool segsum_fast_ok(int width, int lam) {
   if (width % 8) return false;
@@ -674,12 +683,11 @@ __global__ void sample_split_kernel(const __nv_bfloat16* __restrict__ src, int64
 // uses, so alpha * c + beta_c is centred on zero and its bf16 rounding error is that of the weight's own spread,
 // whatever shift a merge has put into beta'), and gamma = beta' - beta_c, kept as a bf16 hi + lo pair for the
 // offset-term K-blocks.  The last block of a row also zeroes the row's padding columns.
-__global__ void __launch_bounds__(256) lowbit_center_kernel(const uint8_t* __restrict__ codes, const float* __restrict__ alpha,
-                                                           const float* __restrict__ beta, int64_t nblocks, int G, int ldg,
-                                                           float* __restrict__ beta_c, __nv_bfloat16* __restrict__ gam_h,
-                                                           __nv_bfloat16* __restrict__ gam_l) {
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  const int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+__device__ __forceinline__ void lowbit_center_body(int64_t block, const uint8_t* __restrict__ codes, const float* __restrict__ alpha,
+                                                   const float* __restrict__ beta, int64_t nblocks, int G, int ldg,
+                                                   float* __restrict__ beta_c, __nv_bfloat16* __restrict__ gam_h,
+                                                   __nv_bfloat16* __restrict__ gam_l) {
+  const int64_t b = block * blockDim.x + threadIdx.x;
   if (b >= nblocks) return;
   const uint4* src = reinterpret_cast<const uint4*>(codes + b * 32);
   const uint4 q0 = __ldg(src), q1 = __ldg(src + 1);
@@ -702,6 +710,19 @@ __global__ void __launch_bounds__(256) lowbit_center_kernel(const uint8_t* __res
   store_split(gm, gam_h, gam_l, row * ldg + g);
   if (g == G - 1)
     for (int k = G; k < ldg; ++k) { gam_h[row * ldg + k] = __float2bfloat16_rn(0.0f); gam_l[row * ldg + k] = __float2bfloat16_rn(0.0f); }
+}
+
+// The two preparations of the low-bit product in ONE launch (they are independent and each is too small to fill the
+// GPU for long): CTAs [0, center_ctas) split the offsets, the rest form the group sums of x.
+__global__ void __launch_bounds__(256, 8) lowbit_prepare_kernel(int center_ctas, const uint8_t* __restrict__ codes,
+                                                               const float* __restrict__ alpha, const float* __restrict__ beta,
+                                                               int64_t nblocks, int G, int ldg, float* __restrict__ beta_c,
+                                                               __nv_bfloat16* __restrict__ gam_h, __nv_bfloat16* __restrict__ gam_l,
+                                                               const __nv_bfloat16* __restrict__ X, int64_t T, int d_in,
+                                                               __nv_bfloat16* __restrict__ s_h, __nv_bfloat16* __restrict__ s_l) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the contraction that follows may set up now
+  if ((int)blockIdx.x < center_ctas) lowbit_center_body(blockIdx.x, codes, alpha, beta, nblocks, G, ldg, beta_c, gam_h, gam_l);
+  else segsum_split_body<false>((int64_t)blockIdx.x - center_ctas, X, T, d_in, BK, 1.0f, ldg, s_h, s_l);
 }
 
 int num_sms() {
@@ -939,14 +960,13 @@ int tc_lowbit_gemm(const QwView& qw, const __nv_bfloat16* X, int64_t T, void* Y,
   if (!tc_lowbit_split_offsets(qw)) return launch_main(0, qw, nullptr, X, nullptr, 0, T, Y, y_dtype, status, st);
   const LowbitWs w = carve_lowbit(qw, T, ws);
   const int64_t nblocks = (int64_t)qw.d_out * qw.G;
-  lowbit_center_kernel<<<(unsigned)((nblocks + 255) / 256), 256, 0, st>>>(qw.codes, qw.alpha, qw.beta, nblocks, qw.G, w.ldg,
-                                                                      w.beta_c, w.gam_h, w.gam_l);
-  count_launch();
-  QB_CUDA(cudaGetLastError());
-  // group sums of x (d_in is a multiple of 64 here, so the one-load-per-thread kernel applies)
+  // offsets split per block and group sums of x (d_in is a multiple of 64 here, so the one-load-per-thread
+  // segment sum applies), in one launch
   const int64_t chunks = T * (qw.d_in / 8);
-  segsum_split_kernel<false><<<(unsigned)((chunks + 256 * SEGSUM_UNROLL - 1) / (256 * SEGSUM_UNROLL)), 256, 0, st>>>(
-      X, T, qw.d_in, BK, 1.0f, w.ldg, w.s_h, w.s_l);
+  const int center_ctas = (int)((nblocks + 255) / 256);
+  const int64_t sum_ctas = (chunks + 256 * SEGSUM_UNROLL - 1) / (256 * SEGSUM_UNROLL);
+  lowbit_prepare_kernel<<<(unsigned)(center_ctas + sum_ctas), 256, 0, st>>>(center_ctas, qw.codes, qw.alpha, qw.beta, nblocks, qw.G,
+                                                                          w.ldg, w.beta_c, w.gam_h, w.gam_l, X, T, qw.d_in, w.s_h, w.s_l);
   count_launch();
   QB_CUDA(cudaGetLastError());
   const LowbitTerm lb{w.beta_c, w.gam_h, w.gam_l, w.s_h, w.s_l, w.ldg};
