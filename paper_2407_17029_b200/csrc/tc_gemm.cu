@@ -6,19 +6,19 @@
 //   forward : Y^T[o][t]  = sum_i w~[o][i] X[t][i]   + sum_k B[k][o/l2]      (s u)[t][k]
 //   backward: dX^T[i][t] = sum_o w~[o][i] dY[t][o]  + sum_k A[i/l1][k]      (du/l1)[t][k]
 //
-// Two CTAs on the two SMs of a TPC form a cluster and issue tcgen05.mma with cta_group::2: the
-// pair computes a 256 (weight rows) x 256 (tokens) tile.  Each CTA dequantizes its own 128 weight
-// rows into shared memory (the MMA's A operand, canonical 128-byte-swizzled layout: K-major in the
-// forward, MN-major in the backward, so the same [o][i]-packed codes serve both) and stages half of
-// the token tile by TMA (the B operand; no multicast), which halves the shared-memory traffic per
-// MMA cycle compared with a single-CTA tile -- the resource that bounds this kernel.  Accumulators
-// live in TMEM (2 x 256 columns, double-buffered so the epilogue of one tile overlaps the mainloop
-// of the next).
+// Two CTAs on the two SMs of a TPC form a cluster and issue tcgen05.mma with cta_group::2: one MMA covers
+// 256 weight rows x 256 tokens.  Each CTA dequantizes its own 128 weight rows into shared memory (the MMA's A
+// operand, canonical 128-byte-swizzled layout: K-major in the forward, MN-major in the backward, so the same
+// [o][i]-packed codes serve both) and stages its half of every 256-token group by TMA (the B operand; no
+// multicast).  Accumulators live in TMEM (2 x 256 columns).  Two tile shapes (Shape<NH>): 256 x 256 with the
+// two TMEM halves double-buffering the accumulator, and 256 x 512, where one dequantized weight stage feeds the
+// MMAs of two token groups -- half the dequantization work, shared-memory stores and ALU time per flop, which
+// is what bounds this kernel -- and the tile's epilogue runs on eight warps without a mainloop beside it.
 //
 // Warp roles: warp 0 TMA producer; warp 1 MMA issuer (leader CTA only) and TMEM owner; then the dequant
 // groups of four warps each, taking the K-blocks in turn (two groups in the forward, three in the backward;
-// those of the other CTA report each finished stage to the leader's barrier); the last four warps are the
-// epilogue.  Every mbarrier wait is bounded; on expiry the kernel stores QBLORA_ERR_TIMEOUT in the workspace
+// those of the other CTA report each finished stage to the leader's barrier); the last four (eight) warps are
+// the epilogue.  Every mbarrier wait is bounded; on expiry the kernel stores QBLORA_ERR_TIMEOUT in the workspace
 // status word and every role leaves its loop.
 #include <cuda.h>
 
@@ -36,15 +36,27 @@ using namespace ptx;
 namespace {
 
 constexpr int BM = 128;        // rows of the weight-side operand per CTA (256 per CTA pair)
-constexpr int BN = 256;        // tokens per tile (each CTA of the pair stages 128 of them)
+constexpr int BN = 256;        // tokens per MMA (each CTA of the pair stages 128 of them)
 constexpr int BN_HALF = BN / 2;
 constexpr int BK = 64;         // contraction elements per stage = one quantization block
-constexpr int STAGES = 6;
 constexpr int A_BYTES = BM * BK * 2;        // 16 KB dequantized weight tile
-constexpr int B_BYTES = BN_HALF * BK * 2;   // 16 KB: this CTA's half of the token tile
+constexpr int BH_BYTES = BN_HALF * BK * 2;  // 16 KB: this CTA's half of one 256-token group
 constexpr int P_BYTES = BM * BK / 2;        // 4 KB packed codes
-constexpr int SMEM_BYTES = STAGES * (A_BYTES + B_BYTES + P_BYTES) + 512 + 1024;
-static_assert(SMEM_BYTES <= 227 * 1024, "shared memory of the fused contraction");
+
+// Tile shape.  NH = 1: a 256 x 256 tile per CTA pair, the two halves of tensor memory double-buffer the
+// accumulator (the epilogue of one tile overlaps the mainloop of the next).  NH = 2: a 256 x 512 tile, both
+// halves of tensor memory hold the one tile's accumulators and every dequantized weight stage feeds two MMA
+// groups (tokens [0, 256) and [256, 512) of the tile), which halves the dequantization work, its shared-memory
+// stores and its ALU time per flop; the price is an epilogue that no longer overlaps a mainloop (eight
+// epilogue warps drain both halves at once) and coarser tiles.  The host picks per launch (tile_halves()).
+template <int NH>
+struct Shape {
+  static constexpr int STAGES = NH == 2 ? 4 : 6;
+  static constexpr int TILE_N = NH * BN;
+  static constexpr int B_BYTES = NH * BH_BYTES;
+  static constexpr int SMEM_BYTES = STAGES * (A_BYTES + B_BYTES + P_BYTES) + 512 + 1024;
+};
+static_assert(Shape<1>::SMEM_BYTES <= 227 * 1024 && Shape<2>::SMEM_BYTES <= 227 * 1024, "shared memory of the fused contraction");
 
 // Warp roles.  Dequant groups of 128 threads take the K-blocks in turn (group g: index % NG == g).  The forward
 // runs two groups; the backward three: its scale loads touch a new row of alpha / beta in every K-block (the
@@ -52,11 +64,11 @@ static_assert(SMEM_BYTES <= 227 * 1024, "shared memory of the fused contraction"
 // them could not keep the tensor pipe fed (C4 shapes, kernel alone: backward 950 -> 1100 TFLOP/s with three
 // groups and the scales of a group's next K-block loaded one K-block ahead; the forward measured the same with
 // two or three groups and slower with the early load).
-template <int MODE>
+template <int MODE, int NH>
 struct Roles {
   static constexpr int NG = MODE == 0 ? 2 : 3;
-  static constexpr int EPI_WARP0 = 2 + 4 * NG;            // four epilogue warps behind the dequant warps
-  static constexpr int NUM_THREADS = (EPI_WARP0 + 4) * 32;
+  static constexpr int EPI_WARP0 = 2 + 4 * NG;            // the epilogue warps (four per accumulator half in use at once) come last
+  static constexpr int NUM_THREADS = (EPI_WARP0 + 4 * NH) * 32;
   static constexpr bool SCALES_AHEAD = MODE == 1;
 };
 
@@ -150,12 +162,13 @@ __device__ __forceinline__ void dequant_direct8(uint32_t w, int word, const floa
   for (int e = 0; e < 4; ++e) o[e] = pack_bf16x2(v[2 * e], v[2 * e + 1]);
 }
 
-template <int MODE>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(Roles<MODE>::NUM_THREADS, 1)
+template <int MODE, int NH>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(Roles<MODE, NH>::NUM_THREADS, 1)
 tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ CUtensorMap tm_bx,
                   const __grid_constant__ CUtensorMap tm_p, const __grid_constant__ CUtensorMap tm_s,
                   const __grid_constant__ CUtensorMap tm_sl, const __grid_constant__ TcParams p) {
-  constexpr int NG = Roles<MODE>::NG, EPI_WARP0 = Roles<MODE>::EPI_WARP0;
+  constexpr int NG = Roles<MODE, NH>::NG, EPI_WARP0 = Roles<MODE, NH>::EPI_WARP0;
+  constexpr int STAGES = Shape<NH>::STAGES, B_BYTES = Shape<NH>::B_BYTES, TILE_N = Shape<NH>::TILE_N;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -204,17 +217,21 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
       bool adapter_input_ready = false;
       for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
         const int m0 = (tile % p.m_tiles) * (2 * BM) + (int)rank * BM;
-        const int t0 = (tile / p.m_tiles) * BN + (int)rank * BN_HALF;
+        const int tt0 = (tile / p.m_tiles) * TILE_N;            // first token of the tile
+        const int t0 = tt0 + (int)rank * BN_HALF;               // this CTA's 128 tokens of the first 256-token group
+        const bool two = NH == 2 && tt0 + BN < p.T;             // the tile's second 256-token group holds tokens
+        const uint32_t b_bytes = two ? 2 * BH_BYTES : BH_BYTES;
         for (int kb = 0; kb < kb_total; ++kb, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1u;
           if (!mbar_wait(empty(s), ph ^ 1u, p.status, p.wait_limit)) { ok = false; break; }
           if (kb < p.kb_base) {
-            mbar_arrive_expect_tx(full(s), B_BYTES + P_BYTES);
+            mbar_arrive_expect_tx(full(s), b_bytes + P_BYTES);
             // test hook (qblora_debug_drop_load): the bytes are announced and never sent, so this stage's
             // barrier cannot complete and every role has to run into its wait limit and leave by itself
             if ((int)it != p.drop_load) {
               tma_load_2d(sB + s * B_BYTES, &tm_b, full(s), kb * BK, t0);
+              if (two) tma_load_2d(sB + s * B_BYTES + BH_BYTES, &tm_b, full(s), kb * BK, t0 + BN);
               if (MODE == 0) {
                 tma_load_2d(sP + s * P_BYTES, &tm_p, full(s), kb * (BK / 2), m0);
               } else {   // two boxes of 64 rows x 32 bytes: packed[ng][k][32 B]
@@ -230,12 +247,14 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
               asm volatile("griddepcontrol.wait;" ::: "memory");
               adapter_input_ready = true;
             }
-            mbar_arrive_expect_tx(full(s), B_BYTES);
+            mbar_arrive_expect_tx(full(s), b_bytes);
             if (kb < kb_gamma0) {
               tma_load_2d(sB + s * B_BYTES, &tm_bx, full(s), (kb - p.kb_base) * BK, t0);
+              if (two) tma_load_2d(sB + s * B_BYTES + BH_BYTES, &tm_bx, full(s), (kb - p.kb_base) * BK, t0 + BN);
             } else {   // group sums of x: hi for the first two segments, lo for the third
               const int kg = kb - kb_gamma0, seg = kg / p.ng_blocks, blk = kg - seg * p.ng_blocks;
               tma_load_2d(sB + s * B_BYTES, seg == 2 ? &tm_sl : &tm_s, full(s), blk * BK, t0);
+              if (two) tma_load_2d(sB + s * B_BYTES + BH_BYTES, seg == 2 ? &tm_sl : &tm_s, full(s), blk * BK, t0 + BN);
             }
           }
         }
@@ -263,11 +282,16 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
       int lt = 0, s = 0;
       uint32_t ph = 0;
       for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters, ++lt) {
-        const int a = lt & 1;
-        const uint32_t aph = (lt >> 1) & 1u;
+        // NH == 1: the tile's accumulator is half (lt & 1) of tensor memory, used every other tile.  NH == 2: the
+        // tile's two 256-token groups take both halves, every tile (a half without tokens gets no MMAs but still
+        // goes through its full / empty hand-over, so the phases stay in step).
+        const int a = NH == 2 ? 0 : (lt & 1);
+        const uint32_t aph = NH == 2 ? (lt & 1u) : ((lt >> 1) & 1u);
         if (!mbar_wait(accempty(a), aph ^ 1u, p.status, p.wait_limit)) { ok = false; break; }
+        if (NH == 2 && !mbar_wait(accempty(1), aph ^ 1u, p.status, p.wait_limit)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(a * BN);
+        const bool two = NH == 2 && (tile / p.m_tiles) * TILE_N + BN < p.T;
         uint32_t acc = 0;   // the first MMA of a tile overwrites the accumulator
         // weight K-blocks [0, kb_base): K-major tile in the forward, MN-major in the backward; adapter K-blocks
         // [kb_base, kb_gamma0): the other way round (see the dequant warps); offset-term K-blocks: K-major
@@ -284,15 +308,22 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
             const uint64_t adesc = dhi_a | (uint64_t)(a_lo0 + (uint32_t)s * (A_BYTES >> 4));
             const uint64_t bdesc = dhi_k | (uint64_t)(b_lo0 + (uint32_t)s * (B_BYTES >> 4));
 #pragma unroll
-            for (int k = 0; k < BK / 16; ++k) {
-              tc_mma_pair(d_tmem, adesc + (uint64_t)(k * a_step), bdesc + (uint64_t)(k * 2), idesc, acc);
-              acc = 1u;
+            for (int k = 0; k < BK / 16; ++k)
+              tc_mma_pair(d_tmem, adesc + (uint64_t)(k * a_step), bdesc + (uint64_t)(k * 2), idesc, k == 0 ? acc : 1u);
+            if (two) {   // the same weight stage against the tile's second token group
+#pragma unroll
+              for (int k = 0; k < BK / 16; ++k)
+                tc_mma_pair(d_tmem + BN, adesc + (uint64_t)(k * a_step), bdesc + (uint64_t)((BH_BYTES >> 4) + k * 2), idesc, k == 0 ? acc : 1u);
             }
+            acc = 1u;
             tc_commit_pair(empty(s));
             if (++s == STAGES) { s = 0; ph ^= 1u; }
           }
         }
-        if (ok) tc_commit_pair(accfull(a));
+        if (ok) {
+          tc_commit_pair(accfull(a));
+          if (NH == 2) tc_commit_pair(accfull(1));
+        }
       }
     }
   } else if (warp < EPI_WARP0) {
@@ -377,7 +408,7 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
         } else if (kb < p.kb_base) {
           float al, be;
           if (have_next) { al = al_next; be = be_next; } else load_scale(kb, al, be);
-          have_next = Roles<MODE>::SCALES_AHEAD && kb + NG < p.kb_base;
+          have_next = Roles<MODE, NH>::SCALES_AHEAD && kb + NG < p.kb_base;
           if (have_next) load_scale(kb + NG, al_next, be_next);
           BlockTable tab;
           tab.build(p.level, al, be);
@@ -495,14 +526,15 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
   } else {
     // ------------------------------------------------------------------ epilogue warps (128 threads)
     const int q = warp & 3;                       // TMEM lane quadrant this warp may read
+    const int h = NH == 2 ? (warp - EPI_WARP0) >> 2 : 0;   // NH == 2: which 256-token group of the tile this warp drains
     const uint32_t leader_accempty0 = map_to_cta(accempty(0), 0), leader_accempty1 = map_to_cta(accempty(1), 0);
     bool ok = true;
     int lt = 0;
     for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters, ++lt) {
-      const int a = lt & 1;
-      const uint32_t aph = (lt >> 1) & 1u;
+      const int a = NH == 2 ? h : (lt & 1);
+      const uint32_t aph = NH == 2 ? (lt & 1u) : ((lt >> 1) & 1u);
       const int m = (tile % p.m_tiles) * (2 * BM) + (int)rank * BM + q * 32 + lane;
-      const int t0 = (tile / p.m_tiles) * BN;
+      const int t0 = (tile / p.m_tiles) * TILE_N + h * BN;
       if (!mbar_wait(accfull(a), aph, p.status, p.wait_limit)) { ok = false; break; }
       tc_fence_after();
       for (int c = 0; c < BN / 32; ++c) {
@@ -782,30 +814,47 @@ struct LowbitTerm {
   int ldg;
 };
 
+// Tile shape of a launch (Shape<NH>): 512-token tiles when the problem has more than one 256-token group and the
+// coarser tiles do not cost more in idle CTA pairs of the last round than they save per tile.  A 512-token tile
+// is costed at kWideTileCost 256-token tiles.  QBLORA_TILE_HALVES=1|2 forces a shape (for A/B timing).
+constexpr double kWideTileCost = 1.5;
+int tile_halves(int m_tiles, int64_t T, int pairs) {
+  static const int forced = []() { const char* v = getenv("QBLORA_TILE_HALVES"); return v ? atoi(v) : 0; }();
+  if (T <= BN) return 1;
+  if (forced == 1 || forced == 2) return forced;
+  const int64_t tiles1 = (int64_t)m_tiles * ((T + BN - 1) / BN), tiles2 = (int64_t)m_tiles * ((T + 2 * BN - 1) / (2 * BN));
+  const double cost1 = (double)((tiles1 + pairs - 1) / pairs), cost2 = kWideTileCost * (double)((tiles2 + pairs - 1) / pairs);
+  return cost2 <= cost1 ? 2 : 1;
+}
+
 int launch_main(int mode, const QwView& qw, const AdView* ad, const __nv_bfloat16* Bop, const __nv_bfloat16* Bx,
                 int ldx, int64_t T, void* out, int out_dtype, int* status, cudaStream_t st,
                 const LowbitTerm* lb = nullptr) {
   // the shared-memory opt-in is a per-device function attribute: set once per device and kernel (the flags are
   // atomic, so concurrent host threads at worst set it twice)
-  static std::atomic<bool> attr_set[64][2];
+  static std::atomic<bool> attr_set[64][2][2];
   int dev = 0;
   QB_CUDA(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64) return QBLORA_ERR_UNSUPPORTED;
-  if (!attr_set[dev][mode].load(std::memory_order_acquire)) {
-    cudaError_t e = mode == 0
-        ? cudaFuncSetAttribute(tc_dq_gemm_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES)
-        : cudaFuncSetAttribute(tc_dq_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-    if (e != cudaSuccess) return QBLORA_ERR_CUDA;
-    attr_set[dev][mode].store(true, std::memory_order_release);
-  }
   TcParams p{};
   p.M = mode == 0 ? qw.d_out : qw.d_in;
   const int Kq = mode == 0 ? qw.d_in : qw.d_out;
+  const int pairs = num_sms() / 2;
+  const int nh = tile_halves((p.M + 2 * BM - 1) / (2 * BM), T, pairs);
+  const void* kernel = mode == 0 ? (nh == 2 ? (const void*)tc_dq_gemm_kernel<0, 2> : (const void*)tc_dq_gemm_kernel<0, 1>)
+                                 : (nh == 2 ? (const void*)tc_dq_gemm_kernel<1, 2> : (const void*)tc_dq_gemm_kernel<1, 1>);
+  const int smem_bytes = nh == 2 ? Shape<2>::SMEM_BYTES : Shape<1>::SMEM_BYTES;
+  const int threads = mode == 0 ? (nh == 2 ? Roles<0, 2>::NUM_THREADS : Roles<0, 1>::NUM_THREADS)
+                                : (nh == 2 ? Roles<1, 2>::NUM_THREADS : Roles<1, 1>::NUM_THREADS);
+  if (!attr_set[dev][mode][nh - 1].load(std::memory_order_acquire)) {
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess) return QBLORA_ERR_CUDA;
+    attr_set[dev][mode][nh - 1].store(true, std::memory_order_release);
+  }
   p.kb_base = (Kq + BK - 1) / BK;
   p.kb_extra = ad ? (ad->r + BK - 1) / BK : 0;
   p.T = (int)T;
   p.m_tiles = (p.M + 2 * BM - 1) / (2 * BM);
-  p.n_tiles = (int)((T + BN - 1) / BN);
+  p.n_tiles = (int)((T + nh * BN - 1) / (nh * BN));
   p.d_in = qw.d_in; p.d_out = qw.d_out; p.G = qw.G;
   p.block_in = qw.block_in; p.block_out = qw.block_out;
   p.direct = qw.block_in != BK ? 1 : 0;   // (for 64 x 1 blocks the table is faster: 883 vs 702 TFLOP/s on the C5 up shape)
@@ -846,14 +895,13 @@ int launch_main(int mode, const QwView& qw, const AdView* ad, const __nv_bfloat1
   }
 
   const int tiles = p.m_tiles * p.n_tiles;                      // one tile per CTA pair
-  const int pairs = num_sms() / 2;
   const int grid = 2 * (tiles < pairs ? tiles : pairs);
   // With an adapter the kernel in front of this one on the stream is the small product that writes Bx, and only
   // the last K-blocks of a tile read it: launch as its programmatic dependent, so that the weight K-blocks run
   // while that product finishes (the producer warp waits for it before the first adapter K-block).  Without an
   // adapter the predecessor is the caller's own work and the launch is an ordinary one.
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(mode == 0 ? Roles<0>::NUM_THREADS : Roles<1>::NUM_THREADS); cfg.dynamicSmemBytes = SMEM_BYTES; cfg.stream = st;
+  cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3((unsigned)threads); cfg.dynamicSmemBytes = (size_t)smem_bytes; cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -861,8 +909,8 @@ int launch_main(int mode, const QwView& qw, const AdView* ad, const __nv_bfloat1
   cudaError_t le;
   {
     DominantKernelTimer timer(st);
-    le = mode == 0 ? cudaLaunchKernelEx(&cfg, tc_dq_gemm_kernel<0>, tm_b, tm_bx, tm_p, tm_s, tm_sl, p)
-                   : cudaLaunchKernelEx(&cfg, tc_dq_gemm_kernel<1>, tm_b, tm_bx, tm_p, tm_s, tm_sl, p);
+    void* args[6] = {&tm_b, &tm_bx, &tm_p, &tm_s, &tm_sl, &p};
+    le = cudaLaunchKernelExC(&cfg, kernel, args);
     count_launch();
   }
   QB_CUDA(le);
