@@ -358,10 +358,12 @@ def measure_workload(ctx, wl, geom, steps, warmup, min_region_s, no_graph=False,
     if not want_e2e:
         return res
 
-    # ---- end to end: host (pinned) inputs in, results out, copies inside the timed region.  Up to three lanes
-    # (stream + device buffer set + pinned host buffers each) take the steps in turn, so the copies of
-    # one step overlap the other's compute and opposite-direction copies; every step still moves all of
-    # its inputs and results.
+    # ---- end to end: host (pinned) inputs in, results out, copies inside the timed region.  Three streams form
+    # a pipeline over the linears of a step -- one issues the host-to-device copies, one the library calls, one
+    # the device-to-host copies -- tied together per linear by events, so that the two copy directions (separate
+    # copy engines, full-duplex link) and the compute overlap; the steps alternate between the device buffer sets,
+    # and a buffer is written again only after its previous reader is done.  Every step still moves all of its
+    # inputs and results.
     lanes = []
     h2d = d2h = 0
     lane_bytes = sum((X.numel() + dY.numel() + Y.numel() + dX.numel()) * 2 for _, _, _, X, dY, Y, dX, *_ in sets[0])
@@ -372,21 +374,31 @@ def measure_workload(ctx, wl, geom, steps, warmup, min_region_s, no_graph=False,
             hX, hdY = X.cpu().pin_memory(), dY.cpu().pin_memory()
             hY, hdX = torch.empty_like(Y, device="cpu").pin_memory(), torch.empty_like(dX, device="cpu").pin_memory()
             hdA, hdB = torch.empty_like(dA, device="cpu").pin_memory(), torch.empty_like(dB, device="cpu").pin_memory()
-            host.append((hX, hdY, hY, hdX, hdA, hdB))
+            ev = tuple(torch.cuda.Event() for _ in range(3))                # inputs landed / calls done / results copied out
+            host.append((hX, hdY, hY, hdX, hdA, hdB, ev))
             if li_ == 0:
                 h2d += hX.numel() * 2 + hdY.numel() * 2
                 d2h += hY.numel() * 2 + hdX.numel() * 2 + hdA.numel() * 4 + hdB.numel() * 4
-        lanes.append((torch.cuda.Stream(), sets[li_], host))
+        lanes.append((sets[li_], host))
+    s_in, s_run, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
 
     def e2e_step(i=0):
-        stream, items, host = lanes[i % n_lanes]
-        with torch.cuda.stream(stream):
-            for (spec, q2, ad, X, dY, Y, dX, dA, dB, wsf, wsb), (hX, hdY, hY, hdX, hdA, hdB) in zip(items, host):
+        items, host = lanes[i % n_lanes]
+        for (spec, q2, ad, X, dY, Y, dX, dA, dB, wsf, wsb), (hX, hdY, hY, hdX, hdA, hdB, (ev_in, ev_run, ev_out)) in zip(items, host):
+            with torch.cuda.stream(s_in):
+                s_in.wait_event(ev_run)                  # the previous calls on this buffer set have read X and dY
                 X.copy_(hX, non_blocking=True); dY.copy_(hdY, non_blocking=True)
+                ev_in.record(s_in)
+            with torch.cuda.stream(s_run):
+                s_run.wait_event(ev_in); s_run.wait_event(ev_out)   # inputs are here; the previous results are out
                 qb.linear_fwd(q2, ad, X, ws=wsf, out=Y)
                 qb.linear_bwd(q2, ad, X, dY, ws=wsb, outs=(dX, dA, dB))
+                ev_run.record(s_run)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_run)
                 hY.copy_(Y, non_blocking=True); hdX.copy_(dX, non_blocking=True)
                 hdA.copy_(dA, non_blocking=True); hdB.copy_(dB, non_blocking=True)
+                ev_out.record(s_out)
 
     e2e_steps = max(3, min(steps, 10))
     for i in range(n_lanes):
@@ -398,7 +410,8 @@ def measure_workload(ctx, wl, geom, steps, warmup, min_region_s, no_graph=False,
     ctx.barrier()
     e2e_s = ctx.max_over_ranks(time.perf_counter() - t0)
     res["e2e"] = {"value": flops_step * ctx.world * e2e_steps / e2e_s / 1e12, "unit": "TFLOP/s",
-                  "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps, "lanes": n_lanes}
+                  "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps, "lanes": n_lanes,
+                  "pipeline": "copy-in, compute and copy-out streams, chained per linear by events"}
     return res
 
 

@@ -232,6 +232,23 @@ def test_linear_bwd_parity(qb, path, case, qfmt, visible):
     assert torch.equal(dA, dA2) and torch.equal(dB, dB2)
 
 
+@pytest.mark.parametrize("d_out,d_in", [(4864, 128), (128, 4864)])
+def test_wide_tiles_several_rounds_and_ragged_tokens(qb, d_out, d_in):
+    # 19 row tiles x 5 token positions of 512 = 95 tiles on 74 CTA pairs (two rounds); T = 2100 leaves 52 tokens
+    # in the last position, so its tiles have an empty second half.  (4864, 128) lays the forward's rows out this
+    # way, (128, 4864) the backward's.
+    T = 2100
+    qw, ad, X, dY = make_case(47, T, d_out, d_in, 64, 8, 16, 1)
+    Wt = oracle.dequantize(qw)
+    dq, da, Xd, dYd = qweight_to_dev(qw), adapter_to_dev(ad), to_bf16_dev(X), to_bf16_dev(dY)
+    gate_strict(to_np64(g_linear_fwd(dq, da, Xd, torch.float32)), oracle.linear_fwd(Wt, ad, X), "Y f32")
+    rdX, rdA, rdB = oracle.linear_bwd(Wt, ad, X, dY)
+    dX, dA, dB = g_linear_bwd(dq, da, Xd, dYd, torch.float32)
+    gate_strict(to_np64(dX), rdX, "dX f32")
+    gate_strict(to_np64(dA), rdA, "dA", per_row=False)
+    gate_strict(to_np64(dB), rdB, "dB", per_row=False)
+
+
 def test_zero_B_is_bit_identical_to_no_adapter(qb, path):
     qw, ad, X, dY = make_case(43, 300, 320, 448, 64, 8, 48)
     ad.B = np.zeros_like(ad.B)
