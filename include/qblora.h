@@ -169,9 +169,14 @@ int qblora_set_timing_events(void* start_event, void* stop_event);
  *   its `iteration`-th weight K-block to the stage's barrier but issues no copy, so that barrier never
  *   completes: every role of the kernel runs into its wait limit, the kernel stores QBLORA_ERR_TIMEOUT in the
  *   status word, releases its tensor memory and returns by itself; the outputs of that call are undefined.
- *   Negative = disarm.  Use together with a short wait limit. */
+ *   Negative = disarm.  Use together with a short wait limit.
+ * qblora_debug_hold_producer(cycles): in the NEXT launch of the fused dequant contraction with an adapter, the
+ *   producer of every CTA idles for `cycles` SM clock cycles (at most 10^8, about 50 ms) in front of the first
+ *   adapter K-block of its first tile -- what a long wait for the adapter's compressed activation looks like to
+ *   the other roles of the kernel.  The results must not change.  0 = disarm. */
 int qblora_debug_set_wait_limit(int64_t cycles);
 int qblora_debug_drop_load(int32_t iteration);
+int qblora_debug_hold_producer(int64_t cycles);
 
 /*
  * Block-wise 4-bit quantization, Eq. 1 (Sec. 3.1).

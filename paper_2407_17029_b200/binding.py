@@ -31,7 +31,7 @@ EXPORTS = ["qblora_default_code_table", "qblora_workspace_bytes", "qblora_status
            "qblora_device_status", "qblora_quantize_blockwise", "qblora_linear_fwd",
            "qblora_linear_bwd", "qablora_merge", "qablora_lowbit_gemm", "qblora_kernel_launches",
            "qblora_set_timing_events", "qablora_merge_noalloc", "qblora_merge_dense",
-           "qblora_quantize_minmax_nbit", "qblora_debug_set_wait_limit", "qblora_debug_drop_load", "qblora_dense_gemm", "qblora_pack_codes", "qblora_unpack_codes"]
+           "qblora_quantize_minmax_nbit", "qblora_debug_set_wait_limit", "qblora_debug_drop_load", "qblora_debug_hold_producer", "qblora_dense_gemm", "qblora_pack_codes", "qblora_unpack_codes"]
 
 
 class _CQWeight(ctypes.Structure):
@@ -90,6 +90,7 @@ _lib.qblora_pack_codes.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int
 _lib.qblora_unpack_codes.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]
 _lib.qblora_debug_set_wait_limit.argtypes = [ctypes.c_int64]
 _lib.qblora_debug_drop_load.argtypes = [ctypes.c_int32]
+_lib.qblora_debug_hold_producer.argtypes = [ctypes.c_int64]
 
 
 def kernel_launches() -> int:
@@ -112,6 +113,12 @@ def debug_set_wait_limit(cycles: int) -> None:
 def debug_drop_load(iteration: int) -> None:
     """Test hook: the next fused-contraction launch leaves out one weight load (see the header); negative = disarm."""
     _check_plain(_lib.qblora_debug_drop_load(int(iteration)))
+
+
+def debug_hold_producer(cycles: int) -> None:
+    """Test hook: the producers of the next adapted fused-contraction launch idle `cycles` cycles before their
+    first adapter K-block (see the header); 0 = disarm."""
+    _check_plain(_lib.qblora_debug_hold_producer(int(cycles)))
 
 
 def _check_plain(status: int):

@@ -54,6 +54,8 @@ constexpr long long kDefaultWaitLimitCycles = 2000000000LL;
 long long wait_limit_cycles();
 // Test hook armed by qblora_debug_drop_load: returns the armed producer iteration once (then -1 again).
 int take_dropped_load();
+// Test hook armed by qblora_debug_hold_producer: returns the armed number of cycles once (then 0 again).
+long long take_producer_hold();
 // Brackets the dominant kernel of a call with the armed event pair (if any), then disarms.
 struct DominantKernelTimer {
   cudaStream_t st; cudaEvent_t stop;

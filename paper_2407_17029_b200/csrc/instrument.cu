@@ -11,6 +11,7 @@ thread_local cudaEvent_t t_start = nullptr;
 thread_local cudaEvent_t t_stop = nullptr;
 std::atomic<long long> g_wait_limit{0};   // 0 = default
 std::atomic<int> g_drop_load{-1};
+std::atomic<long long> g_hold_producer{0};
 }  // namespace
 
 long long wait_limit_cycles() {
@@ -18,6 +19,7 @@ long long wait_limit_cycles() {
   return v > 0 ? v : kDefaultWaitLimitCycles;
 }
 int take_dropped_load() { return g_drop_load.exchange(-1, std::memory_order_relaxed); }
+long long take_producer_hold() { return g_hold_producer.exchange(0, std::memory_order_relaxed); }
 
 void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 
@@ -40,6 +42,11 @@ int qblora_debug_set_wait_limit(int64_t cycles) {
 }
 int qblora_debug_drop_load(int32_t iteration) {
   qb::g_drop_load.store(iteration < 0 ? -1 : (int)iteration, std::memory_order_relaxed);
+  return QBLORA_OK;
+}
+int qblora_debug_hold_producer(int64_t cycles) {
+  if (cycles < 0 || cycles > 100000000) return QBLORA_ERR_INVALID_ARG;
+  qb::g_hold_producer.store((long long)cycles, std::memory_order_relaxed);
   return QBLORA_OK;
 }
 int qblora_set_timing_events(void* start_event, void* stop_event) {

@@ -98,6 +98,7 @@ struct TcParams {
   int* status;
   long long wait_limit;     // cycles after which a device-side wait gives up
   int drop_load;            // test hook: the producers leave out the loads of this K-block iteration (-1: none)
+  long long hold_producer;  // test hook: the producers idle this many cycles in front of their first adapter K-block
 };
 
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
@@ -246,6 +247,8 @@ tc_dq_gemm_kernel(const __grid_constant__ CUtensorMap tm_b, const __grid_constan
             if (!adapter_input_ready) {
               asm volatile("griddepcontrol.wait;" ::: "memory");
               adapter_input_ready = true;
+              // test hook (qblora_debug_hold_producer): as if that wait had taken this much longer
+              if (p.hold_producer > 0) { const long long h0 = clock64(); while (clock64() - h0 < p.hold_producer) {} }
             }
             mbar_arrive_expect_tx(full(s), b_bytes);
             if (kb < kb_gamma0) {
@@ -882,6 +885,7 @@ int launch_main(int mode, const QwView& qw, const AdView* ad, const __nv_bfloat1
   p.out = out; p.out_dtype = out_dtype; p.status = status;
   p.wait_limit = wait_limit_cycles();
   p.drop_load = take_dropped_load();
+  p.hold_producer = ad ? take_producer_hold() : 0;
   if (lb) {
     p.beta = lb->beta_c;
     p.ng_blocks = (qw.G + BK - 1) / BK;
@@ -956,24 +960,6 @@ int launch_u_gemm(const AdView& ad, int64_t T, const TcWs& w, const SgOut& out, 
   return small_gemm((int)T, ad.r, segs, 2, out, status, st, nullptr, overlap_adapter_prologue(), before_contraction);
 }
 
-// Compression and first adapter product in one launch (tc_segsum_gemm.cu) where the pooling window allows it:
-// x' = AvgPool(X) and u = x' A (forward, and the backward's gradient chain), dv and du = dv B^T (backward).
-// Off unless QBLORA_FUSED_COMPRESS=1: as it stands the one launch is slower than the two it replaces.
-bool fused_compress(const AdView& ad, int width, int lam) {
-  static const bool off = []() { const char* v = getenv("QBLORA_FUSED_COMPRESS"); return !(v && v[0] == '1'); }();
-  return !off && ad.op == QBLORA_SCALE_AVGPOOL_REPEAT && segsum_gemm_ok(width, lam, ad.r);
-}
-// u = AvgPool(X) A: `out` as for launch_u_gemm; keep_x also stores x' (hi / lo) for the dA product
-int launch_pool_u(const QwView& qw, const AdView& ad, const __nv_bfloat16* X, int64_t T, const TcWs& w, const SgOut& out,
-                  bool keep_x, int* status, cudaStream_t st) {
-  SegGemm g{};
-  g.src = X; g.T = T; g.width = qw.d_in; g.lam = ad.l1; g.divide = true; g.scale = 1.0f;
-  g.m = SgOperand{ad.A, ad.r, false}; g.N = ad.r;
-  g.c_hi = keep_x ? w.xh : nullptr; g.c_lo = keep_x ? w.xl : nullptr; g.ld_c = w.ldp;
-  g.out = out;
-  return segsum_gemm(g, status, st);
-}
-
 }  // namespace
 
 bool tc_supported(const QwView& qw, const AdView* ad, int64_t T) {
@@ -994,17 +980,12 @@ int tc_linear_fwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, in
   TcWs w = carve(QBLORA_OP_LINEAR_FWD, ad, T, ws);
   int* status = reinterpret_cast<int*>(ws);
   if (ad) {
+    int rc = launch_pool(qw, *ad, X, T, w, st);
+    if (rc) return rc;
     // u16 = bf16(s * x' A): the scaling rides on the compressed activation, B stays exact
     SgOut out{};
     out.scaled = w.u16; out.ld16 = w.ldr; out.scale = ad->s; out.divide = false;
-    int rc;
-    if (fused_compress(*ad, qw.d_in, ad->l1)) {
-      rc = launch_pool_u(qw, *ad, X, T, w, out, false, status, st);
-    } else {
-      rc = launch_pool(qw, *ad, X, T, w, st);
-      if (rc) return rc;
-      rc = launch_u_gemm(*ad, T, w, out, status, st, true);
-    }
+    rc = launch_u_gemm(*ad, T, w, out, status, st, true);
     if (rc) return rc;
   }
   return launch_main(0, qw, ad, X, w.u16, w.ldr, T, Y, y_dtype, status, st);
@@ -1104,56 +1085,37 @@ int tc_linear_bwd(const QwView& qw, const AdView* ad, const __nv_bfloat16* X, co
   // whatever happens below, it is joined back into the caller's stream before the call returns.
   const int rc = [&]() -> int {
     int rc;
-    const float du_div = ad->op == QBLORA_SCALE_AVGPOOL_REPEAT ? (float)ad->l1 : 1.0f;   // only the average carries 1 / lambda_in
-    if (fused_compress(*ad, qw.d_out, ad->l2)) {
-      // dv, du = dv B^T (hi + lo for dA) and du16 = bf16(du / lambda_in) for the dX contraction, in one launch
-      SegGemm g{};
-      g.src = dY; g.T = T; g.width = qw.d_out; g.lam = ad->l2; g.divide = false; g.scale = ad->s;
-      g.m = SgOperand{ad->B, ad->Q, true}; g.N = ad->r;
-      g.c_hi = w.dvh; g.c_lo = w.dvl; g.ld_c = w.ldq;
-      g.out.hi = w.duh; g.out.lo = w.dul; g.out.scaled = w.du16; g.out.ld16 = w.ldr; g.out.divide = true; g.out.scale = du_div;
-      rc = segsum_gemm(g, status, st);
-      if (rc) return rc;
+    const int64_t n = T * ad->Q;
+    if (ad->op != QBLORA_SCALE_AVGPOOL_REPEAT) {
+      sample_split_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(
+          dY, T, qw.d_out, ad->Q, ad->op == QBLORA_SCALE_TRUNCATE_ZEROPAD ? 1 : ad->l2, ad->s, w.ldq, w.dvh, w.dvl);
+    } else if (segsum_fast_ok(qw.d_out, ad->l2)) {
+      const int64_t chunks = T * (qw.d_out / 8);
+      segsum_split_kernel<false><<<(unsigned)((chunks + 256 * SEGSUM_UNROLL - 1) / (256 * SEGSUM_UNROLL)), 256, 0, st>>>(dY, T, qw.d_out, ad->l2, ad->s, w.ldq, w.dvh, w.dvl);
     } else {
-      const int64_t n = T * ad->Q;
-      if (ad->op != QBLORA_SCALE_AVGPOOL_REPEAT) {
-        sample_split_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(
-            dY, T, qw.d_out, ad->Q, ad->op == QBLORA_SCALE_TRUNCATE_ZEROPAD ? 1 : ad->l2, ad->s, w.ldq, w.dvh, w.dvl);
-      } else if (segsum_fast_ok(qw.d_out, ad->l2)) {
-        const int64_t chunks = T * (qw.d_out / 8);
-        segsum_split_kernel<false><<<(unsigned)((chunks + 256 * SEGSUM_UNROLL - 1) / (256 * SEGSUM_UNROLL)), 256, 0, st>>>(dY, T, qw.d_out, ad->l2, ad->s, w.ldq, w.dvh, w.dvl);
-      } else {
-        dv_split_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(dY, T, qw.d_out, ad->l2, ad->s, w.ldq, w.dvh, w.dvl);
-      }
-      count_launch();
-      QB_CUDA(cudaGetLastError());
-      {  // du = dv B^T (hi + lo for dA) and du16 = bf16(du / lambda_in) for the dX contraction
-        const SgOperand b_mat{ad->B, ad->Q, true};   // (n = rank index, k = q) at B[n * Q + k]
-        SgSegment segs[2] = {{{w.dvh, w.ldq, true}, b_mat, ad->Q}, {{w.dvl, w.ldq, true}, b_mat, ad->Q}};
-        SgOut out{};
-        out.hi = w.duh; out.lo = w.dul; out.scaled = w.du16; out.ld16 = w.ldr; out.divide = true;
-        out.scale = du_div;
-        rc = small_gemm((int)T, ad->r, segs, 2, out, status, st, nullptr, overlap_adapter_prologue(), false);   // behind dv's kernel (narrow tiles: wide ones start the contraction earlier, which costs the gradient chain beside it more than it saves: C2 backward 115 vs 119 us)
-        if (rc) return rc;
-      }
+      dv_split_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(dY, T, qw.d_out, ad->l2, ad->s, w.ldq, w.dvh, w.dvl);
+    }
+    count_launch();
+    QB_CUDA(cudaGetLastError());
+    {  // du = dv B^T (hi + lo for dA) and du16 = bf16(du / lambda_in) for the dX contraction
+      const SgOperand b_mat{ad->B, ad->Q, true};   // (n = rank index, k = q) at B[n * Q + k]
+      SgSegment segs[2] = {{{w.dvh, w.ldq, true}, b_mat, ad->Q}, {{w.dvl, w.ldq, true}, b_mat, ad->Q}};
+      SgOut out{};
+      out.hi = w.duh; out.lo = w.dul; out.scaled = w.du16; out.ld16 = w.ldr; out.divide = true;
+      out.scale = ad->op == QBLORA_SCALE_AVGPOOL_REPEAT ? (float)ad->l1 : 1.0f;   // only the average carries 1 / lambda_in
+      rc = small_gemm((int)T, ad->r, segs, 2, out, status, st, nullptr, overlap_adapter_prologue(), false);   // behind dv's kernel (narrow tiles: wide ones start the contraction earlier, which costs the gradient chain beside it more than it saves: C2 backward 115 vs 119 us)
+      if (rc) return rc;
     }
     if (lane) QB_CUDA(cudaEventRecord(lane->du_done, st));
-    if (dB && fused_compress(*ad, qw.d_in, ad->l1)) {   // x' (for dA) and u = x' A (for dB) in one launch
+    if (dA || dB) {
+      rc = launch_pool(qw, *ad, X, T, w, sb);
+      if (rc) return rc;
+    }
+    if (dB) {
       SgOut uo{};
       uo.hi = w.uh; uo.lo = w.ul; uo.ld16 = w.ldr;
-      rc = launch_pool_u(qw, *ad, X, T, w, uo, dA != nullptr, status, sb);
+      rc = launch_u_gemm(*ad, T, w, uo, status, sb, false);
       if (rc) return rc;
-    } else {
-      if (dA || dB) {
-        rc = launch_pool(qw, *ad, X, T, w, sb);
-        if (rc) return rc;
-      }
-      if (dB) {
-        SgOut uo{};
-        uo.hi = w.uh; uo.lo = w.ul; uo.ld16 = w.ldr;
-        rc = launch_u_gemm(*ad, T, w, uo, status, sb, false);
-        if (rc) return rc;
-      }
     }
     if (lane) QB_CUDA(cudaStreamWaitEvent(lane->stream, lane->du_done, 0));   // dv and du are complete
     if (dB) {

@@ -39,20 +39,6 @@ int small_gemm(int M, int N, const SgSegment* segs, int nseg, const SgOut& out, 
                float* partial = nullptr, bool dependent = false, bool wide_tiles = false);
 int small_gemm_splits(int M, int N, int K);
 
-// The adapter's first product with the compression of its input fused in front (tc_segsum_gemm.cu):
-//   c[t][w] = (sum of lam consecutive src[t][lam w ..]) / lam  (divide)  or  * scale;   out[t][n] = sum_w c[t][w] m(n, w)
-// with c taken as a bf16 hi + lo pair.  src bf16 [T][width]; m: the adapter matrix seen as (n, w), N rows;
-// c_hi / c_lo (both or neither): copy of c, [T][ld_c]; out: hi / lo / scaled only, [T][ld16].
-struct SegGemm {
-  const __nv_bfloat16* src; int64_t T; int width, lam;
-  bool divide; float scale;
-  SgOperand m; int N;
-  __nv_bfloat16 *c_hi, *c_lo; int64_t ld_c;
-  SgOut out;
-};
-bool segsum_gemm_ok(int width, int lam, int N);   // lam in {8, 16, 32, 64} dividing width, N <= 256 a multiple of 8
-int segsum_gemm(const SegGemm& a, int* status, cudaStream_t st);
-
 // Encodes a 2-D tensor map (shared with the main kernel's host code).
 int make_tensor_map_2d(void* tm, bool is_u8, const void* ptr, uint64_t inner, uint64_t rows, uint64_t pitch_bytes,
                        uint32_t box_inner, uint32_t box_rows, bool swizzle128);
