@@ -232,12 +232,11 @@ def test_linear_bwd_parity(qb, path, case, qfmt, visible):
     assert torch.equal(dA, dA2) and torch.equal(dB, dB2)
 
 
-@pytest.mark.parametrize("d_out,d_in", [(4864, 128), (128, 4864)])
-def test_wide_tiles_several_rounds_and_ragged_tokens(qb, d_out, d_in):
+@pytest.mark.parametrize("d_out,d_in,T", [(4864, 128, 2100), (128, 4864, 2100), (4864, 128, 2400)])
+def test_wide_tiles_several_rounds_and_ragged_tokens(qb, d_out, d_in, T):
     # 19 row tiles x 5 token positions of 512 = 95 tiles on 74 CTA pairs (two rounds); T = 2100 leaves 52 tokens
-    # in the last position, so its tiles have an empty second half.  (4864, 128) lays the forward's rows out this
-    # way, (128, 4864) the backward's.
-    T = 2100
+    # in the last position, so its tiles have an empty second half; T = 2400 leaves 352, a second half with 96
+    # tokens.  (4864, 128) lays the forward's rows out this way, (128, 4864) the backward's.
     qw, ad, X, dY = make_case(47, T, d_out, d_in, 64, 8, 16, 1)
     Wt = oracle.dequantize(qw)
     dq, da, Xd, dYd = qweight_to_dev(qw), adapter_to_dev(ad), to_bf16_dev(X), to_bf16_dev(dY)
