@@ -11,15 +11,17 @@ from tests._parity import gate_strict, qweight_to_dev, to_bf16_dev, to_np64
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("direction", ["fwd", "bwd"])
-def test_a_wait_that_runs_out_sets_the_status_word_and_the_kernel_returns(direction):
+@pytest.mark.parametrize("direction,T,d_out,d_in", [("fwd", 300, 512, 512), ("bwd", 300, 512, 512),
+                                                    ("fwd", 2100, 4864, 256), ("bwd", 2100, 256, 4864)])
+def test_a_wait_that_runs_out_sets_the_status_word_and_the_kernel_returns(direction, T, d_out, d_in):
     from paper_2407_17029_b200 import binding as qb
     # Two token tiles by two row tiles, eight K-blocks: the producers of every CTA leave out the copy of their
     # fourth K-block (the bytes are announced to the stage's barrier and never arrive).  With the wait limit set to
     # 2 * 10^6 cycles (about a millisecond) the MMA issuer, the dequant warps, the producers and the epilogue warps
     # each run into the limit, the pair frees its tensor memory and the kernel ends on its own: no trap, no fault,
     # no endless loop.  The call itself returns OK (the launch succeeded); the status word says what happened.
-    T, d_out, d_in = 300, 512, 512
+    # The two larger shapes (19 row tiles x 5 token tiles of 512, four K-blocks) run the 256 x 512 tile form of
+    # the kernel, with its four-stage ring and eight epilogue warps.
     W = synth.normal(81, "timeout/W", (d_out, d_in), 0.02)
     X = synth.round_to_bf16(synth.normal(81, "timeout/X", (T, d_in)))
     dY = synth.round_to_bf16(synth.normal(81, "timeout/dY", (T, d_out)))
