@@ -78,3 +78,33 @@ def test_tensor_core_path_against_general_path_on_random_shapes(seed, monkeypatc
             for name, got, want in (("dA", outs[0][2], ref[2]), ("dB", outs[0][3], ref[3])):
                 e = float((got - want).abs().max() / want.pow(2).mean().sqrt().clamp_min(1e-30))
                 assert e <= 1e-2, f"{what}: {name} max/rms {e:.3e}"
+
+
+@pytest.mark.parametrize("seed", range(3))
+def test_low_bit_product_against_general_path_on_random_shapes(seed, monkeypatch):
+    # the merged layer's product at every kind of token count: the one-token and K-outer decode kernels (1..16),
+    # the fused contraction with its offset-term K-blocks in both tile forms (17 and up)
+    from paper_2407_17029_b200 import binding as qb
+    dev = torch.device("cuda", 0)
+    rng = np.random.default_rng(2000 + seed)
+    gen = torch.Generator(device=dev).manual_seed(2000 + seed)
+    for case in range(40):
+        d_out, d_in = int(rng.integers(1, 120)) * 64, int(rng.integers(1, 60)) * 64
+        T = int(rng.choice([1, 2, 3, 5, 8, 9, 12, 16, 17, 40, 200, 257, 600, 1500, 2600]))
+        W = torch.randn(d_out, d_in, device=dev, generator=gen) * 0.02
+        dq = qb.quantize_blockwise(W, 64, 1, qb.FMT_AFFINE_MINMAX)
+        A = (torch.randn(d_in // 64, 64, device=dev, generator=gen) * 0.3).to(torch.bfloat16)
+        B = (torch.randn(64, d_out // 8, device=dev, generator=gen) * 0.3).to(torch.bfloat16)
+        merged = qb.merge(dq, qb.Adapter(64, 8, 64, float(rng.choice([1.0, 20.0])), A, B))
+        X = torch.randn(T, d_in, device=dev, generator=gen).to(torch.bfloat16)
+        monkeypatch.setenv("QBLORA_FORCE_GENERAL", "1")
+        ref = qb.lowbit_gemm(merged, X, torch.float32)
+        monkeypatch.delenv("QBLORA_FORCE_GENERAL")
+        ws = qb.alloc_workspace(qb.OP_LOWBIT_GEMM, merged, None, T)
+        Y1 = qb.lowbit_gemm(merged, X, torch.float32, ws=ws)
+        Y2 = qb.lowbit_gemm(merged, X, torch.float32, ws=ws)
+        what = f"seed {seed} case {case}: T={T} d_out={d_out} d_in={d_in}"
+        assert qb.device_status(ws) == qb.OK, what
+        assert torch.equal(Y1, Y2), what + " (second call differs from the first)"
+        mx, rm = _err(Y1, ref)
+        assert mx <= 3e-2 and rm <= 5e-3, f"{what}: max/row-rms {mx:.3e}, rms/rms {rm:.3e}"
